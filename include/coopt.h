@@ -1,0 +1,170 @@
+/*
+ * coopt.h — C ABI of the paged FP8 grouped-query attention library (libcoopt.so).
+ *
+ * One attention layer's hot path of LLM-CoOpt: the Opt-KV cache write (Algorithm 1,
+ * phase 1), the Opt-KV / Opt-GQA read (Algorithm 1 phase 2, Algorithm 2, Eq. 6-8) and the
+ * Opt-Pa valid-block / chunk-and-merge path (Algorithm 3, Eq. 9-10).  sm_100a only; there
+ * is no CPU fallback.
+ *
+ * General rules for every call
+ *   - Pointers marked DEVICE must point to memory of the current CUDA device; the caller
+ *     owns all of it.  The library allocates no device memory and never synchronises: work
+ *     is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the default stream).
+ *   - The return value is a coopt_status: 0 on success, negative after host-side argument
+ *     checks or a failed launch.  Nothing is thrown, nothing aborts.
+ *   - Problems seen on the device (a bounded wait that ran out) are reported in the first
+ *     int32 of the workspace (0 = none, otherwise a coopt_status); read it after the
+ *     stream has been synchronised.
+ *
+ * Cache layout (DEVICE memory, `coopt_cache.data`)
+ *   The cache is an array of granules, one per (physical block, kv head):
+ *       granule(blk, h) starts at byte (blk * num_kv_heads + h) * coopt_granule_bytes().
+ *   block_size is 16 tokens.  FP8 E4M3 cache (COOPT_KV_FP8_E4M3):
+ *       bytes  0..3   fp32 K scale of the granule     bytes 4..7  fp32 V scale
+ *       bytes  8..31  zero
+ *       bytes 32..32+16*D-1        K codes, 16 tokens x D, in tensor-core fragment order
+ *       bytes 32+16*D..32+32*D-1   V codes, 16 tokens x D, in tensor-core fragment order
+ *   A dequantised element is decode_e4m3(code) * scale (Eq. 6).  A scale of 0 marks a
+ *   granule that holds only zeros.  bf16 cache (COOPT_KV_BF16, the un-quantised ablation):
+ *   no header; 16*D bf16 K values then 16*D bf16 V values, also in fragment order.
+ *   "Fragment order" is a fixed permutation of (token, dim) inside the granule chosen so
+ *   that a warp reads the operands of its matrix instructions with 16-byte loads;
+ *   coopt_cache_offset() returns the byte offset of any element, which is all a caller
+ *   needs to inspect or build a cache by hand.
+ *   A cache that has never been written must be zero-filled once by the caller.
+ */
+#ifndef COOPT_H_
+#define COOPT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  COOPT_OK = 0,
+  COOPT_ERR_INVALID_ARG = -1, /* null pointer, negative size, inconsistent shapes       */
+  COOPT_ERR_UNSUPPORTED = -2, /* shape outside the compiled set (see each call)          */
+  COOPT_ERR_WORKSPACE = -3,   /* workspace missing or smaller than coopt_workspace_bytes */
+  COOPT_ERR_CUDA = -4,        /* a CUDA runtime call or the launch failed                */
+  COOPT_ERR_TIMEOUT = -5      /* device side: a bounded wait ran out (workspace word 0)  */
+} coopt_status;
+
+typedef enum { COOPT_KV_FP8_E4M3 = 0, COOPT_KV_BF16 = 1 } coopt_kv_dtype;
+
+typedef struct coopt_cache {
+  void* data;           /* DEVICE, coopt_cache_bytes() bytes, 32-byte aligned, layout above */
+  int32_t num_blocks;   /* physical blocks                                                 */
+  int32_t num_kv_heads; /* H_k of Eq. 7                                                    */
+  int32_t head_dim;     /* 64 or 128                                                       */
+  int32_t block_size;   /* must be 16                                                      */
+  int32_t dtype;        /* coopt_kv_dtype                                                  */
+} coopt_cache;
+
+/* Bytes of one (block, kv head) granule / of a whole cache; 0 for unsupported shapes. */
+size_t coopt_granule_bytes(int32_t head_dim, int32_t dtype);
+size_t coopt_cache_bytes(int32_t num_blocks, int32_t num_kv_heads, int32_t head_dim, int32_t dtype);
+
+/* Byte offset, from `data`, of element (block, kv_head, which, token, dim); which = 0 for K,
+ * 1 for V.  For the FP8 cache the granule's K (V) scale is at coopt_scale_offset(..., which).
+ * Pure host arithmetic (no CUDA call); returns -1 for arguments out of range. */
+int64_t coopt_cache_offset(const coopt_cache* cache, int32_t block, int32_t kv_head, int32_t which,
+                           int32_t token, int32_t dim);
+int64_t coopt_scale_offset(const coopt_cache* cache, int32_t block, int32_t kv_head, int32_t which);
+
+/*
+ * coopt_kv_write — Opt-KV write (Algorithm 1 phase 1; Eq. 5; Section 3.1 "compressing
+ * valid blocks into FP8").
+ *   k, v          DEVICE bf16 [num_tokens][num_kv_heads][head_dim]; consecutive tokens are
+ *                 kv_token_stride elements apart (>= num_kv_heads * head_dim)
+ *   slot_mapping  DEVICE int64 [num_tokens]; slot = block * 16 + offset.  A negative slot
+ *                 skips the token (Eq. 5; the caller expresses SkipSet membership this way).
+ * FP8 semantics, per group of the call's tokens that land in one block, per kv head and
+ * for K and V separately: amax = largest |value| of the group; a group that writes offset 0
+ * opens the block anew (old scale ignored, all other slots cleared to code 0); otherwise
+ * s_old is the granule's scale.  s_new = max(s_old, amax / 448).  If s_new > s_old > 0 the
+ * codes already in the granule are re-expressed: enc((dec(code) * s_old) / s_new).  New
+ * values are stored as enc(x / s_new).  All of this in IEEE fp32; enc is round-to-nearest-
+ * even with saturation to +-448.  bf16 cache: values are stored unchanged.
+ * Preconditions (not checked): inputs finite; the non-skipped tokens of one call that land
+ * in the same block are consecutive in the call (skipped tokens may sit between them) and
+ * have distinct offsets; no other work touches those blocks concurrently.  Tokens whose
+ * block index is >= num_blocks are ignored.
+ * Errors: INVALID_ARG (null pointers, num_tokens < 0, stride too small), UNSUPPORTED
+ * (head_dim not 64/128, block_size != 16, unknown dtype), CUDA.  num_tokens == 0 is a no-op.
+ */
+int coopt_kv_write(const coopt_cache* cache, const void* k, const void* v, int64_t kv_token_stride,
+                   const int64_t* slot_mapping, int32_t num_tokens, void* stream);
+
+/*
+ * coopt_paged_decode — one new query token per sequence attends over its paged cache
+ * (Eq. 1; Eq. 6 dequantisation on load; Eq. 7-8 grouped-query sharing: query head i reads
+ * kv head floor(i / (num_q_heads / num_kv_heads)); Eq. 9: only blocks 0..ceil(len/16)-1 of a
+ * sequence are read and the last one is masked past len; Eq. 10 max-subtracted softmax).
+ *   q, out        DEVICE bf16 [batch][num_q_heads][head_dim], contiguous
+ *   block_table   DEVICE int32 [batch][max_blocks_per_seq]; entry j of row b is the physical
+ *                 block of tokens 16j..16j+15 of sequence b; entries past the context are
+ *                 never read
+ *   context_lens  DEVICE int32 [batch]; 0 gives an all-zero output row
+ *   sm_scale      logit scale, normally 1/sqrt(head_dim)
+ *   workspace     DEVICE, >= coopt_workspace_bytes(...) with chunk_size = 0, prepared once by
+ *                 coopt_workspace_init(); reusable by later calls on the same stream
+ * The context of every (sequence, kv head) is cut into byte-balanced pieces across the SMs;
+ * pieces are merged by a log-sum-exp reduction inside the same launch.
+ * Errors: INVALID_ARG, UNSUPPORTED (group size num_q_heads/num_kv_heads not in 1..8 or not
+ * integral, batch > 1024, head_dim/block_size/dtype as above), WORKSPACE, CUDA.
+ */
+int coopt_paged_decode(const coopt_cache* cache, const void* q, void* out, const int32_t* block_table,
+                       int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch,
+                       int32_t num_q_heads, float sm_scale, void* workspace, size_t workspace_bytes,
+                       void* stream);
+
+/*
+ * coopt_paged_chunked — Opt-Pa long-sequence path (abstract and conclusion: the context is
+ * segmented into chunks that are processed independently and merged) and chunked prefill.
+ *   cu_q_lens     DEVICE int32 [batch + 1], prefix sums of the number of query tokens per
+ *                 sequence; q/out are bf16 [cu_q_lens[batch]][num_q_heads][head_dim]
+ *   context_lens  include the new tokens; the n query tokens of a sequence are its last n
+ *                 positions and, when causal != 0, query i sees positions 0..len-n+i
+ *   chunk_size    tokens per chunk, a multiple of 16, at most 32768
+ *   total_q       cu_q_lens[batch] as known by the host (sizes the launch)
+ * When every sequence has exactly one query token (total_q == batch) each chunk c of
+ * (sequence b, query head h) produces m_c (max logit, natural-log units after sm_scale),
+ * l_c (sum of exp(logit - m_c)) and o_c (softmax-weighted V inside the chunk, fp32), stored
+ * in the workspace where coopt_chunk_partials() points, and the chunks are merged with
+ * weights l_c * exp(m_c - max_c m_c).  With longer query runs (chunked prefill) the tiles
+ * run on tensor cores and no partials are exported.
+ * Errors: as coopt_paged_decode, plus INVALID_ARG for a bad chunk_size.
+ */
+int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, const int32_t* cu_q_lens,
+                        const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
+                        int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t chunk_size, int32_t causal,
+                        float sm_scale, void* workspace, size_t workspace_bytes, void* stream);
+
+/* Workspace size for a call with these arguments (chunk_size = 0 for coopt_paged_decode).
+ * Host arithmetic only (it asks the current device for its SM count once). */
+size_t coopt_workspace_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                             int32_t max_blocks_per_seq, int32_t chunk_size, int32_t total_q);
+
+/* Zero the control words of a freshly allocated workspace (enqueued on `stream`).  Needed
+ * once; every call leaves the workspace ready for the next.  Call it again after a call
+ * reported a device-side error. */
+int coopt_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
+
+/* Where a q_len == 1 coopt_paged_chunked call leaves its per-chunk partials: byte offsets
+ * from `workspace` of o_c fp32 [batch][num_q_heads][max_chunks][head_dim] and of m_c and l_c,
+ * both fp32 [batch][num_q_heads][max_chunks], max_chunks = ceil(max_blocks_per_seq * 16 /
+ * chunk_size).  Host arithmetic only. */
+int coopt_chunk_partials(int32_t batch, int32_t num_q_heads, int32_t head_dim, int32_t max_blocks_per_seq,
+                         int32_t chunk_size, size_t* o_offset, size_t* m_offset, size_t* l_offset,
+                         int32_t* max_chunks);
+
+const char* coopt_status_string(int status);
+int coopt_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* COOPT_H_ */

@@ -1,0 +1,199 @@
+"""Thin ctypes binding of ``libcoopt.so``: argument marshalling only.
+
+Every function has the name of the C entry point it wraps (without the ``coopt_`` prefix is
+also exported for convenience).  Tensors are torch CUDA tensors; their ``data_ptr()`` and the
+current torch stream are passed through.  Nothing is computed here, and there is no fallback:
+if the shared library is missing or a call returns an error status, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+import torch
+
+KV_FP8_E4M3 = 0
+KV_BF16 = 1
+BLOCK_SIZE = 16
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcoopt.so")
+_lib: Optional[ctypes.CDLL] = None
+
+
+class CooptError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: status {status} ({status_string(status)})")
+
+
+class coopt_cache(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("num_blocks", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("block_size", ctypes.c_int32), ("dtype", ctypes.c_int32)]
+
+
+_SIGNATURES = {
+    "coopt_granule_bytes": (ctypes.c_size_t, [ctypes.c_int32, ctypes.c_int32]),
+    "coopt_cache_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 4),
+    "coopt_cache_offset": (ctypes.c_int64, [ctypes.POINTER(coopt_cache)] + [ctypes.c_int32] * 5),
+    "coopt_scale_offset": (ctypes.c_int64, [ctypes.POINTER(coopt_cache)] + [ctypes.c_int32] * 3),
+    "coopt_kv_write": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                      ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p]),
+    "coopt_paged_decode": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p,
+                                          ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32,
+                                          ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
+                                          ctypes.c_void_p]),
+    "coopt_paged_chunked": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p,
+                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
+                                           ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
+                                           ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
+                                           ctypes.c_void_p]),
+    "coopt_workspace_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 7),
+    "coopt_workspace_init": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "coopt_chunk_partials": (ctypes.c_int, [ctypes.c_int32] * 5 + [ctypes.POINTER(ctypes.c_size_t)] * 3
+                             + [ctypes.POINTER(ctypes.c_int32)]),
+    "coopt_status_string": (ctypes.c_char_p, [ctypes.c_int]),
+    "coopt_version": (ctypes.c_int, []),
+}
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library() -> ctypes.CDLL:
+    """dlopen ``libcoopt.so`` (built by ``paper_2602_09323_b200.build``) and type its symbols."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: run `python -m paper_2602_09323_b200.build` "
+                               "(there is no CPU fallback)")
+        lib = ctypes.CDLL(_LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(lib, name)
+            fn.restype, fn.argtypes = res, args
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load_library().coopt_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str) -> None:
+    if status != 0:
+        raise CooptError(status, what)
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t: torch.Tensor) -> ctypes.c_void_p:
+    return ctypes.c_void_p(t.data_ptr())
+
+
+class Cache:
+    """A paged KV cache in device memory plus the C descriptor that names it."""
+
+    def __init__(self, num_blocks: int, num_kv_heads: int, head_dim: int, dtype: int = KV_FP8_E4M3,
+                 device: str = "cuda"):
+        lib = load_library()
+        nbytes = lib.coopt_cache_bytes(num_blocks, num_kv_heads, head_dim, dtype)
+        if nbytes == 0:
+            raise CooptError(-2, "coopt_cache_bytes")
+        self.data = torch.zeros(nbytes, dtype=torch.uint8, device=device)
+        self.num_blocks, self.num_kv_heads, self.head_dim, self.dtype = num_blocks, num_kv_heads, head_dim, dtype
+        self.granule_bytes = lib.coopt_granule_bytes(head_dim, dtype)
+        self.desc = coopt_cache(self.data.data_ptr(), num_blocks, num_kv_heads, head_dim, BLOCK_SIZE, dtype)
+
+    def ref(self):
+        return ctypes.byref(self.desc)
+
+
+def cache_offset(cache: Cache, block: int, kv_head: int, which: int, token: int, dim: int) -> int:
+    return load_library().coopt_cache_offset(cache.ref(), block, kv_head, which, token, dim)
+
+
+def scale_offset(cache: Cache, block: int, kv_head: int, which: int) -> int:
+    return load_library().coopt_scale_offset(cache.ref(), block, kv_head, which)
+
+
+def kv_write(cache: Cache, k: torch.Tensor, v: torch.Tensor, slot_mapping: torch.Tensor) -> None:
+    """coopt_kv_write: k, v bf16 [T, Hkv, D] (token stride taken from the tensor), slots int64 [T]."""
+    assert k.dtype == torch.bfloat16 and v.dtype == torch.bfloat16 and slot_mapping.dtype == torch.int64
+    assert k.is_cuda and v.is_cuda and slot_mapping.is_cuda and slot_mapping.is_contiguous()
+    assert k.shape == v.shape and k.stride() == v.stride() and k.stride(2) == 1 and k.stride(1) == k.shape[2]
+    st = load_library().coopt_kv_write(cache.ref(), _ptr(k), _ptr(v), k.stride(0) if k.shape[0] > 1 else k.shape[1] * k.shape[2],
+                                       _ptr(slot_mapping), k.shape[0], _stream())
+    _check(st, "coopt_kv_write")
+
+
+def workspace_bytes(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, max_blocks_per_seq: int,
+                    chunk_size: int = 0, total_q: Optional[int] = None) -> int:
+    return load_library().coopt_workspace_bytes(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq,
+                                                chunk_size, batch if total_q is None else total_q)
+
+
+def workspace_init(workspace: torch.Tensor) -> None:
+    _check(load_library().coopt_workspace_init(_ptr(workspace), workspace.numel(), _stream()), "coopt_workspace_init")
+
+
+def new_workspace(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, max_blocks_per_seq: int,
+                  chunk_size: int = 0, total_q: Optional[int] = None, device: str = "cuda") -> torch.Tensor:
+    """Allocate (torch) and initialise a workspace large enough for the given call."""
+    n = workspace_bytes(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq, chunk_size, total_q)
+    ws = torch.empty(n, dtype=torch.uint8, device=device)
+    workspace_init(ws)
+    return ws
+
+
+def workspace_status(workspace: torch.Tensor) -> int:
+    """Device-side status word (synchronises)."""
+    return int(workspace[:4].view(torch.int32).item())
+
+
+def paged_decode(cache: Cache, q: torch.Tensor, block_table: torch.Tensor, context_lens: torch.Tensor,
+                 sm_scale: float, workspace: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """coopt_paged_decode: q bf16 [B, Hq, D] -> out bf16 [B, Hq, D]."""
+    assert q.dtype == torch.bfloat16 and q.is_contiguous() and q.is_cuda
+    assert block_table.dtype == torch.int32 and block_table.is_contiguous() and context_lens.dtype == torch.int32
+    if out is None:
+        out = torch.empty_like(q)
+    st = load_library().coopt_paged_decode(cache.ref(), _ptr(q), _ptr(out), _ptr(block_table), block_table.shape[1],
+                                           _ptr(context_lens), q.shape[0], q.shape[1], float(sm_scale),
+                                           _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "coopt_paged_decode")
+    return out
+
+
+def paged_chunked(cache: Cache, q: torch.Tensor, cu_q_lens: torch.Tensor, block_table: torch.Tensor,
+                  context_lens: torch.Tensor, chunk_size: int, causal: bool, sm_scale: float,
+                  workspace: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """coopt_paged_chunked: q bf16 [total_q, Hq, D]; cu_q_lens int32 [B + 1] on the device."""
+    assert q.dtype == torch.bfloat16 and q.is_contiguous() and q.is_cuda
+    assert block_table.dtype == torch.int32 and block_table.is_contiguous()
+    assert cu_q_lens.dtype == torch.int32 and context_lens.dtype == torch.int32
+    if out is None:
+        out = torch.empty_like(q)
+    batch = context_lens.shape[0]
+    st = load_library().coopt_paged_chunked(cache.ref(), _ptr(q), _ptr(out), _ptr(cu_q_lens), _ptr(block_table),
+                                            block_table.shape[1], _ptr(context_lens), batch, q.shape[1], q.shape[0],
+                                            int(chunk_size), int(bool(causal)), float(sm_scale), _ptr(workspace),
+                                            workspace.numel(), _stream())
+    _check(st, "coopt_paged_chunked")
+    return out
+
+
+def chunk_partials(workspace: torch.Tensor, batch: int, num_q_heads: int, head_dim: int, max_blocks_per_seq: int,
+                   chunk_size: int):
+    """Views (o_c, m_c, l_c) of the per-chunk partials a q_len == 1 chunked call left in the workspace."""
+    o, m, l = ctypes.c_size_t(), ctypes.c_size_t(), ctypes.c_size_t()
+    mc = ctypes.c_int32()
+    _check(load_library().coopt_chunk_partials(batch, num_q_heads, head_dim, max_blocks_per_seq, chunk_size,
+                                               ctypes.byref(o), ctypes.byref(m), ctypes.byref(l), ctypes.byref(mc)),
+           "coopt_chunk_partials")
+    rows = batch * num_q_heads * mc.value
+    f = lambda off, n: workspace[off:off + 4 * n].view(torch.float32)
+    return (f(o.value, rows * head_dim).view(batch, num_q_heads, mc.value, head_dim),
+            f(m.value, rows).view(batch, num_q_heads, mc.value), f(l.value, rows).view(batch, num_q_heads, mc.value))

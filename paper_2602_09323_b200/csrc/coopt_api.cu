@@ -1,0 +1,207 @@
+// Host side of the C ABI: argument checks, workspace arithmetic, dispatch to the launchers.
+#include <mutex>
+
+#include "coopt_common.cuh"
+
+namespace coopt {
+
+int launch_kv_write(const coopt_cache* c, const void* k, const void* v, int64_t stride, const int64_t* slots,
+                    int num_tokens, cudaStream_t stream);
+int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
+                        int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                        float sm_scale, int32_t chunk_size, void* workspace, int planned_ctas, cudaStream_t stream);
+int launch_paged_prefill(const coopt_cache* c, const void* q, void* out, const int32_t* cu_q_lens,
+                         const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
+                         int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t causal, float sm_scale,
+                         void* workspace, cudaStream_t stream);
+size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int batch, int num_q_heads, int max_chunks);
+size_t workspace_control_bytes();
+int decode_planned_ctas(int num_sms, long long upper_blocks);
+int decode_max_batch();
+int decode_counter_slots();
+int decode_max_chunk_blocks();
+void chunk_partial_offsets(int batch, int num_q_heads, int head_dim, int max_chunks, size_t* o, size_t* m, size_t* l);
+
+const DeviceInfo* device_info() {
+  static DeviceInfo info[64];
+  static bool known[64] = {};
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!known[dev]) {
+    int sms = 0, smem = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) return nullptr;
+    info[dev].num_sms = sms;
+    info[dev].max_smem_optin = smem;
+    known[dev] = true;
+  }
+  return &info[dev];
+}
+
+namespace {
+
+bool cache_shape_ok(int head_dim, int block_size, int dtype) {
+  return (head_dim == 64 || head_dim == 128) && block_size == kBlockSize &&
+         (dtype == COOPT_KV_FP8_E4M3 || dtype == COOPT_KV_BF16);
+}
+
+int check_cache(const coopt_cache* c) {
+  if (c == nullptr || c->data == nullptr || c->num_blocks <= 0 || c->num_kv_heads <= 0) return COOPT_ERR_INVALID_ARG;
+  if (!cache_shape_ok(c->head_dim, c->block_size, c->dtype)) return COOPT_ERR_UNSUPPORTED;
+  if (reinterpret_cast<uintptr_t>(c->data) % 32 != 0) return COOPT_ERR_INVALID_ARG;
+  return COOPT_OK;
+}
+
+int max_chunks_of(int max_blocks_per_seq, int chunk_size) {
+  return static_cast<int>((static_cast<long long>(max_blocks_per_seq) * kBlockSize + chunk_size - 1) / chunk_size);
+}
+
+// number of CTAs planned for a decode-style launch; the same on the sizing and the launching side
+int planned_ctas(int batch, int num_kv_heads, int max_blocks_per_seq) {
+  const DeviceInfo* di = device_info();
+  const int sms = di ? di->num_sms : 148;
+  return decode_planned_ctas(sms, static_cast<long long>(batch) * num_kv_heads * max_blocks_per_seq);
+}
+
+int check_attention_args(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
+                         int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads) {
+  const int rc = check_cache(c);
+  if (rc != COOPT_OK) return rc;
+  if (!q || !out || !block_table || !context_lens || batch < 0 || max_blocks_per_seq <= 0 || num_q_heads <= 0)
+    return COOPT_ERR_INVALID_ARG;
+  if (num_q_heads % c->num_kv_heads != 0) return COOPT_ERR_UNSUPPORTED;
+  const int group = num_q_heads / c->num_kv_heads;
+  if (group < 1 || group > 8) return COOPT_ERR_UNSUPPORTED;
+  if (batch > decode_max_batch() || static_cast<long long>(batch) * c->num_kv_heads > decode_counter_slots())
+    return COOPT_ERR_UNSUPPORTED;
+  return COOPT_OK;
+}
+
+}  // namespace
+}  // namespace coopt
+
+using namespace coopt;
+
+extern "C" {
+
+size_t coopt_granule_bytes(int32_t head_dim, int32_t dtype) {
+  if (!cache_shape_ok(head_dim, kBlockSize, dtype)) return 0;
+  return granule_bytes(head_dim, dtype == COOPT_KV_FP8_E4M3);
+}
+
+size_t coopt_cache_bytes(int32_t num_blocks, int32_t num_kv_heads, int32_t head_dim, int32_t dtype) {
+  if (num_blocks <= 0 || num_kv_heads <= 0) return 0;
+  return static_cast<size_t>(num_blocks) * num_kv_heads * coopt_granule_bytes(head_dim, dtype);
+}
+
+int64_t coopt_cache_offset(const coopt_cache* c, int32_t block, int32_t kv_head, int32_t which, int32_t token,
+                           int32_t dim) {
+  if (!c || !cache_shape_ok(c->head_dim, c->block_size, c->dtype)) return -1;
+  if (block < 0 || block >= c->num_blocks || kv_head < 0 || kv_head >= c->num_kv_heads || which < 0 || which > 1 ||
+      token < 0 || token >= kBlockSize || dim < 0 || dim >= c->head_dim)
+    return -1;
+  const bool fp8 = c->dtype == COOPT_KV_FP8_E4M3;
+  const int64_t gran = (static_cast<int64_t>(block) * c->num_kv_heads + kv_head) * granule_bytes(c->head_dim, fp8);
+  const int inner = which == 0 ? k_elem_offset(c->head_dim, fp8, token, dim) : v_elem_offset(c->head_dim, fp8, token, dim);
+  return gran + part_offset(c->head_dim, fp8, which) + inner;
+}
+
+int64_t coopt_scale_offset(const coopt_cache* c, int32_t block, int32_t kv_head, int32_t which) {
+  if (!c || !cache_shape_ok(c->head_dim, c->block_size, c->dtype) || c->dtype != COOPT_KV_FP8_E4M3) return -1;
+  if (block < 0 || block >= c->num_blocks || kv_head < 0 || kv_head >= c->num_kv_heads || which < 0 || which > 1) return -1;
+  return (static_cast<int64_t>(block) * c->num_kv_heads + kv_head) * granule_bytes(c->head_dim, true) + 4 * which;
+}
+
+int coopt_kv_write(const coopt_cache* cache, const void* k, const void* v, int64_t kv_token_stride,
+                   const int64_t* slot_mapping, int32_t num_tokens, void* stream) {
+  const int rc = check_cache(cache);
+  if (rc != COOPT_OK) return rc;
+  if (num_tokens < 0) return COOPT_ERR_INVALID_ARG;
+  if (num_tokens == 0) return COOPT_OK;
+  if (!k || !v || !slot_mapping) return COOPT_ERR_INVALID_ARG;
+  if (kv_token_stride < static_cast<int64_t>(cache->num_kv_heads) * cache->head_dim) return COOPT_ERR_INVALID_ARG;
+  return launch_kv_write(cache, k, v, kv_token_stride, slot_mapping, num_tokens, static_cast<cudaStream_t>(stream));
+}
+
+size_t coopt_workspace_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                             int32_t max_blocks_per_seq, int32_t chunk_size, int32_t total_q) {
+  (void)total_q;
+  if (batch < 0 || num_q_heads <= 0 || num_kv_heads <= 0 || max_blocks_per_seq <= 0 || chunk_size < 0) return 0;
+  const int group = (num_q_heads + num_kv_heads - 1) / num_kv_heads;
+  const int P = planned_ctas(batch, num_kv_heads, max_blocks_per_seq);
+  const int mc = chunk_size > 0 ? max_chunks_of(max_blocks_per_seq, chunk_size) : 0;
+  return decode_workspace_bytes(P, group, head_dim, batch, num_q_heads, mc);
+}
+
+int coopt_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+  if (!workspace) return COOPT_ERR_INVALID_ARG;
+  if (workspace_bytes < workspace_control_bytes()) return COOPT_ERR_WORKSPACE;
+  return cudaMemsetAsync(workspace, 0, workspace_control_bytes(), static_cast<cudaStream_t>(stream)) == cudaSuccess
+             ? COOPT_OK
+             : COOPT_ERR_CUDA;
+}
+
+int coopt_chunk_partials(int32_t batch, int32_t num_q_heads, int32_t head_dim, int32_t max_blocks_per_seq,
+                         int32_t chunk_size, size_t* o_offset, size_t* m_offset, size_t* l_offset, int32_t* max_chunks) {
+  if (batch < 0 || num_q_heads <= 0 || head_dim <= 0 || max_blocks_per_seq <= 0 || chunk_size <= 0 ||
+      chunk_size % kBlockSize != 0 || !o_offset || !m_offset || !l_offset || !max_chunks)
+    return COOPT_ERR_INVALID_ARG;
+  *max_chunks = max_chunks_of(max_blocks_per_seq, chunk_size);
+  chunk_partial_offsets(batch, num_q_heads, head_dim, *max_chunks, o_offset, m_offset, l_offset);
+  return COOPT_OK;
+}
+
+int coopt_paged_decode(const coopt_cache* cache, const void* q, void* out, const int32_t* block_table,
+                       int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                       float sm_scale, void* workspace, size_t workspace_bytes, void* stream) {
+  const int rc = check_attention_args(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads);
+  if (rc != COOPT_OK) return rc;
+  if (batch == 0) return COOPT_OK;
+  if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, cache->num_kv_heads, cache->head_dim,
+                                                            max_blocks_per_seq, 0, batch))
+    return COOPT_ERR_WORKSPACE;
+  const int P = planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq);
+  return launch_paged_decode(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads, sm_scale,
+                             0, workspace, P, static_cast<cudaStream_t>(stream));
+}
+
+int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, const int32_t* cu_q_lens,
+                        const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
+                        int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t chunk_size, int32_t causal,
+                        float sm_scale, void* workspace, size_t workspace_bytes, void* stream) {
+  const int rc = check_attention_args(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads);
+  if (rc != COOPT_OK) return rc;
+  if (!cu_q_lens || total_q < batch) return COOPT_ERR_INVALID_ARG;
+  if (chunk_size <= 0 || chunk_size % kBlockSize != 0 || chunk_size / kBlockSize > decode_max_chunk_blocks())
+    return COOPT_ERR_INVALID_ARG;
+  if (batch == 0) return COOPT_OK;
+  if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, cache->num_kv_heads, cache->head_dim,
+                                                            max_blocks_per_seq, chunk_size, total_q))
+    return COOPT_ERR_WORKSPACE;
+  if (total_q == batch) {
+    // one query token per sequence: the Opt-Pa chunk-and-merge decode
+    const int P = planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq);
+    return launch_paged_decode(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads,
+                               sm_scale, chunk_size, workspace, P, static_cast<cudaStream_t>(stream));
+  }
+  return launch_paged_prefill(cache, q, out, cu_q_lens, block_table, max_blocks_per_seq, context_lens, batch,
+                              num_q_heads, total_q, causal, sm_scale, workspace, static_cast<cudaStream_t>(stream));
+}
+
+const char* coopt_status_string(int status) {
+  switch (status) {
+    case COOPT_OK: return "ok";
+    case COOPT_ERR_INVALID_ARG: return "invalid argument";
+    case COOPT_ERR_UNSUPPORTED: return "unsupported shape";
+    case COOPT_ERR_WORKSPACE: return "workspace missing or too small";
+    case COOPT_ERR_CUDA: return "CUDA runtime error";
+    case COOPT_ERR_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown status";
+  }
+}
+
+int coopt_version(void) { return 100; }
+
+}  // extern "C"

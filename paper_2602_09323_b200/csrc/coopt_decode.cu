@@ -1,0 +1,678 @@
+// Paged GQA decode over the FP8 (or bf16) cache: Algorithm 1 phase 2 (Eq. 6 dequantisation on
+// load), Algorithm 2 (Eq. 7-8: the G query heads of a group consume one K/V stream),
+// Algorithm 3 (Eq. 9 valid blocks only, Eq. 10 max-subtracted softmax) and the Opt-Pa
+// chunk-and-merge reduction.
+//
+// Work decomposition.  All (sequence, kv head, block) triples form one flat list.  In decode
+// mode CTA i takes the i-th of P equal slices of that list (split-KV balanced by bytes); in
+// chunk mode it takes a contiguous run of fixed-size chunks.  A slice is cut into segments at
+// (sequence, kv head) boundaries (and chunk boundaries).  Inside a segment the CTA's warps take
+// blocks round-robin; each warp streams its granules through a private ring of shared-memory
+// stages filled by bulk async copies (one elected lane issues, an mbarrier per stage counts the
+// bytes), runs both contractions on mma.sync with the G query heads padded to the 16 rows of
+// the instruction, and keeps an online softmax per query head (warp shuffles inside the quad
+// that owns a head, one shared-memory step across warps at the end of the segment).  A segment
+// that does not cover its whole sequence leaves (m, l, o) in the workspace; the CTA that
+// delivers the last piece of a (sequence, kv head) merges them by log-sum-exp and writes the
+// bf16 output.  The K scale of a granule factors out of the dot product and is applied to the
+// logits; the V scale is folded into the probabilities.
+#include "coopt_common.cuh"
+
+namespace coopt {
+
+namespace {
+
+constexpr int kWarps = 8;
+constexpr int kThreads = kWarps * 32;
+constexpr int kCap = 2048;            // block ids staged in shared memory per round
+constexpr int kMaxSeg = 32;           // segments planned per round
+constexpr int kMaxBatch = 1024;
+constexpr int kMinBlocksPerCta = 16;
+constexpr int kMaxGroup = 8;
+constexpr int kCounterSlots = 16384;
+constexpr int kWsHeaderBytes = 256;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+struct Segment {
+  int b, g;          // sequence, kv head
+  int j0, n;         // first block of the sequence in this segment, number of blocks
+  int list_off;      // position of block j0 in the staged id list
+  int partial;       // 0: covers the whole sequence, write the output directly
+  int slot;          // partial: workspace slot (decode mode) or chunk index (chunk mode)
+  int expected;      // partial: number of pieces the (sequence, kv head) is cut into
+  int seq_blocks;    // blocks of the whole sequence
+  int ctx_len;       // tokens of the whole sequence
+};
+
+struct DecodeParams {
+  const uint8_t* cache;
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  const int* block_table;
+  const int* context_lens;
+  int max_blocks_per_seq;
+  int batch, num_q_heads, num_kv_heads, group;
+  int num_blocks;
+  float sm_scale_log2;     // sm_scale * log2(e)
+  int planned_ctas;        // P
+  int chunk_blocks;        // 0 = decode mode
+  int max_chunks;
+  int* status;
+  int* counters;
+  float* part_o;           // decode: [2P][G][D]        chunk: [B][Hq][max_chunks][D]
+  float* part_m;           // decode: [2P][G]           chunk: [B][Hq][max_chunks]
+  float* part_l;
+};
+
+template <int D, bool FP8>
+struct Cfg {
+  static constexpr int kGran = granule_bytes(D, FP8);
+  static constexpr int kStages = FP8 ? 4 : 2;
+  static constexpr int kKSteps = D / 16;
+  static constexpr int kNTiles = D / 8;
+  static constexpr int kOAcc = FP8 ? 2 : 4;     // accumulator registers kept per n-tile
+  // shared memory carve-up (bytes)
+  static constexpr int kRingOff = 0;
+  static constexpr int kRingBytes = kWarps * kStages * kGran;
+  static constexpr int kBarOff = kRingOff + kRingBytes;
+  static constexpr int kIdsOff = kBarOff + kWarps * kStages * 8;
+  static constexpr int kPreBlkOff = kIdsOff + kCap * 4;
+  static constexpr int kPreUnitOff = kPreBlkOff + (kMaxBatch + 4) * 4;
+  static constexpr int kSegOff = kPreUnitOff + (kMaxBatch + 4) * 4;
+  static constexpr int kMergeOff = kSegOff + kMaxSeg * static_cast<int>(sizeof(Segment));
+  static constexpr int kMergeStride = D + 4;    // floats per (warp, row): o[D], m, l, pad
+  static constexpr int kMiscOff = kMergeOff + kWarps * kMaxGroup * kMergeStride * 4;
+  static constexpr int kSmemBytes = kMiscOff + 64;
+};
+
+__device__ __forceinline__ float quad_max(float x) {
+  x = fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 1));
+  return fmaxf(x, __shfl_xor_sync(0xffffffffu, x, 2));
+}
+__device__ __forceinline__ float quad_sum(float x) {
+  x += __shfl_xor_sync(0xffffffffu, x, 1);
+  return x + __shfl_xor_sync(0xffffffffu, x, 2);
+}
+
+// mma with only the top 8 rows of A in use (rows 8..15 are zero): two live accumulators.
+template <bool F16>
+__device__ __forceinline__ void mma_top(float& d0, float& d1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
+  float t2, t3;
+  if constexpr (F16) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
+                 : "+f"(d0), "+f"(d1), "=f"(t2), "=f"(t3)
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.0f));
+  } else {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
+                 : "+f"(d0), "+f"(d1), "=f"(t2), "=f"(t3)
+                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.0f));
+  }
+}
+
+// Position of a flat block index in (sequence, kv head, block) order.
+struct Cursor {
+  int b, g, j;
+};
+
+__device__ __forceinline__ int find_seq(const int* pre, int batch, long long x, int heads) {
+  // largest b in [0, batch) with heads * pre[b] <= x
+  int lo = 0, hi = batch - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (static_cast<long long>(heads) * pre[mid] <= x) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+template <int D, bool FP8>
+__global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeParams p) {
+  using C = Cfg<D, FP8>;
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* ring = smem + C::kRingOff;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
+  int* ids = reinterpret_cast<int*>(smem + C::kIdsOff);
+  int* pre_blk = reinterpret_cast<int*>(smem + C::kPreBlkOff);
+  int* pre_unit = reinterpret_cast<int*>(smem + C::kPreUnitOff);
+  Segment* segs = reinterpret_cast<Segment*>(smem + C::kSegOff);
+  float* merge = reinterpret_cast<float*>(smem + C::kMergeOff);
+  int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] nseg, [1..2] next x, [3] last-arriver flag
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int row = lane >> 2, quad = lane & 3;
+  const int B = p.batch, Hkv = p.num_kv_heads, G = p.group, Hq = p.num_q_heads;
+  const bool chunk_mode = p.chunk_blocks > 0;
+
+  // ---- plan: blocks (and chunks) per sequence, prefix sums ------------------------------------
+  for (int b = tid; b < B; b += kThreads) {
+    int L = p.context_lens[b];
+    L = max(0, min(L, p.max_blocks_per_seq * kBlockSize));
+    const int nb = (L + kBlockSize - 1) / kBlockSize;
+    pre_blk[b + 1] = nb;
+    pre_unit[b + 1] = chunk_mode ? (nb + p.chunk_blocks - 1) / p.chunk_blocks : 0;
+  }
+  if (tid == 0) { pre_blk[0] = 0; pre_unit[0] = 0; }
+  __syncthreads();
+  if (warp == 0) {
+    int carry_b = 0, carry_u = 0;
+    for (int base = 0; base < B; base += 32) {
+      const int i = base + lane;
+      int vb = i < B ? pre_blk[i + 1] : 0, vu = i < B ? pre_unit[i + 1] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int tb = __shfl_up_sync(0xffffffffu, vb, o), tu = __shfl_up_sync(0xffffffffu, vu, o);
+        if (lane >= o) { vb += tb; vu += tu; }
+      }
+      if (i < B) { pre_blk[i + 1] = vb + carry_b; pre_unit[i + 1] = vu + carry_u; }
+      carry_b += __shfl_sync(0xffffffffu, vb, 31);
+      carry_u += __shfl_sync(0xffffffffu, vu, 31);
+    }
+  }
+  if (tid == 0) {
+    for (int i = 0; i < kWarps * C::kStages; ++i) mbar_init(&bars[i], 1);
+    mbar_fence_init();
+  }
+  __syncthreads();
+
+  // sequences with an empty context: all-zero output rows
+  for (int b = blockIdx.x; b < B; b += gridDim.x) {
+    if (pre_blk[b + 1] == pre_blk[b])
+      for (int i = tid; i < Hq * D; i += kThreads) p.out[static_cast<size_t>(b) * Hq * D + i] = __float2bfloat16(0.0f);
+  }
+
+  const long long N = static_cast<long long>(Hkv) * pre_blk[B];
+  if (N == 0) return;
+  long long lo, hi;
+  int P;
+  if (!chunk_mode) {
+    P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), max(1ll, N / kMinBlocksPerCta)));
+    if (static_cast<int>(blockIdx.x) >= P) return;
+    lo = blockIdx.x * N / P;
+    hi = (blockIdx.x + 1ll) * N / P;
+  } else {
+    const long long U = static_cast<long long>(Hkv) * pre_unit[B];
+    P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), U));
+    if (static_cast<int>(blockIdx.x) >= P) return;
+    const long long ulo = blockIdx.x * U / P, uhi = (blockIdx.x + 1ll) * U / P;
+    auto unit_to_block = [&](long long u) -> long long {
+      if (u >= U) return N;
+      const int b = find_seq(pre_unit, B, u, Hkv);
+      const int nch = pre_unit[b + 1] - pre_unit[b], nb = pre_blk[b + 1] - pre_blk[b];
+      const long long rem = u - static_cast<long long>(Hkv) * pre_unit[b];
+      const int g = static_cast<int>(rem / nch), c = static_cast<int>(rem % nch);
+      return static_cast<long long>(Hkv) * pre_blk[b] + static_cast<long long>(g) * nb + static_cast<long long>(c) * p.chunk_blocks;
+    };
+    lo = unit_to_block(ulo);
+    hi = unit_to_block(uhi);
+  }
+  auto cta_of = [&](long long x) -> int { return static_cast<int>(((x + 1) * P - 1) / N); };
+
+  // ---- per-warp pipeline state (persists across rounds) ----------------------------------------
+  uint8_t* my_ring = ring + warp * C::kStages * C::kGran;
+  uint64_t* my_bars = bars + warp * C::kStages;
+  uint32_t issued = 0, consumed = 0;
+  bool dead = false;   // a bounded wait ran out: stop touching the pipeline, keep the barriers' company
+
+  long long x = lo;
+  while (x < hi) {
+    // ---- round: thread 0 plans up to kMaxSeg segments / kCap blocks starting at x -------------
+    if (tid == 0) {
+      int nseg = 0, used = 0;
+      long long xx = x;
+      Cursor cur;
+      cur.b = find_seq(pre_blk, B, xx, Hkv);
+      {
+        const int nb = pre_blk[cur.b + 1] - pre_blk[cur.b];
+        const long long rem = xx - static_cast<long long>(Hkv) * pre_blk[cur.b];
+        cur.g = static_cast<int>(rem / nb);
+        cur.j = static_cast<int>(rem % nb);
+      }
+      while (xx < hi && nseg < kMaxSeg) {
+        const int nb = pre_blk[cur.b + 1] - pre_blk[cur.b];
+        long long n = min(static_cast<long long>(nb - cur.j), hi - xx);
+        if (chunk_mode) n = min(n, static_cast<long long>(p.chunk_blocks - cur.j % p.chunk_blocks));
+        if (used + n > kCap) {
+          if (nseg > 0) break;
+          n = kCap;   // cannot happen with the host's sizing; keeps the kernel in bounds regardless
+        }
+        Segment s;
+        s.b = cur.b; s.g = cur.g; s.j0 = cur.j; s.n = static_cast<int>(n); s.list_off = used;
+        s.seq_blocks = nb;
+        s.ctx_len = max(0, min(p.context_lens[cur.b], p.max_blocks_per_seq * kBlockSize));
+        if (chunk_mode) {
+          s.partial = 1;
+          s.slot = cur.j / p.chunk_blocks;
+          s.expected = pre_unit[cur.b + 1] - pre_unit[cur.b];
+        } else {
+          s.partial = !(cur.j == 0 && n == nb);
+          s.slot = 2 * blockIdx.x + (cur.j > 0 ? 0 : 1);
+          const long long fs = static_cast<long long>(Hkv) * pre_blk[cur.b] + static_cast<long long>(cur.g) * nb;
+          s.expected = cta_of(fs + nb - 1) - cta_of(fs) + 1;
+        }
+        segs[nseg++] = s;
+        used += static_cast<int>(n);
+        xx += n;
+        cur.j += static_cast<int>(n);
+        if (cur.j >= nb) {
+          cur.j = 0;
+          if (++cur.g == Hkv) {
+            cur.g = 0;
+            ++cur.b;
+            while (cur.b < B && pre_blk[cur.b + 1] == pre_blk[cur.b]) ++cur.b;
+          }
+        }
+      }
+      misc[0] = nseg;
+      misc[1] = static_cast<int>(xx & 0xffffffffll);
+      misc[2] = static_cast<int>(xx >> 32);
+    }
+    __syncthreads();
+    const int nseg = misc[0];
+    const long long x_next = (static_cast<long long>(misc[2]) << 32) | static_cast<unsigned int>(misc[1]);
+
+    // stage the physical block ids of every segment
+    for (int s = 0; s < nseg; ++s) {
+      const Segment& sg = segs[s];
+      const int* trow = p.block_table + static_cast<size_t>(sg.b) * p.max_blocks_per_seq + sg.j0;
+      for (int k = tid; k < sg.n; k += kThreads) {
+        int id = trow[k];
+        if (id < 0 || id >= p.num_blocks) { atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG); id = 0; }
+        ids[sg.list_off + k] = id;
+      }
+    }
+    __syncthreads();
+
+    // ---- producer cursor of this warp: (segment, block-in-segment) --------------------------
+    int pseg = 0, pk = warp;
+    auto prod_normalise = [&]() {
+      while (pseg < nseg && pk >= segs[pseg].n) { ++pseg; pk = warp; }
+    };
+    auto prod_issue = [&]() {
+      const Segment& sg = segs[pseg];
+      const int id = ids[sg.list_off + pk];
+      const uint8_t* src = p.cache + (static_cast<size_t>(id) * Hkv + sg.g) * C::kGran;
+      const uint32_t stage = issued % C::kStages;
+      if (lane == 0) {
+        mbar_expect_tx(&my_bars[stage], C::kGran);
+        bulk_copy_g2s(my_ring + stage * C::kGran, src, C::kGran, &my_bars[stage]);
+      }
+      ++issued;
+      pk += kWarps;
+    };
+    prod_normalise();
+    if (!dead) {
+#pragma unroll 1
+      for (int s = 0; s < C::kStages && pseg < nseg; ++s) { prod_issue(); prod_normalise(); }
+    }
+
+    // raw query registers of the next segment, loaded one segment ahead
+    uint32_t qraw[C::kKSteps][2];
+    auto load_q_raw = [&](const Segment& sg) {
+      const bool live = row < G;
+      const __nv_bfloat16* qp = p.q + (static_cast<size_t>(sg.b) * Hq + sg.g * G + (live ? row : 0)) * D + 2 * quad;
+#pragma unroll
+      for (int s = 0; s < C::kKSteps; ++s) {
+        qraw[s][0] = live ? *reinterpret_cast<const uint32_t*>(qp + 16 * s) : 0u;
+        qraw[s][1] = live ? *reinterpret_cast<const uint32_t*>(qp + 16 * s + 8) : 0u;
+      }
+    };
+    if (nseg > 0) load_q_raw(segs[0]);
+
+    for (int si = 0; si < nseg; ++si) {
+      const Segment sg = segs[si];
+
+      // ---- query fragments (A operand), converted for the tensor-core input type ------------
+      uint32_t qa[C::kKSteps][2];
+      float qscale = p.sm_scale_log2;
+      if constexpr (FP8) {
+        float amax = 0.0f;
+#pragma unroll
+        for (int s = 0; s < C::kKSteps; ++s)
+#pragma unroll
+          for (int e = 0; e < 2; ++e)
+            amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(qraw[s][e])), fabsf(bf16_hi(qraw[s][e]))));
+        amax = quad_max(amax);
+        // power-of-two scaling into f16's comfortable range: exact, undone on the logits
+        int k2 = 0;
+        if (amax > 0.0f) k2 = max(-64, min(64, 134 - static_cast<int>((__float_as_uint(amax) >> 23) & 0xFF)));
+        const float up = __uint_as_float(static_cast<uint32_t>(k2 + 127) << 23);
+        const float down = __uint_as_float(static_cast<uint32_t>(127 - k2) << 23);
+        qscale *= down;
+#pragma unroll
+        for (int s = 0; s < C::kKSteps; ++s)
+#pragma unroll
+          for (int e = 0; e < 2; ++e)
+            qa[s][e] = pack_f16x2(bf16_lo(qraw[s][e]) * up, bf16_hi(qraw[s][e]) * up);
+      } else {
+#pragma unroll
+        for (int s = 0; s < C::kKSteps; ++s) { qa[s][0] = qraw[s][0]; qa[s][1] = qraw[s][1]; }
+      }
+      if (si + 1 < nseg) load_q_raw(segs[si + 1]);
+
+      // ---- online softmax state of this warp for the segment ---------------------------------
+      float m_run = -INFINITY, l_run = 0.0f, vref = 0.0f;
+      float o[C::kNTiles][C::kOAcc];
+#pragma unroll
+      for (int t = 0; t < C::kNTiles; ++t)
+#pragma unroll
+        for (int e = 0; e < C::kOAcc; ++e) o[t][e] = 0.0f;
+
+#pragma unroll 1
+      for (int k = warp; k < sg.n; k += kWarps) {
+        const uint32_t stage = consumed % C::kStages;
+        const uint32_t parity = (consumed / C::kStages) & 1u;
+        if (!dead && !mbar_wait_bounded(&my_bars[stage], parity)) {
+          dead = true;
+          if (lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+        }
+        ++consumed;
+        if (dead) continue;
+        const uint8_t* st = my_ring + stage * C::kGran;
+        const int nvalid = min(kBlockSize, sg.ctx_len - (sg.j0 + k) * kBlockSize);   // Eq. 9 tail
+
+        float sK = 1.0f, sV = 1.0f;
+        if constexpr (FP8) {
+          sK = reinterpret_cast<const float*>(st)[0];
+          sV = reinterpret_cast<const float*>(st)[1];
+        }
+
+        // ---- S = Q K^T for 16 tokens (two n-tiles of 8) ---------------------------------------
+        float s0[2] = {0.0f, 0.0f}, s1[2] = {0.0f, 0.0f};
+        const uint8_t* kp = st + part_offset(D, FP8, 0) + lane * 16;
+        if constexpr (FP8) {
+#pragma unroll
+          for (int i = 0; i < D / 64; ++i) {
+            const uint4 w0 = lds128(kp + (0 * (D / 64) + i) * 512);
+            const uint4 w1 = lds128(kp + (1 * (D / 64) + i) * 512);
+            const uint32_t a[4] = {w0.x, w0.y, w0.z, w0.w}, c[4] = {w1.x, w1.y, w1.z, w1.w};
+#pragma unroll
+            for (int ss = 0; ss < 4; ++ss) {
+              const int s = 4 * i + ss;
+              mma_top<true>(s0[0], s0[1], qa[s][0], qa[s][1], e4m3x2_to_f16x2_lo(a[ss]), e4m3x2_to_f16x2_hi(a[ss]));
+              mma_top<true>(s1[0], s1[1], qa[s][0], qa[s][1], e4m3x2_to_f16x2_lo(c[ss]), e4m3x2_to_f16x2_hi(c[ss]));
+            }
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < D / 32; ++i) {
+            const uint4 w0 = lds128(kp + (0 * (D / 32) + i) * 512);
+            const uint4 w1 = lds128(kp + (1 * (D / 32) + i) * 512);
+            mma_top<false>(s0[0], s0[1], qa[2 * i][0], qa[2 * i][1], w0.x, w0.y);
+            mma_top<false>(s0[0], s0[1], qa[2 * i + 1][0], qa[2 * i + 1][1], w0.z, w0.w);
+            mma_top<false>(s1[0], s1[1], qa[2 * i][0], qa[2 * i][1], w1.x, w1.y);
+            mma_top<false>(s1[0], s1[1], qa[2 * i + 1][0], qa[2 * i + 1][1], w1.z, w1.w);
+          }
+        }
+
+        // ---- online softmax (Eq. 10), log2 units ---------------------------------------------------
+        const float ks = qscale * sK;
+        float sc[4] = {s0[0] * ks, s0[1] * ks, s1[0] * ks, s1[1] * ks};
+        const int tok[4] = {2 * quad, 2 * quad + 1, 2 * quad + 8, 2 * quad + 9};
+        if (nvalid < kBlockSize) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) sc[e] = tok[e] < nvalid ? sc[e] : -INFINITY;
+        }
+        const float m_blk = quad_max(fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3])));
+        const float m_new = fmaxf(m_run, m_blk);
+        const float a_m = ex2(m_run - m_new);
+        float a_o = a_m, pv = 1.0f;
+        if constexpr (FP8) {
+          // o accumulates sum p * (sV / vref) * codes with vref the largest V scale seen so far
+          const float vnew = fmaxf(vref, sV);
+          if (vnew > 0.0f) {
+            a_o = a_m * __fdividef(vref, vnew);
+            pv = __fdividef(sV, vnew);
+          }
+          vref = vnew;
+        }
+        float pr[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) pr[e] = ex2(sc[e] - m_new);
+        l_run = l_run * a_m + (pr[0] + pr[1]) + (pr[2] + pr[3]);
+        m_run = m_new;
+        if (__any_sync(0xffffffffu, a_o != 1.0f)) {
+#pragma unroll
+          for (int t = 0; t < C::kNTiles; ++t)
+#pragma unroll
+            for (int e = 0; e < C::kOAcc; ++e) o[t][e] *= a_o;
+        }
+
+        // ---- O += P V -----------------------------------------------------------------------------
+        const uint8_t* vp = st + part_offset(D, FP8, 1) + lane * 16;
+        if constexpr (FP8) {
+          const uint32_t pa0 = pack_f16x2(pr[0] * pv, pr[1] * pv), pa2 = pack_f16x2(pr[2] * pv, pr[3] * pv);
+          uint32_t vmask = 0xffffffffu;
+          if (nvalid < kBlockSize) {
+            vmask = 0u;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) vmask |= tok[e] < nvalid ? (0xFFu << (8 * e)) : 0u;
+          }
+#pragma unroll
+          for (int qd = 0; qd < D / 32; ++qd) {
+            const uint4 w = lds128(vp + qd * 512);
+            const uint32_t a[4] = {w.x & vmask, w.y & vmask, w.z & vmask, w.w & vmask};
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              mma_top<true>(o[4 * qd + u][0], o[4 * qd + u][1], pa0, pa2, e4m3x2_to_f16x2_lo(a[u]), e4m3x2_to_f16x2_hi(a[u]));
+          }
+        } else {
+          // bf16 probabilities split into high and low halves; the low halves ride in rows 8..15
+          uint32_t hi0 = pack_bf16x2(pr[0], pr[1]), hi2 = pack_bf16x2(pr[2], pr[3]);
+          const uint32_t lo0 = pack_bf16x2(pr[0] - bf16_lo(hi0), pr[1] - bf16_hi(hi0));
+          const uint32_t lo2 = pack_bf16x2(pr[2] - bf16_lo(hi2), pr[3] - bf16_hi(hi2));
+          uint32_t m01 = 0xffffffffu, m89 = 0xffffffffu;
+          if (nvalid < kBlockSize) {
+            m01 = (tok[0] < nvalid ? 0x0000FFFFu : 0u) | (tok[1] < nvalid ? 0xFFFF0000u : 0u);
+            m89 = (tok[2] < nvalid ? 0x0000FFFFu : 0u) | (tok[3] < nvalid ? 0xFFFF0000u : 0u);
+          }
+#pragma unroll
+          for (int qd = 0; qd < D / 16; ++qd) {
+            const uint4 w = lds128(vp + qd * 512);
+            mma16816<false>(o[2 * qd], hi0, lo0, hi2, lo2, w.x & m01, w.y & m89);
+            mma16816<false>(o[2 * qd + 1], hi0, lo0, hi2, lo2, w.z & m01, w.w & m89);
+          }
+        }
+
+        // ---- hand the stage back to the copy engine ------------------------------------------------
+        __syncwarp();
+        if (pseg < nseg) {
+          if (lane == 0) fence_proxy_async();
+          prod_issue();
+          prod_normalise();
+        }
+      }
+
+      // ---- end of segment: combine the warps' states through shared memory --------------------
+      l_run = quad_sum(l_run);
+      if (row < G) {
+        float* mr = merge + (warp * kMaxGroup + row) * C::kMergeStride;
+        const float os = FP8 ? vref : 1.0f;
+#pragma unroll
+        for (int t = 0; t < C::kNTiles; ++t) {
+          float v0 = o[t][0], v1 = o[t][1];
+          if constexpr (!FP8) { v0 += o[t][2]; v1 += o[t][3]; }
+          *reinterpret_cast<float2*>(mr + 8 * t + 2 * quad) = make_float2(v0 * os, v1 * os);
+        }
+        if (quad == 0) { mr[D] = m_run; mr[D + 1] = l_run; }
+      }
+      __syncthreads();
+
+      const int h0 = sg.g * G;
+      float* po = nullptr; float* pm = nullptr; float* pl = nullptr;
+      if (sg.partial) {
+        if (chunk_mode) {
+          const size_t base = (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks + sg.slot;
+          po = p.part_o + base * D; pm = p.part_m + base; pl = p.part_l + base;
+        } else {
+          const size_t base = static_cast<size_t>(sg.slot) * G;
+          po = p.part_o + base * D; pm = p.part_m + base; pl = p.part_l + base;
+        }
+      }
+      const size_t pstride = chunk_mode ? static_cast<size_t>(p.max_chunks) : 1;   // row stride of partial arrays
+      for (int idx = tid; idx < G * D; idx += kThreads) {
+        const int r = idx / D, d = idx % D;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) M = fmaxf(M, merge[(w * kMaxGroup + r) * C::kMergeStride + D]);
+        float num = 0.0f, den = 0.0f;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+          const float* mw = merge + (w * kMaxGroup + r) * C::kMergeStride;
+          const float wgt = ex2(mw[D] - M);
+          num += wgt * mw[d];
+          den += wgt * mw[D + 1];
+        }
+        const float val = num / den;
+        if (!sg.partial) {
+          p.out[(static_cast<size_t>(sg.b) * Hq + h0 + r) * D + d] = __float2bfloat16(val);
+        } else {
+          po[r * pstride * D + d] = val;
+          if (d == 0) {
+            pm[r * pstride] = chunk_mode ? M * kLn2 : M;   // exported partials use natural-log units
+            pl[r * pstride] = den;
+          }
+        }
+      }
+
+      if (sg.partial) {
+        __threadfence();
+        __syncthreads();
+        int* counter = p.counters + sg.b * Hkv + sg.g;
+        if (tid == 0) {
+          const int old = atomicAdd(counter, 1);
+          const int last = old == sg.expected - 1;
+          if (last) *counter = 0;             // ready for the next call
+          misc[3] = last;
+        }
+        __syncthreads();
+        if (misc[3]) {
+          // this CTA delivered the last piece: log-sum-exp merge of all pieces (split-K merge)
+          __threadfence();
+          int first_cta = 0;
+          if (!chunk_mode) {
+            const long long fs = static_cast<long long>(Hkv) * pre_blk[sg.b] + static_cast<long long>(sg.g) * sg.seq_blocks;
+            first_cta = cta_of(fs);
+          }
+          for (int idx = tid; idx < G * D; idx += kThreads) {
+            const int r = idx / D, d = idx % D;
+            float M = -INFINITY;
+            for (int c = 0; c < sg.expected; ++c) {
+              size_t at;
+              if (chunk_mode) at = (static_cast<size_t>(sg.b) * Hq + h0 + r) * p.max_chunks + c;
+              else at = static_cast<size_t>(2 * (first_cta + c) + (c == 0 ? 1 : 0)) * G + r;
+              M = fmaxf(M, __ldcg(p.part_m + at));
+            }
+            float num = 0.0f, den = 0.0f;
+            for (int c = 0; c < sg.expected; ++c) {
+              size_t at;
+              if (chunk_mode) at = (static_cast<size_t>(sg.b) * Hq + h0 + r) * p.max_chunks + c;
+              else at = static_cast<size_t>(2 * (first_cta + c) + (c == 0 ? 1 : 0)) * G + r;
+              const float mc = __ldcg(p.part_m + at), lc = __ldcg(p.part_l + at);
+              const float wgt = lc * (chunk_mode ? ex2((mc - M) * kLog2e) : ex2(mc - M));
+              num += wgt * __ldcg(p.part_o + at * D + d);
+              den += wgt;
+            }
+            p.out[(static_cast<size_t>(sg.b) * Hq + h0 + r) * D + d] = __float2bfloat16(num / den);
+          }
+        }
+      }
+      __syncthreads();   // merge scratch and misc[3] are reused by the next segment
+    }
+
+    x = x_next;
+    __syncthreads();
+  }
+
+  // a warp that gave up still has copies in flight: give them a bounded time to land before
+  // the CTA's shared memory is released
+  if (dead) {
+    while (consumed < issued) {
+      const uint32_t stage = consumed % C::kStages, parity = (consumed / C::kStages) & 1u;
+      mbar_wait_bounded(&my_bars[stage], parity);
+      ++consumed;
+    }
+  }
+}
+
+}  // namespace
+
+// Workspace layout: [header 256 B: word 0 = status][counters int32 x 16384][partials].
+size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int batch, int num_q_heads, int max_chunks) {
+  size_t bytes = kWsHeaderBytes + static_cast<size_t>(kCounterSlots) * 4;
+  const size_t dec = static_cast<size_t>(2) * planned_ctas * group * (head_dim + 2) * 4;
+  const size_t chk = static_cast<size_t>(batch) * num_q_heads * max_chunks * (head_dim + 2) * 4;
+  return bytes + (dec > chk ? dec : chk) + 256;
+}
+size_t workspace_control_bytes() { return kWsHeaderBytes + static_cast<size_t>(kCounterSlots) * 4; }
+
+int decode_planned_ctas(int num_sms, long long upper_blocks) {
+  const long long need = (upper_blocks + kCap / 2 - 1) / (kCap / 2);
+  return static_cast<int>(need > num_sms ? need : num_sms);
+}
+int decode_max_batch() { return kMaxBatch; }
+int decode_counter_slots() { return kCounterSlots; }
+int decode_max_chunk_blocks() { return kCap; }
+
+void chunk_partial_offsets(int batch, int num_q_heads, int head_dim, int max_chunks, size_t* o, size_t* m, size_t* l) {
+  const size_t rows = static_cast<size_t>(batch) * num_q_heads * max_chunks;
+  *o = workspace_control_bytes();
+  *m = *o + rows * head_dim * 4;
+  *l = *m + rows * 4;
+}
+
+template <int D, bool FP8>
+static int launch_one(const DecodeParams& p, int grid, cudaStream_t stream) {
+  using C = Cfg<D, FP8>;
+  static bool configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
+  if (dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(paged_decode_kernel<D, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+      return COOPT_ERR_CUDA;
+    configured[dev] = true;
+  }
+  paged_decode_kernel<D, FP8><<<grid, kThreads, C::kSmemBytes, stream>>>(p);
+  return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
+}
+
+int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
+                        int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                        float sm_scale, int32_t chunk_size, void* workspace, int planned_ctas, cudaStream_t stream) {
+  DecodeParams p;
+  p.cache = static_cast<const uint8_t*>(c->data);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.block_table = block_table;
+  p.context_lens = context_lens;
+  p.max_blocks_per_seq = max_blocks_per_seq;
+  p.batch = batch;
+  p.num_q_heads = num_q_heads;
+  p.num_kv_heads = c->num_kv_heads;
+  p.group = num_q_heads / c->num_kv_heads;
+  p.num_blocks = c->num_blocks;
+  p.sm_scale_log2 = sm_scale * kLog2e;
+  p.planned_ctas = planned_ctas;
+  p.chunk_blocks = chunk_size / kBlockSize;
+  p.max_chunks = chunk_size > 0 ? static_cast<int>((static_cast<long long>(max_blocks_per_seq) * kBlockSize + chunk_size - 1) / chunk_size) : 0;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  p.status = reinterpret_cast<int*>(ws);
+  p.counters = reinterpret_cast<int*>(ws + kWsHeaderBytes);
+  uint8_t* parts = ws + workspace_control_bytes();
+  if (chunk_size > 0) {
+    size_t o, m, l;
+    chunk_partial_offsets(batch, num_q_heads, c->head_dim, p.max_chunks, &o, &m, &l);
+    p.part_o = reinterpret_cast<float*>(ws + o);
+    p.part_m = reinterpret_cast<float*>(ws + m);
+    p.part_l = reinterpret_cast<float*>(ws + l);
+  } else {
+    const size_t rows = static_cast<size_t>(2) * planned_ctas * p.group;
+    p.part_o = reinterpret_cast<float*>(parts);
+    p.part_m = p.part_o + rows * c->head_dim;
+    p.part_l = p.part_m + rows;
+  }
+  const bool fp8 = c->dtype == COOPT_KV_FP8_E4M3;
+  if (c->head_dim == 128) return fp8 ? launch_one<128, true>(p, planned_ctas, stream) : launch_one<128, false>(p, planned_ctas, stream);
+  return fp8 ? launch_one<64, true>(p, planned_ctas, stream) : launch_one<64, false>(p, planned_ctas, stream);
+}
+
+}  // namespace coopt
