@@ -1,0 +1,329 @@
+#!/usr/bin/env python
+"""Benchmark of the paged FP8 GQA decode path (one JSON line on stdout).
+
+A step is one pass of the hot path for one attention layer over one batch: coopt_kv_write
+appends the new token of every sequence, then coopt_paged_decode attends over the updated
+cache.  Workload: LLaMA-13B-shaped decode (batch 32, 40 query heads over 8 KV heads,
+head_dim 128, every context 2048 tokens, block size 16, shuffled block table, FP8 E4M3 cache,
+N(0,1) values with two x20 outlier channels per head).  Steps rotate over several layer caches
+so that the data touched between two visits of a cache exceeds L2.
+
+    python bench.py --gpus N --steps K --warmup W          (N > 1: launched by torchrun)
+    python bench.py --impl reference ...                   (the CPU oracle on the host cores)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "paged FP8 GQA decode tokens/s"
+UNIT = "attention-layer tokens/s"
+BATCH, HQ, HKV, D, CONTEXT = 32, 40, 8, 128, 2048
+WORKLOAD = "llama13b_decode: batch 32, Hq 40, Hkv 8, head_dim 128, context 2048, block 16, fp8 e4m3 cache"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def algorithmic_bytes(batch=BATCH, context=CONTEXT):
+    """Bytes one decode launch must move: FP8 codes of the valid tokens, one K and one V scale
+    per (block, kv head), q and out, block table and context lengths."""
+    blocks = batch * ((context + 15) // 16)
+    kv = batch * context * HKV * D * 2
+    scales = blocks * HKV * 8
+    q_out = 2 * batch * HQ * D * 2
+    table = blocks * 4 + batch * 4
+    return kv + scales + q_out + table
+
+
+class ClockSampler(threading.Thread):
+    """SM clock and throttle reasons of one GPU, sampled through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.005):
+        super().__init__(daemon=True)
+        self.index, self.period, self.samples, self.reasons, self.stop_flag = index, period_s, [], set(), False
+        self.max_mhz, self.ok = None, False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self.stop_flag:
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(s)}
+
+
+class OracleSample:
+    """The CPU oracle, as it stands, on units of the benchmark workload.  A unit is one
+    (sequence, kv head): the write of the new token's K/V for that head and the attention of
+    its 5 query heads over the 2048-token context (float64, gather through the block table,
+    FP8 dequantisation from the oracle's own cache).  The 2047-token history is built once,
+    outside any timing."""
+
+    def __init__(self, seed=0):
+        from oracle import kv_cache
+        from paper_2602_09323_b200 import workloads
+        w = workloads.make_workload("llama13b_decode_sample", [CONTEXT], HQ, HKV, D, seed=seed)
+        self.k, self.v, self.slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
+        self.q, self.table = w.q.float().numpy(), w.block_table.numpy()
+        self.codes, self.scales = kv_cache.new_cache(w.num_blocks, HKV, D)
+        kv_cache.kv_write(self.codes, self.scales, self.k[:-1], self.v[:-1], self.slots[:-1])
+        self.done = 0
+
+    def run(self, units=None, seconds_budget=None):
+        """Returns (units done, seconds)."""
+        from threadpoolctl import threadpool_limits
+        from oracle import attention, kv_cache
+        n, t0 = 0, time.perf_counter()
+        with threadpool_limits(limits=1):
+            while True:
+                g = self.done % HKV
+                kv_cache.kv_write(self.codes, self.scales, self.k[-1:], self.v[-1:], self.slots[-1:], heads=[g])
+                attention.paged_attention(self.q, (self.codes, self.scales), self.table, [CONTEXT],
+                                          pairs=[(0, h) for h in range(g * 5, g * 5 + 5)])
+                self.done += 1
+                n += 1
+                el = time.perf_counter() - t0
+                if (units is not None and n >= units) or (seconds_budget is not None and el >= seconds_budget):
+                    return n, el
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the host cores, same metric and workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = OracleSample()
+    _, t1 = sample.run(units=1)
+    per_step_budget = 120.0 / max(1, args.steps + args.warmup)
+    units_per_step = max(1, min(HKV * 4, int(per_step_budget / max(t1, 1e-6))))
+    for _ in range(args.warmup):
+        sample.run(units=units_per_step)
+    total, el = 0, 0.0
+    for _ in range(args.steps):
+        n, t = sample.run(units=units_per_step)
+        total, el = total + n, el + t
+    value = (total / HKV) / el
+    what = "%d units per step; a unit = the new token's K/V written for one kv head + that head's 5 query heads " \
+           "over a 2048-token context, float64" % units_per_step
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / max(1, args.steps),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "note": "CPU oracle on the host cores, bounded sample per step"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": what},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=8, help="layer caches the steps rotate over")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline leg")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import torch.distributed as dist
+    from paper_2602_09323_b200 import binding, build, workloads
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    warmup = max(3, args.warmup)
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if local == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+    binding.load_library()
+
+    # ---- synthetic workload: NL layer caches, history of 2047 tokens, token 2048 appended per step
+    base = workloads.config_llama13b_decode(seed=rank, batch=BATCH, context=CONTEXT)
+    k_dev, v_dev = base.k.cuda(), base.v.cuda()
+    hist = torch.ones(BATCH * CONTEXT, dtype=torch.bool)
+    hist[CONTEXT - 1::CONTEXT] = False                                     # the last token of each sequence is the new one
+    hist_idx = hist.nonzero().squeeze(1).cuda()
+    new_idx = (~hist).nonzero().squeeze(1).cuda()
+    k_hist, v_hist = k_dev[hist_idx], v_dev[hist_idx]
+    k_new, v_new = k_dev[new_idx].contiguous(), v_dev[new_idx].contiguous()
+    q = base.q.cuda()
+    lens = base.context_lens_tensor.cuda()
+    layers = []
+    for l in range(args.layers):
+        w = base if l == 0 else workloads.relayout(base, seed=1000 * (rank + 1) + l)
+        cache = binding.Cache(w.num_blocks, HKV, D)
+        slots = w.slot_mapping.cuda()
+        binding.kv_write(cache, k_hist, v_hist, slots[hist_idx])
+        layers.append({"cache": cache, "table": w.block_table.clamp(min=0).cuda(), "slots_new": slots[new_idx].contiguous(),
+                       "table_host": w.block_table.clamp(min=0).pin_memory(),
+                       "slots_new_host": w.slot_mapping[new_idx.cpu()].contiguous().pin_memory()})
+    del k_hist, v_hist
+    max_blocks = base.block_table.shape[1]
+    ws = binding.new_workspace(BATCH, HQ, HKV, D, max_blocks)
+    out = torch.empty_like(q)
+    torch.cuda.synchronize()
+
+    def step(i):
+        L = layers[i % args.layers]
+        binding.kv_write(L["cache"], k_new, v_new, L["slots_new"])
+        binding.paged_decode(L["cache"], q, L["table"], lens, base.sm_scale, ws, out=out)
+
+    def step_timed(i, e0, e1):
+        L = layers[i % args.layers]
+        binding.kv_write(L["cache"], k_new, v_new, L["slots_new"])
+        e0.record()
+        binding.paged_decode(L["cache"], q, L["table"], lens, base.sm_scale, ws, out=out)
+        e1.record()
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+
+    # ---- timed region: K steps, CUDA events on the launching stream, decode kernel timed live
+    stride = max(1, args.steps // 4000)
+    kernel_events = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                     for _ in range((args.steps + stride - 1) // stride)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    start.record()
+    for i in range(args.steps):
+        if i % stride == 0:
+            step_timed(i, *kernel_events[i // stride])
+        else:
+            step(i)
+    stop.record()
+    torch.cuda.synchronize()
+    sampler.stop_flag = True
+    if world > 1:
+        dist.barrier()
+    ms = start.elapsed_time(stop)
+    kernel_ms = sum(a.elapsed_time(b) for a, b in kernel_events) / len(kernel_events)
+    assert binding.workspace_status(ws) == 0
+    t = torch.tensor([ms, kernel_ms], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms, kernel_ms = float(t[0]), float(t[1])
+    value = world * BATCH * args.steps / (ms * 1e-3)
+
+    # ---- end to end: host buffers in, host result out, through coopt_decode_step_host ----------
+    e2e = None
+    if not args.no_e2e:
+        staging = torch.empty(binding.step_staging_bytes(BATCH, HQ, HKV, D, max_blocks), dtype=torch.uint8, device="cuda")
+        hq_, hk_, hv_ = base.q.pin_memory(), k_new.cpu().pin_memory(), v_new.cpu().pin_memory()
+        hl_, ho_ = base.context_lens_tensor.pin_memory(), torch.empty_like(base.q).pin_memory()
+        n_e2e = max(1, min(args.steps, 2000))
+
+        def host_step(i):
+            L = layers[i % args.layers]
+            binding.decode_step_host(L["cache"], hq_, hk_, hv_, L["slots_new_host"], L["table_host"], hl_, ho_,
+                                     base.sm_scale, staging, ws)
+            torch.cuda.synchronize()                                       # the step's result is read on the host
+
+        for i in range(3):
+            host_step(i)
+        if world > 1:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for i in range(n_e2e):
+            host_step(i)
+        el = time.perf_counter() - t0
+        te = torch.tensor([el], device="cuda", dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        h2d = hq_.numel() * 2 + hk_.numel() * 2 + hv_.numel() * 2 + BATCH * 8 + BATCH * max_blocks * 4 + BATCH * 4
+        e2e = {"value": world * BATCH * n_e2e / float(te[0]), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": ho_.numel() * 2, "steps": n_e2e}
+        assert torch.equal(ho_.cuda(), out)
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (decode), CPU baseline --------------------------------
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(peaks_path):
+        peak, peak_src = float(json.load(open(peaks_path))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    else:
+        peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    algo = algorithmic_bytes()
+    achieved = algo / (kernel_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": "paged_decode_kernel<128,fp8>", "achieved": achieved, "peak": peak,
+                "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": algo, "kernel_us": kernel_ms * 1e3, "traffic": DRAM_TRAFFIC_PER_LAUNCH}
+    cpu = None
+    if world == 1 and args.cpu_seconds > 0:
+        n_units, el = OracleSample().run(seconds_budget=args.cpu_seconds)
+        cpu = {"value": (n_units / HKV) / el, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": "%d (sequence, kv head) units of one 2048-token sequence in %.1f s; a unit = the new token's "
+                         "K/V written for one kv head + its 5 query heads' float64 attention" % (n_units, el)}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "fp8_e4m3 cache, f16 tensor-core products, f32 accumulate", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "layers_rotated": args.layers,
+                       "l2": "inputs larger than L2: %d layer caches of %.0f MB visited round-robin" %
+                             (args.layers, algo / 1e6), "step": "coopt_kv_write(1 token/seq) + coopt_paged_decode"},
+            "gpu_launches": 2 * args.steps, "clocks": sampler.summary(), "e2e": e2e, "roofline": roofline,
+            "cpu_baseline": cpu}
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode launch on this workload, from the
+# ncu capture summarised under profiles/ (None until a capture has been taken).
+DRAM_TRAFFIC_PER_LAUNCH = None
+
+if __name__ == "__main__":
+    main()

@@ -143,6 +143,29 @@ int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, cons
                         int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t chunk_size, int32_t causal,
                         float sm_scale, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * coopt_decode_step_host — one serving step for callers whose step inputs live in HOST memory
+ * (Section 2's token-insertion phase followed by the attention phase): copies the step's
+ * inputs to the device, runs coopt_kv_write for the one new token of every sequence and
+ * coopt_paged_decode over the updated cache, and copies the bf16 result back.  Everything is
+ * enqueued on `stream`; the host buffers must stay valid (and should be pinned) until the
+ * stream has been synchronised.  The cache and both scratch areas are DEVICE memory.
+ *   q_host, out_host      HOST bf16 [batch][num_q_heads][head_dim]
+ *   k_host, v_host        HOST bf16 [batch][num_kv_heads][head_dim] (the new token of each sequence)
+ *   slot_mapping_host     HOST int64 [batch]
+ *   block_table_host      HOST int32 [batch][max_blocks_per_seq]
+ *   context_lens_host     HOST int32 [batch], counting the new token
+ *   staging               DEVICE, >= coopt_step_staging_bytes(...) bytes, 256-byte aligned
+ * Errors: as coopt_kv_write and coopt_paged_decode, WORKSPACE if staging is too small.
+ */
+int coopt_decode_step_host(const coopt_cache* cache, const void* q_host, const void* k_host, const void* v_host,
+                           const int64_t* slot_mapping_host, const int32_t* block_table_host,
+                           int32_t max_blocks_per_seq, const int32_t* context_lens_host, void* out_host,
+                           int32_t batch, int32_t num_q_heads, float sm_scale, void* staging, size_t staging_bytes,
+                           void* workspace, size_t workspace_bytes, void* stream);
+size_t coopt_step_staging_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                                int32_t max_blocks_per_seq);
+
 /* Workspace size for a call with these arguments (chunk_size = 0 for coopt_paged_decode).
  * Host arithmetic only (it asks the current device for its SM count once). */
 size_t coopt_workspace_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,

@@ -52,6 +52,11 @@ _SIGNATURES = {
     "coopt_workspace_init": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "coopt_chunk_partials": (ctypes.c_int, [ctypes.c_int32] * 5 + [ctypes.POINTER(ctypes.c_size_t)] * 3
                              + [ctypes.POINTER(ctypes.c_int32)]),
+    "coopt_decode_step_host": (ctypes.c_int, [ctypes.POINTER(coopt_cache)] + [ctypes.c_void_p] * 5 + [ctypes.c_int32]
+                               + [ctypes.c_void_p] * 2 + [ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
+                                                          ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
+                                                          ctypes.c_size_t, ctypes.c_void_p]),
+    "coopt_step_staging_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 5),
     "coopt_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "coopt_version": (ctypes.c_int, []),
 }
@@ -197,3 +202,20 @@ def chunk_partials(workspace: torch.Tensor, batch: int, num_q_heads: int, head_d
     f = lambda off, n: workspace[off:off + 4 * n].view(torch.float32)
     return (f(o.value, rows * head_dim).view(batch, num_q_heads, mc.value, head_dim),
             f(m.value, rows).view(batch, num_q_heads, mc.value), f(l.value, rows).view(batch, num_q_heads, mc.value))
+
+
+def step_staging_bytes(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, max_blocks_per_seq: int) -> int:
+    return load_library().coopt_step_staging_bytes(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq)
+
+
+def decode_step_host(cache: Cache, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, slot_mapping: torch.Tensor,
+                     block_table: torch.Tensor, context_lens: torch.Tensor, out: torch.Tensor, sm_scale: float,
+                     staging: torch.Tensor, workspace: torch.Tensor) -> None:
+    """coopt_decode_step_host: all step inputs and ``out`` are HOST (pinned) tensors; asynchronous."""
+    for t in (q, k, v, slot_mapping, block_table, context_lens, out):
+        assert not t.is_cuda and t.is_contiguous()
+    st = load_library().coopt_decode_step_host(cache.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(slot_mapping),
+                                               _ptr(block_table), block_table.shape[1], _ptr(context_lens), _ptr(out),
+                                               q.shape[0], q.shape[1], float(sm_scale), _ptr(staging), staging.numel(),
+                                               _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "coopt_decode_step_host")

@@ -190,6 +190,68 @@ int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, cons
                               num_q_heads, total_q, causal, sm_scale, workspace, static_cast<cudaStream_t>(stream));
 }
 
+namespace {
+struct StepStaging {
+  size_t q, out, k, v, slots, table, lens, total;
+};
+StepStaging step_staging(int batch, int hq, int hkv, int d, int max_blocks) {
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  StepStaging s;
+  size_t at = 0;
+  s.q = at;     at += up(static_cast<size_t>(batch) * hq * d * 2);
+  s.out = at;   at += up(static_cast<size_t>(batch) * hq * d * 2);
+  s.k = at;     at += up(static_cast<size_t>(batch) * hkv * d * 2);
+  s.v = at;     at += up(static_cast<size_t>(batch) * hkv * d * 2);
+  s.slots = at; at += up(static_cast<size_t>(batch) * 8);
+  s.table = at; at += up(static_cast<size_t>(batch) * max_blocks * 4);
+  s.lens = at;  at += up(static_cast<size_t>(batch) * 4);
+  s.total = at;
+  return s;
+}
+}  // namespace
+
+size_t coopt_step_staging_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                                int32_t max_blocks_per_seq) {
+  if (batch < 0 || num_q_heads <= 0 || num_kv_heads <= 0 || head_dim <= 0 || max_blocks_per_seq <= 0) return 0;
+  return step_staging(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq).total;
+}
+
+int coopt_decode_step_host(const coopt_cache* cache, const void* q_host, const void* k_host, const void* v_host,
+                           const int64_t* slot_mapping_host, const int32_t* block_table_host,
+                           int32_t max_blocks_per_seq, const int32_t* context_lens_host, void* out_host,
+                           int32_t batch, int32_t num_q_heads, float sm_scale, void* staging, size_t staging_bytes,
+                           void* workspace, size_t workspace_bytes, void* stream) {
+  int rc = check_cache(cache);
+  if (rc != COOPT_OK) return rc;
+  if (!q_host || !k_host || !v_host || !slot_mapping_host || !block_table_host || !context_lens_host || !out_host ||
+      batch < 0 || num_q_heads <= 0 || max_blocks_per_seq <= 0)
+    return COOPT_ERR_INVALID_ARG;
+  if (batch == 0) return COOPT_OK;
+  const int hkv = cache->num_kv_heads, d = cache->head_dim;
+  const StepStaging s = step_staging(batch, num_q_heads, hkv, d, max_blocks_per_seq);
+  if (!staging || staging_bytes < s.total) return COOPT_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(staging) % 256 != 0) return COOPT_ERR_INVALID_ARG;
+  uint8_t* dev = static_cast<uint8_t*>(staging);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t qb = static_cast<size_t>(batch) * num_q_heads * d * 2, kb = static_cast<size_t>(batch) * hkv * d * 2;
+  bool ok = true;
+  ok &= cudaMemcpyAsync(dev + s.q, q_host, qb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dev + s.k, k_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dev + s.v, v_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dev + s.slots, slot_mapping_host, static_cast<size_t>(batch) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dev + s.table, block_table_host, static_cast<size_t>(batch) * max_blocks_per_seq * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  ok &= cudaMemcpyAsync(dev + s.lens, context_lens_host, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
+  if (!ok) return COOPT_ERR_CUDA;
+  rc = coopt_kv_write(cache, dev + s.k, dev + s.v, static_cast<int64_t>(hkv) * d,
+                      reinterpret_cast<const int64_t*>(dev + s.slots), batch, stream);
+  if (rc != COOPT_OK) return rc;
+  rc = coopt_paged_decode(cache, dev + s.q, dev + s.out, reinterpret_cast<const int32_t*>(dev + s.table),
+                          max_blocks_per_seq, reinterpret_cast<const int32_t*>(dev + s.lens), batch, num_q_heads,
+                          sm_scale, workspace, workspace_bytes, stream);
+  if (rc != COOPT_OK) return rc;
+  return cudaMemcpyAsync(out_host, dev + s.out, qb, cudaMemcpyDeviceToHost, st) == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
+}
+
 const char* coopt_status_string(int status) {
   switch (status) {
     case COOPT_OK: return "ok";

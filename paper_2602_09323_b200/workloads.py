@@ -146,6 +146,20 @@ def make_workload(name: str, context_lens: Sequence[int], num_q_heads: int, num_
                     q, k, v, slot_mapping, block_table, kv_offsets, seed)
 
 
+def relayout(w: Workload, seed: int) -> Workload:
+    """The same tokens placed in a different random set of physical blocks (another layer's
+    cache has its own placement); q, k, v are shared, not copied."""
+    gen = torch.Generator(device="cpu")
+    gen.manual_seed(seed)
+    width = w.block_table.shape[1]
+    table, num_blocks = make_block_table(gen, [width * BLOCK_SIZE] * w.batch)
+    need = torch.tensor([(L + BLOCK_SIZE - 1) // BLOCK_SIZE for L in w.context_lens])
+    table[torch.arange(width)[None, :] >= need[:, None]] = -1
+    slots = [slots_for(table, b, 0, L) for b, L in enumerate(w.context_lens)]
+    slot_mapping = torch.cat(slots) if slots else torch.zeros(0, dtype=torch.int64)
+    return dataclasses.replace(w, block_table=table, slot_mapping=slot_mapping, num_blocks=num_blocks)
+
+
 def uniform_lengths(batch: int, lo: int, hi: int, seed: int) -> List[int]:
     """``batch`` context lengths uniform in [lo, hi] (inclusive), seeded."""
     gen = torch.Generator(device="cpu")
