@@ -122,6 +122,33 @@ int coopt_paged_decode(const coopt_cache* cache, const void* q, void* out, const
                        void* stream);
 
 /*
+ * coopt_paged_decode_static -- coopt_paged_decode without a caller-provided workspace.  (The
+ * paper has no counterpart of this call; the result is the one coopt_paged_decode gives.)
+ * It exists for callers that cannot allocate device memory where they call from: a plug-in
+ * whose enqueue hook must not allocate, a server that handed all device memory to its own
+ * pool at start-up so that a later cudaMalloc would fail or stall the device, a C program
+ * without a device allocator.  The split-KV partials and control words go to a fixed array of
+ * COOPT_STATIC_SCRATCH_BYTES inside the library; every device that loads the library holds
+ * that much memory until the process exits.  The call itself allocates nothing.
+ *   - Arguments as coopt_paged_decode, minus the workspace.
+ *   - Problems whose coopt_workspace_bytes(..., chunk_size = 0) exceeds
+ *     COOPT_STATIC_SCRATCH_BYTES are refused with COOPT_ERR_WORKSPACE before anything is
+ *     enqueued (the LLaMA-13B decode shape needs about 0.8 MB).
+ *   - The first call on a device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the array.  Each call clears the control words on `stream`
+ *     before its launch, so calls ordered on one stream are safe back to back; calls that can
+ *     overlap on the GPU (different streams, different host threads) race on the array and
+ *     must be serialised by the caller.
+ *   - The device-side status word lives in the array and is not visible to the caller; use
+ *     coopt_paged_decode where it must be read.
+ */
+#define COOPT_STATIC_SCRATCH_BYTES (4 * 1024 * 1024)
+int coopt_paged_decode_static(const coopt_cache* cache, const void* q, void* out, const int32_t* block_table,
+                              int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch,
+                              int32_t num_q_heads, float sm_scale, void* stream);
+
+/*
  * coopt_paged_chunked — Opt-Pa long-sequence path (abstract and conclusion: the context is
  * segmented into chunks that are processed independently and merged) and chunked prefill.
  *   cu_q_lens     DEVICE int32 [batch + 1], prefix sums of the number of query tokens per

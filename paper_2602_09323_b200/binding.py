@@ -43,6 +43,9 @@ _SIGNATURES = {
                                           ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32,
                                           ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
                                           ctypes.c_void_p]),
+    "coopt_paged_decode_static": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p,
+                                                 ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32,
+                                                 ctypes.c_int32, ctypes.c_float, ctypes.c_void_p]),
     "coopt_paged_chunked": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p,
                                            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p,
                                            ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32,
@@ -169,6 +172,22 @@ def paged_decode(cache: Cache, q: torch.Tensor, block_table: torch.Tensor, conte
                                            _ptr(context_lens), q.shape[0], q.shape[1], float(sm_scale),
                                            _ptr(workspace), workspace.numel(), _stream())
     _check(st, "coopt_paged_decode")
+    return out
+
+
+def paged_decode_static(cache: Cache, q: torch.Tensor, block_table: torch.Tensor, context_lens: torch.Tensor,
+                        sm_scale: float, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """coopt_paged_decode_static: as ``paged_decode`` but the scratch memory is the fixed array inside
+    the library, for callers that cannot allocate a workspace (see the header).  ``out`` is still the
+    caller's; pass one in if even the output must not be allocated here."""
+    assert q.dtype == torch.bfloat16 and q.is_contiguous() and q.is_cuda
+    assert block_table.dtype == torch.int32 and block_table.is_contiguous() and context_lens.dtype == torch.int32
+    if out is None:
+        out = torch.empty_like(q)
+    st = load_library().coopt_paged_decode_static(cache.ref(), _ptr(q), _ptr(out), _ptr(block_table),
+                                                  block_table.shape[1], _ptr(context_lens), q.shape[0], q.shape[1],
+                                                  float(sm_scale), _stream())
+    _check(st, "coopt_paged_decode_static")
     return out
 
 
