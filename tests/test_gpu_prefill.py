@@ -1,0 +1,87 @@
+"""GPU parity: coopt_paged_chunked with runs of several query tokens per sequence (chunked prefill on
+tensor cores) against the float64 oracle evaluated on the oracle's own cache."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import attention, kv_cache
+from paper_2602_09323_b200 import binding, workloads
+from tests import helpers
+
+pytestmark = pytest.mark.gpu
+
+
+def _gpu_prefill(w, cache, causal=True):
+    ws = binding.new_workspace(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_table.shape[1], 2048,
+                               sum(w.q_lens))
+    out = binding.paged_chunked(cache, w.q.cuda(), w.cu_q_lens.cuda(), w.block_table.cuda(),
+                                w.context_lens_tensor.cuda(), 2048, causal, w.sm_scale, ws)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    return out
+
+
+def _oracle(w, causal=True, pairs=None):
+    codes, scales = helpers.oracle_fp8_cache(w)
+    return attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), w.context_lens,
+                                     cu_q_lens=w.cu_q_lens.numpy(), causal=causal, pairs=pairs)
+
+
+@pytest.mark.parametrize("hq,hkv,d", [(8, 2, 64), (10, 2, 128), (8, 8, 128), (16, 2, 64), (3, 1, 128)])
+@pytest.mark.parametrize("causal", [True, False])
+def test_ragged_query_runs_group_sizes_and_head_dims(hq, hkv, d, causal):
+    lens = [70, 333, 16, 129, 1, 200]
+    q_lens = [70, 40, 3, 129, 1, 7]          # whole-sequence prefill, partial runs, single tokens
+    w = workloads.make_workload("prefill", lens, hq, hkv, d, seed=hq + d, q_lens=q_lens)
+    out = _gpu_prefill(w, helpers.gpu_fill(w), causal)
+    helpers.check_attention(out, _oracle(w, causal), what=f"prefill hq{hq} hkv{hkv} d{d} causal={causal}")
+
+
+def test_rows_past_the_tile_and_tail_positions_are_left_alone():
+    w = workloads.make_workload("guard", [500, 77], 10, 2, 128, seed=4, q_lens=[130, 77])
+    cache = helpers.gpu_fill(w)
+    want = _gpu_prefill(w, cache)
+    total = sum(w.q_lens)
+    padded = torch.full((total + 2, 10, 128), 7.0, dtype=torch.bfloat16, device="cuda")
+    ws = binding.new_workspace(w.batch, 10, 2, 128, w.block_table.shape[1], 2048, total)
+    binding.paged_chunked(cache, w.q.cuda(), w.cu_q_lens.cuda(), w.block_table.cuda(), w.context_lens_tensor.cuda(),
+                          2048, True, w.sm_scale, ws, out=padded[1:-1])
+    torch.cuda.synchronize()
+    assert torch.equal(padded[1:-1], want) and (padded[0] == 7).all() and (padded[-1] == 7).all()
+
+
+def test_causal_row_equals_decode_over_the_truncated_context():
+    """Row i of a causal run sees exactly what a decode call with context L - n + i + 1 sees."""
+    L, n = 300, 37
+    w = workloads.make_workload("rowdec", [L], 8, 2, 128, seed=11, q_lens=[n])
+    cache = helpers.gpu_fill(w)
+    out = _gpu_prefill(w, cache)
+    ws = binding.new_workspace(1, 8, 2, 128, w.block_table.shape[1])
+    for i in (0, 5, n - 1):
+        lens = torch.tensor([L - n + i + 1], dtype=torch.int32).cuda()
+        dec = binding.paged_decode(cache, w.q[i:i + 1].cuda(), w.block_table.cuda(), lens, w.sm_scale, ws)
+        torch.cuda.synchronize()
+        diff = (dec[0].float() - out[i].float()).abs()
+        assert float((diff - 2.0 ** -7 * out[i].float().abs()).max()) <= 5e-3
+
+
+def test_chunked_prefill_full_size_sampled():
+    """BASELINE configuration 5 at full size: 8 sequences, 4096 cached + 512 new tokens, causal; the
+    oracle recomputes a sample of (query row, query head) outputs from its own cache."""
+    w = workloads.config_chunked_prefill()
+    out = _gpu_prefill(w, helpers.gpu_fill(w))
+    assert torch.isfinite(out.float()).all()
+    rng = np.random.default_rng(2)
+    k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
+    ref = np.full((8 * 512, 40, 128), np.nan)
+    q = w.q.float().numpy()
+    for b, h in zip(rng.integers(0, 8, 4), rng.integers(0, 40, 4)):
+        rows_kv = slice(w.kv_offsets[b], w.kv_offsets[b] + 4608)
+        codes, scales = kv_cache.new_cache(w.num_blocks, 8, 128)
+        kv_cache.kv_write(codes, scales, k[rows_kv], v[rows_kv], slots[rows_kv], heads=[h // 5])
+        rows = [int(b) * 512 + int(i) for i in (0, 1, 24, 25, 255, 511, int(rng.integers(0, 512)))]
+        part = attention.paged_attention(q, (codes, scales), w.block_table.numpy(), w.context_lens,
+                                         cu_q_lens=w.cu_q_lens.numpy(), causal=True, pairs=[(r, int(h)) for r in rows])
+        for r in rows:
+            ref[r, h] = part[r, h]
+    helpers.check_attention(out, ref, what="chunked prefill full size")
