@@ -22,15 +22,16 @@
  *   block_size is 16 tokens.  FP8 E4M3 cache (COOPT_KV_FP8_E4M3):
  *       bytes  0..3   fp32 K scale of the granule     bytes 4..7  fp32 V scale
  *       bytes  8..31  zero
- *       bytes 32..32+16*D-1        K codes, 16 tokens x D, in tensor-core fragment order
- *       bytes 32+16*D..32+32*D-1   V codes, 16 tokens x D, in tensor-core fragment order
+ *       bytes 32..32+16*D-1        K codes: token t, dim d at (t/8)*8D + (d/16)*128 + (t%8)*16 + d%16
+ *       bytes 32+16*D..32+32*D-1   V codes, transposed: token t, dim d at (d/8)*128 + (d%8)*16 + t
  *   A dequantised element is decode_e4m3(code) * scale (Eq. 6).  A scale of 0 marks a
- *   granule that holds only zeros.  bf16 cache (COOPT_KV_BF16, the un-quantised ablation):
- *   no header; 16*D bf16 K values then 16*D bf16 V values, also in fragment order.
- *   "Fragment order" is a fixed permutation of (token, dim) inside the granule chosen so
- *   that a warp reads the operands of its matrix instructions with 16-byte loads;
- *   coopt_cache_offset() returns the byte offset of any element, which is all a caller
- *   needs to inspect or build a cache by hand.
+ *   granule that holds only zeros.  Both parts are laid out as the tensor cores read matrix
+ *   operands from shared memory (8 rows x 16 bytes form one contiguous 128-byte unit), so a part
+ *   needs one copy and no rearrangement on its way from HBM to the matrix instruction.
+ *   bf16 cache (COOPT_KV_BF16, the un-quantised ablation): no header; 16*D bf16 K values then
+ *   16*D bf16 V values, permuted into the register order of the warp-level matrix instruction.
+ *   coopt_cache_offset() returns the byte offset of any element, which is all a caller needs to
+ *   inspect or build a cache by hand.  Slots of a block past the context should hold finite codes.
  *   A cache that has never been written must be zero-filled once by the caller.
  */
 #ifndef COOPT_H_

@@ -15,13 +15,19 @@ constexpr int kFp8Header = 32;     // bytes in front of an FP8 granule: K scale,
 constexpr float kE4m3Max = 448.0f;
 
 // ---- cache layout ---------------------------------------------------------------------------
-// A granule holds 16 tokens x D of K and of V for one (block, kv head), permuted so that lane
-// `l` of a warp finds the B-operand registers of mma.m16n8k16 in consecutive 16-byte chunks:
+// A granule holds 16 tokens x D of K and of V for one (block, kv head).
+// FP8 granule: the layout the tensor cores read from shared memory without any rearrangement, so
+// that one bulk copy per part is all the staging there is.  Both parts are "K-major, no swizzle"
+// operands of tcgen05.mma: 8 rows x 16 bytes form a contiguous 128-byte core matrix.
+//   K part (rows = tokens, contraction over dims): token t, dim d at
+//       (t / 8) * 8D + (d / 16) * 128 + (t % 8) * 16 + d % 16
+//   V part (rows = dims, contraction over tokens; i.e. V transposed): token t, dim d at
+//       (d / 8) * 128 + (d % 8) * 16 + t
+// bf16 granule (ablation cache, mma.sync kernel): values permuted so that lane `l` of a warp finds
+// the B-operand registers of mma.m16n8k16 in consecutive 16-byte chunks:
 //   K tile (QK^T: n = token, k = dim):   lane = 4 * (token % 8) + (dim % 8) / 2
 //   V tile (P V : k = token, n = dim):   lane = 4 * (dim % 8)   + (token % 8) / 2
-// FP8: a 32-bit word holds the four codes a lane feeds to one k-step (K) or one n-tile (V),
-// in the order b0,b1,b2,b3 of the instruction; a 16-byte chunk holds four such words.
-// bf16: a 16-byte chunk holds two k-steps (K) or two n-tiles (V) of two registers each.
+// a chunk holds two k-steps (K) or two n-tiles (V) of two registers each.
 
 __host__ __device__ constexpr int granule_bytes(int D, bool fp8) {
   return fp8 ? kFp8Header + 2 * kBlockSize * D : 2 * kBlockSize * D * 2;
@@ -33,26 +39,20 @@ __host__ __device__ constexpr int part_offset(int D, bool fp8, int which) {
 
 // Byte offset of K element (token t, dim d) inside the K part.
 __host__ __device__ inline int k_elem_offset(int D, bool fp8, int t, int d) {
+  if (fp8) return (t >> 3) * 8 * D + (d >> 4) * 128 + (t & 7) * 16 + (d & 15);
   const int nt = t >> 3, n = t & 7;
   const int s = d >> 4, r = d & 15;
   const int c = (r & 7) >> 1;
   const int lane = 4 * n + c;
-  if (fp8) {
-    const int j = (r & 1) + 2 * (r >> 3);
-    return ((nt * (D / 64) + (s >> 2)) * 32 + lane) * 16 + (s & 3) * 4 + j;
-  }
   return ((nt * (D / 32) + (s >> 1)) * 32 + lane) * 16 + (s & 1) * 8 + (r >> 3) * 4 + (r & 1) * 2;
 }
 
 // Byte offset of V element (token t, dim d) inside the V part.
 __host__ __device__ inline int v_elem_offset(int D, bool fp8, int t, int d) {
+  if (fp8) return (d >> 3) * 128 + (d & 7) * 16 + t;
   const int n = d & 7;
   const int c = (t & 7) >> 1;
   const int lane = 4 * n + c;
-  if (fp8) {
-    const int j = (t & 1) + 2 * (t >> 3);
-    return ((d >> 5) * 32 + lane) * 16 + ((d & 31) >> 3) * 4 + j;
-  }
   return ((d >> 4) * 32 + lane) * 16 + ((d & 15) >> 3) * 8 + (t >> 3) * 4 + (t & 1) * 2;
 }
 

@@ -16,7 +16,7 @@
 // delivers the last piece of a (sequence, kv head) merges them by log-sum-exp and writes the
 // bf16 output.  The K scale of a granule factors out of the dot product and is applied to the
 // logits; the V scale is folded into the probabilities.
-#include "coopt_common.cuh"
+#include "coopt_plan.cuh"
 
 namespace coopt {
 
@@ -24,46 +24,8 @@ namespace {
 
 constexpr int kWarps = 8;
 constexpr int kThreads = kWarps * 32;
-constexpr int kCap = 2048;            // block ids staged in shared memory per round
-constexpr int kMaxSeg = 32;           // segments planned per round
-constexpr int kMaxBatch = 1024;
-constexpr int kMinBlocksPerCta = 16;
-constexpr int kMaxGroup = 8;
-constexpr int kCounterSlots = 16384;
-constexpr int kWsHeaderBytes = 256;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
-
-struct Segment {
-  int b, g;          // sequence, kv head
-  int j0, n;         // first block of the sequence in this segment, number of blocks
-  int list_off;      // position of block j0 in the staged id list
-  int partial;       // 0: covers the whole sequence, write the output directly
-  int slot;          // partial: workspace slot (decode mode) or chunk index (chunk mode)
-  int expected;      // partial: number of pieces the (sequence, kv head) is cut into
-  int seq_blocks;    // blocks of the whole sequence
-  int ctx_len;       // tokens of the whole sequence
-};
-
-struct DecodeParams {
-  const uint8_t* cache;
-  const __nv_bfloat16* q;
-  __nv_bfloat16* out;
-  const int* block_table;
-  const int* context_lens;
-  int max_blocks_per_seq;
-  int batch, num_q_heads, num_kv_heads, group;
-  int num_blocks;
-  float sm_scale_log2;     // sm_scale * log2(e)
-  int planned_ctas;        // P
-  int chunk_blocks;        // 0 = decode mode
-  int max_chunks;
-  int* status;
-  int* counters;
-  float* part_o;           // decode: [2P][G][D]        chunk: [B][Hq][max_chunks][D]
-  float* part_m;           // decode: [2P][G]           chunk: [B][Hq][max_chunks]
-  float* part_l;
-};
 
 template <int D, bool FP8>
 struct Cfg {
@@ -110,21 +72,6 @@ __device__ __forceinline__ void mma_top(float& d0, float& d1, uint32_t a0, uint3
   }
 }
 
-// Position of a flat block index in (sequence, kv head, block) order.
-struct Cursor {
-  int b, g, j;
-};
-
-__device__ __forceinline__ int find_seq(const int* pre, int batch, long long x, int heads) {
-  // largest b in [0, batch) with heads * pre[b] <= x
-  int lo = 0, hi = batch - 1;
-  while (lo < hi) {
-    const int mid = (lo + hi + 1) >> 1;
-    if (static_cast<long long>(heads) * pre[mid] <= x) lo = mid; else hi = mid - 1;
-  }
-  return lo;
-}
-
 template <int D, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeParams p) {
   using C = Cfg<D, FP8>;
@@ -143,36 +90,14 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
   const int B = p.batch, Hkv = p.num_kv_heads, G = p.group, Hq = p.num_q_heads;
   const bool chunk_mode = p.chunk_blocks > 0;
 
-  // ---- plan: blocks (and chunks) per sequence, prefix sums ------------------------------------
-  for (int b = tid; b < B; b += kThreads) {
-    int L = p.context_lens[b];
-    L = max(0, min(L, p.max_blocks_per_seq * kBlockSize));
-    const int nb = (L + kBlockSize - 1) / kBlockSize;
-    pre_blk[b + 1] = nb;
-    pre_unit[b + 1] = chunk_mode ? (nb + p.chunk_blocks - 1) / p.chunk_blocks : 0;
-  }
-  if (tid == 0) { pre_blk[0] = 0; pre_unit[0] = 0; }
-  __syncthreads();
-  if (warp == 0) {
-    int carry_b = 0, carry_u = 0;
-    for (int base = 0; base < B; base += 32) {
-      const int i = base + lane;
-      int vb = i < B ? pre_blk[i + 1] : 0, vu = i < B ? pre_unit[i + 1] : 0;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        const int tb = __shfl_up_sync(0xffffffffu, vb, o), tu = __shfl_up_sync(0xffffffffu, vu, o);
-        if (lane >= o) { vb += tb; vu += tu; }
-      }
-      if (i < B) { pre_blk[i + 1] = vb + carry_b; pre_unit[i + 1] = vu + carry_u; }
-      carry_b += __shfl_sync(0xffffffffu, vb, 31);
-      carry_u += __shfl_sync(0xffffffffu, vu, 31);
-    }
-  }
+  // ---- plan: blocks (and chunks) per sequence, this CTA's slice of the flat block list ---------
+  PlanSmem plan;
+  plan.pre_blk = pre_blk; plan.pre_unit = pre_unit; plan.segs = segs; plan.ids = ids; plan.misc = misc;
   if (tid == 0) {
     for (int i = 0; i < kWarps * C::kStages; ++i) mbar_init(&bars[i], 1);
     mbar_fence_init();
   }
-  __syncthreads();
+  plan_prefix(p, plan, tid, kThreads);
 
   // sequences with an empty context: all-zero output rows
   for (int b = blockIdx.x; b < B; b += gridDim.x) {
@@ -180,32 +105,10 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
       for (int i = tid; i < Hq * D; i += kThreads) p.out[static_cast<size_t>(b) * Hq * D + i] = __float2bfloat16(0.0f);
   }
 
-  const long long N = static_cast<long long>(Hkv) * pre_blk[B];
-  if (N == 0) return;
-  long long lo, hi;
-  int P;
-  if (!chunk_mode) {
-    P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), max(1ll, N / kMinBlocksPerCta)));
-    if (static_cast<int>(blockIdx.x) >= P) return;
-    lo = blockIdx.x * N / P;
-    hi = (blockIdx.x + 1ll) * N / P;
-  } else {
-    const long long U = static_cast<long long>(Hkv) * pre_unit[B];
-    P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), U));
-    if (static_cast<int>(blockIdx.x) >= P) return;
-    const long long ulo = blockIdx.x * U / P, uhi = (blockIdx.x + 1ll) * U / P;
-    auto unit_to_block = [&](long long u) -> long long {
-      if (u >= U) return N;
-      const int b = find_seq(pre_unit, B, u, Hkv);
-      const int nch = pre_unit[b + 1] - pre_unit[b], nb = pre_blk[b + 1] - pre_blk[b];
-      const long long rem = u - static_cast<long long>(Hkv) * pre_unit[b];
-      const int g = static_cast<int>(rem / nch), c = static_cast<int>(rem % nch);
-      return static_cast<long long>(Hkv) * pre_blk[b] + static_cast<long long>(g) * nb + static_cast<long long>(c) * p.chunk_blocks;
-    };
-    lo = unit_to_block(ulo);
-    hi = unit_to_block(uhi);
-  }
-  auto cta_of = [&](long long x) -> int { return static_cast<int>(((x + 1) * P - 1) / N); };
+  PlanSlice sl;
+  if (!plan_slice(p, plan, sl)) return;
+  const long long lo = sl.lo, hi = sl.hi;
+  auto cta_of = [&](long long x) -> int { return plan_cta_of(sl, x); };
 
   // ---- per-warp pipeline state (persists across rounds) ----------------------------------------
   uint8_t* my_ring = ring + warp * C::kStages * C::kGran;
@@ -216,70 +119,11 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
   long long x = lo;
   while (x < hi) {
     // ---- round: thread 0 plans up to kMaxSeg segments / kCap blocks starting at x -------------
-    if (tid == 0) {
-      int nseg = 0, used = 0;
-      long long xx = x;
-      Cursor cur;
-      cur.b = find_seq(pre_blk, B, xx, Hkv);
-      {
-        const int nb = pre_blk[cur.b + 1] - pre_blk[cur.b];
-        const long long rem = xx - static_cast<long long>(Hkv) * pre_blk[cur.b];
-        cur.g = static_cast<int>(rem / nb);
-        cur.j = static_cast<int>(rem % nb);
-      }
-      while (xx < hi && nseg < kMaxSeg) {
-        const int nb = pre_blk[cur.b + 1] - pre_blk[cur.b];
-        long long n = min(static_cast<long long>(nb - cur.j), hi - xx);
-        if (chunk_mode) n = min(n, static_cast<long long>(p.chunk_blocks - cur.j % p.chunk_blocks));
-        if (used + n > kCap) {
-          if (nseg > 0) break;
-          n = kCap;   // cannot happen with the host's sizing; keeps the kernel in bounds regardless
-        }
-        Segment s;
-        s.b = cur.b; s.g = cur.g; s.j0 = cur.j; s.n = static_cast<int>(n); s.list_off = used;
-        s.seq_blocks = nb;
-        s.ctx_len = max(0, min(p.context_lens[cur.b], p.max_blocks_per_seq * kBlockSize));
-        if (chunk_mode) {
-          s.partial = 1;
-          s.slot = cur.j / p.chunk_blocks;
-          s.expected = pre_unit[cur.b + 1] - pre_unit[cur.b];
-        } else {
-          s.partial = !(cur.j == 0 && n == nb);
-          s.slot = 2 * blockIdx.x + (cur.j > 0 ? 0 : 1);
-          const long long fs = static_cast<long long>(Hkv) * pre_blk[cur.b] + static_cast<long long>(cur.g) * nb;
-          s.expected = cta_of(fs + nb - 1) - cta_of(fs) + 1;
-        }
-        segs[nseg++] = s;
-        used += static_cast<int>(n);
-        xx += n;
-        cur.j += static_cast<int>(n);
-        if (cur.j >= nb) {
-          cur.j = 0;
-          if (++cur.g == Hkv) {
-            cur.g = 0;
-            ++cur.b;
-            while (cur.b < B && pre_blk[cur.b + 1] == pre_blk[cur.b]) ++cur.b;
-          }
-        }
-      }
-      misc[0] = nseg;
-      misc[1] = static_cast<int>(xx & 0xffffffffll);
-      misc[2] = static_cast<int>(xx >> 32);
-    }
+    if (tid == 0) plan_round(p, plan, sl, x);
     __syncthreads();
     const int nseg = misc[0];
     const long long x_next = (static_cast<long long>(misc[2]) << 32) | static_cast<unsigned int>(misc[1]);
-
-    // stage the physical block ids of every segment
-    for (int s = 0; s < nseg; ++s) {
-      const Segment& sg = segs[s];
-      const int* trow = p.block_table + static_cast<size_t>(sg.b) * p.max_blocks_per_seq + sg.j0;
-      for (int k = tid; k < sg.n; k += kThreads) {
-        int id = trow[k];
-        if (id < 0 || id >= p.num_blocks) { atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG); id = 0; }
-        ids[sg.list_off + k] = id;
-      }
-    }
+    plan_stage_ids(p, plan, nseg, tid, kThreads);
     __syncthreads();
 
     // ---- producer cursor of this warp: (segment, block-in-segment) --------------------------
@@ -635,6 +479,8 @@ static int launch_one(const DecodeParams& p, int grid, cudaStream_t stream) {
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
 
+int launch_paged_decode_umma(const DecodeParams& p, int head_dim, int grid, cudaStream_t stream);
+
 int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
                         int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
                         float sm_scale, int32_t chunk_size, void* workspace, int planned_ctas, cudaStream_t stream) {
@@ -670,9 +516,9 @@ int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const in
     p.part_m = p.part_o + rows * c->head_dim;
     p.part_l = p.part_m + rows;
   }
-  const bool fp8 = c->dtype == COOPT_KV_FP8_E4M3;
-  if (c->head_dim == 128) return fp8 ? launch_one<128, true>(p, planned_ctas, stream) : launch_one<128, false>(p, planned_ctas, stream);
-  return fp8 ? launch_one<64, true>(p, planned_ctas, stream) : launch_one<64, false>(p, planned_ctas, stream);
+  // FP8 cache: the tcgen05 kernel; bf16 ablation cache: the mma.sync kernel of this file
+  if (c->dtype == COOPT_KV_FP8_E4M3) return launch_paged_decode_umma(p, c->head_dim, planned_ctas, stream);
+  return c->head_dim == 128 ? launch_one<128, false>(p, planned_ctas, stream) : launch_one<64, false>(p, planned_ctas, stream);
 }
 
 }  // namespace coopt

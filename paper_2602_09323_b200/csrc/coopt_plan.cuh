@@ -1,0 +1,212 @@
+// Work decomposition shared by the decode kernels (Eq. 9: only the valid blocks of every sequence
+// are ever listed).  All (sequence, kv head, block) triples form one flat list.  In decode mode
+// CTA i takes the i-th of P equal slices of the list (split-KV balanced by bytes); in chunk mode
+// (Opt-Pa) it takes a contiguous run of fixed-size chunks.  A slice is cut into segments at
+// (sequence, kv head) boundaries and at chunk boundaries; a CTA walks its slice in rounds of at
+// most kMaxSeg segments / kCap blocks whose physical block ids are staged in shared memory.
+#pragma once
+
+#include "coopt_common.cuh"
+
+namespace coopt {
+
+constexpr int kCap = 2048;            // block ids staged in shared memory per round
+constexpr int kMaxSeg = 32;           // segments planned per round
+constexpr int kMaxBatch = 1024;
+constexpr int kMinBlocksPerCta = 16;
+constexpr int kMaxGroup = 8;
+constexpr int kCounterSlots = 16384;
+constexpr int kWsHeaderBytes = 256;
+
+struct Segment {
+  int b, g;          // sequence, kv head
+  int j0, n;         // first block of the sequence in this segment, number of blocks
+  int list_off;      // position of block j0 in the staged id list
+  int partial;       // 0: covers the whole sequence, write the output directly
+  int slot;          // partial: workspace slot (decode mode) or chunk index (chunk mode)
+  int expected;      // partial: number of pieces the (sequence, kv head) is cut into
+  int seq_blocks;    // blocks of the whole sequence
+  int ctx_len;       // tokens of the whole sequence
+};
+
+struct DecodeParams {
+  const uint8_t* cache;
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  const int* block_table;
+  const int* context_lens;
+  int max_blocks_per_seq;
+  int batch, num_q_heads, num_kv_heads, group;
+  int num_blocks;
+  float sm_scale_log2;     // sm_scale * log2(e)
+  int planned_ctas;        // P
+  int chunk_blocks;        // 0 = decode mode
+  int max_chunks;
+  int* status;
+  int* counters;
+  float* part_o;           // decode: [2P][G][D]        chunk: [B][Hq][max_chunks][D]
+  float* part_m;           // decode: [2P][G]           chunk: [B][Hq][max_chunks]
+  float* part_l;
+};
+
+#ifdef __CUDACC__
+
+// Shared-memory arrays of the planner; the kernel owns the storage.
+struct PlanSmem {
+  int* pre_blk;      // [kMaxBatch + 4] prefix sums of blocks per sequence
+  int* pre_unit;     // [kMaxBatch + 4] prefix sums of chunks per sequence (chunk mode)
+  Segment* segs;     // [kMaxSeg]
+  int* ids;          // [kCap]
+  int* misc;         // [4]: nseg, next x (lo, hi), scratch flag
+};
+
+__device__ __forceinline__ int plan_find_seq(const int* pre, int batch, long long x, int heads) {
+  // largest b in [0, batch) with heads * pre[b] <= x
+  int lo = 0, hi = batch - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi + 1) >> 1;
+    if (static_cast<long long>(heads) * pre[mid] <= x) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// Blocks (and chunks) per sequence and their prefix sums.  Every thread of the CTA calls this.
+__device__ inline void plan_prefix(const DecodeParams& p, const PlanSmem& s, int tid, int nthreads) {
+  const int B = p.batch;
+  const bool chunk_mode = p.chunk_blocks > 0;
+  for (int b = tid; b < B; b += nthreads) {
+    int L = p.context_lens[b];
+    L = max(0, min(L, p.max_blocks_per_seq * kBlockSize));
+    const int nb = (L + kBlockSize - 1) / kBlockSize;
+    s.pre_blk[b + 1] = nb;
+    s.pre_unit[b + 1] = chunk_mode ? (nb + p.chunk_blocks - 1) / p.chunk_blocks : 0;
+  }
+  if (tid == 0) { s.pre_blk[0] = 0; s.pre_unit[0] = 0; }
+  __syncthreads();
+  if (tid < 32) {
+    const int lane = tid;
+    int carry_b = 0, carry_u = 0;
+    for (int base = 0; base < B; base += 32) {
+      const int i = base + lane;
+      int vb = i < B ? s.pre_blk[i + 1] : 0, vu = i < B ? s.pre_unit[i + 1] : 0;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int tb = __shfl_up_sync(0xffffffffu, vb, o), tu = __shfl_up_sync(0xffffffffu, vu, o);
+        if (lane >= o) { vb += tb; vu += tu; }
+      }
+      if (i < B) { s.pre_blk[i + 1] = vb + carry_b; s.pre_unit[i + 1] = vu + carry_u; }
+      carry_b += __shfl_sync(0xffffffffu, vb, 31);
+      carry_u += __shfl_sync(0xffffffffu, vu, 31);
+    }
+  }
+  __syncthreads();
+}
+
+// The slice [lo, hi) of the flat block list that belongs to this CTA; false if it has none.
+struct PlanSlice {
+  long long lo, hi, N;
+  int P;
+};
+__device__ inline bool plan_slice(const DecodeParams& p, const PlanSmem& s, PlanSlice& sl) {
+  const int B = p.batch, Hkv = p.num_kv_heads;
+  sl.N = static_cast<long long>(Hkv) * s.pre_blk[B];
+  if (sl.N == 0) return false;
+  if (p.chunk_blocks == 0) {
+    sl.P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), max(1ll, sl.N / kMinBlocksPerCta)));
+    if (static_cast<int>(blockIdx.x) >= sl.P) return false;
+    sl.lo = blockIdx.x * sl.N / sl.P;
+    sl.hi = (blockIdx.x + 1ll) * sl.N / sl.P;
+    return true;
+  }
+  const long long U = static_cast<long long>(Hkv) * s.pre_unit[B];
+  sl.P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), U));
+  if (static_cast<int>(blockIdx.x) >= sl.P) return false;
+  const long long ulo = blockIdx.x * U / sl.P, uhi = (blockIdx.x + 1ll) * U / sl.P;
+  auto unit_to_block = [&](long long u) -> long long {
+    if (u >= U) return sl.N;
+    const int b = plan_find_seq(s.pre_unit, B, u, Hkv);
+    const int nch = s.pre_unit[b + 1] - s.pre_unit[b], nb = s.pre_blk[b + 1] - s.pre_blk[b];
+    const long long rem = u - static_cast<long long>(Hkv) * s.pre_unit[b];
+    const int g = static_cast<int>(rem / nch), c = static_cast<int>(rem % nch);
+    return static_cast<long long>(Hkv) * s.pre_blk[b] + static_cast<long long>(g) * nb + static_cast<long long>(c) * p.chunk_blocks;
+  };
+  sl.lo = unit_to_block(ulo);
+  sl.hi = unit_to_block(uhi);
+  return true;
+}
+// CTA that owns flat block index x (decode mode).
+__device__ __forceinline__ int plan_cta_of(const PlanSlice& sl, long long x) {
+  return static_cast<int>(((x + 1) * sl.P - 1) / sl.N);
+}
+
+// One thread plans the next round starting at flat index x: fills segs, misc[0] = number of
+// segments, misc[1..2] = where the following round starts.
+__device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, const PlanSlice& sl, long long x) {
+  const int B = p.batch, Hkv = p.num_kv_heads;
+  const bool chunk_mode = p.chunk_blocks > 0;
+  int nseg = 0, used = 0;
+  long long xx = x;
+  int cb = plan_find_seq(s.pre_blk, B, xx, Hkv), cg, cj;
+  {
+    const int nb = s.pre_blk[cb + 1] - s.pre_blk[cb];
+    const long long rem = xx - static_cast<long long>(Hkv) * s.pre_blk[cb];
+    cg = static_cast<int>(rem / nb);
+    cj = static_cast<int>(rem % nb);
+  }
+  while (xx < sl.hi && nseg < kMaxSeg) {
+    const int nb = s.pre_blk[cb + 1] - s.pre_blk[cb];
+    long long n = min(static_cast<long long>(nb - cj), sl.hi - xx);
+    if (chunk_mode) n = min(n, static_cast<long long>(p.chunk_blocks - cj % p.chunk_blocks));
+    if (used + n > kCap) {
+      if (nseg > 0) break;
+      n = kCap;   // cannot happen with the host's sizing; keeps the kernel in bounds regardless
+    }
+    Segment sg;
+    sg.b = cb; sg.g = cg; sg.j0 = cj; sg.n = static_cast<int>(n); sg.list_off = used;
+    sg.seq_blocks = nb;
+    sg.ctx_len = max(0, min(p.context_lens[cb], p.max_blocks_per_seq * kBlockSize));
+    if (chunk_mode) {
+      sg.partial = 1;
+      sg.slot = cj / p.chunk_blocks;
+      sg.expected = s.pre_unit[cb + 1] - s.pre_unit[cb];
+    } else {
+      sg.partial = !(cj == 0 && n == nb);
+      sg.slot = 2 * blockIdx.x + (cj > 0 ? 0 : 1);
+      const long long fs = static_cast<long long>(Hkv) * s.pre_blk[cb] + static_cast<long long>(cg) * nb;
+      sg.expected = plan_cta_of(sl, fs + nb - 1) - plan_cta_of(sl, fs) + 1;
+    }
+    s.segs[nseg++] = sg;
+    used += static_cast<int>(n);
+    xx += n;
+    cj += static_cast<int>(n);
+    if (cj >= nb) {
+      cj = 0;
+      if (++cg == Hkv) {
+        cg = 0;
+        ++cb;
+        while (cb < B && s.pre_blk[cb + 1] == s.pre_blk[cb]) ++cb;
+      }
+    }
+  }
+  s.misc[0] = nseg;
+  s.misc[1] = static_cast<int>(xx & 0xffffffffll);
+  s.misc[2] = static_cast<int>(xx >> 32);
+}
+
+// Physical block ids of every planned segment -> shared memory (range-checked: a bad id is
+// reported in the status word and replaced by block 0, never dereferenced).
+__device__ inline void plan_stage_ids(const DecodeParams& p, const PlanSmem& s, int nseg, int tid, int nthreads) {
+  for (int i = 0; i < nseg; ++i) {
+    const Segment& sg = s.segs[i];
+    const int* trow = p.block_table + static_cast<size_t>(sg.b) * p.max_blocks_per_seq + sg.j0;
+    for (int k = tid; k < sg.n; k += nthreads) {
+      int id = trow[k];
+      if (id < 0 || id >= p.num_blocks) { atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG); id = 0; }
+      s.ids[sg.list_off + k] = id;
+    }
+  }
+}
+
+#endif  // __CUDACC__
+
+}  // namespace coopt

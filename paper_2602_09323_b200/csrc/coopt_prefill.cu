@@ -9,7 +9,7 @@
 //   1. one lane per block starts a bulk async copy of the granule into a ring of raw stages
 //      (an mbarrier per stage counts the bytes);
 //   2. all threads widen the E4M3 codes of the stage to f16 (exact) into a double-buffered
-//      operand tile that keeps the cache's fragment order, twice as wide;
+//      operand tile laid out in the register order of the matrix instruction;
 //   3. every warp runs S = Q K^T and O += P V for its 16 rows on tensor cores
 //      (mma.sync m16n8k16, f16 operands, fp32 accumulators) with an online softmax in between.
 // The K scale of a block is applied to the logits of its 16 tokens and the V scale is folded
@@ -167,15 +167,18 @@ __global__ void __launch_bounds__(kPfThreads, 1) paged_prefill_kernel(const Pref
   float qs0 = p.sm_scale_log2, qs1 = p.sm_scale_log2;
   {
     uint32_t w0[kKSteps][2], w1[kKSteps][2];
-    const __nv_bfloat16* qp0 = p.q + grow0 * D + 2 * quad;
-    const __nv_bfloat16* qp1 = p.q + grow1 * D + 2 * quad;
+    // k-step s of the instruction covers dims 16s..16s+15; its logical k positions 2c, 2c+1 (registers
+    // a0/a1 and b0) stand for dims 16s + 4c + {0, 1}, positions 2c+8, 2c+9 (a2/a3 and b1) for dims
+    // 16s + 4c + {2, 3}: the order in which a 16-byte chunk of the cache's K part splits over a quad
+    const __nv_bfloat16* qp0 = p.q + grow0 * D + 4 * quad;
+    const __nv_bfloat16* qp1 = p.q + grow1 * D + 4 * quad;
     float am0 = 0.0f, am1 = 0.0f;
 #pragma unroll
     for (int s = 0; s < kKSteps; ++s)
 #pragma unroll
       for (int e = 0; e < 2; ++e) {
-        w0[s][e] = live0 ? *reinterpret_cast<const uint32_t*>(qp0 + 16 * s + 8 * e) : 0u;
-        w1[s][e] = live1 ? *reinterpret_cast<const uint32_t*>(qp1 + 16 * s + 8 * e) : 0u;
+        w0[s][e] = live0 ? *reinterpret_cast<const uint32_t*>(qp0 + 16 * s + 2 * e) : 0u;
+        w1[s][e] = live1 ? *reinterpret_cast<const uint32_t*>(qp1 + 16 * s + 2 * e) : 0u;
         am0 = fmaxf(am0, fmaxf(fabsf(bf16_lo(w0[s][e])), fabsf(bf16_hi(w0[s][e]))));
         am1 = fmaxf(am1, fmaxf(fabsf(bf16_lo(w1[s][e])), fabsf(bf16_hi(w1[s][e]))));
       }
@@ -218,27 +221,44 @@ __global__ void __launch_bounds__(kPfThreads, 1) paged_prefill_kernel(const Pref
     uint8_t* cv = conv + buf * C::kConvTile;
     const int nb = min(kTileBlocks, n_blocks - tile * kTileBlocks);
 
-    // ---- widen the stage's codes to f16, fragment order kept ------------------------------------
+    // ---- widen the stage's codes to f16 and put them in the register order of mma.m16n8k16 --------
+    // A 16-byte chunk of the K part is one token x 16 dims, of the V part one dim x 16 tokens; either
+    // way it feeds the four lanes of one quad with two registers each.
     if (ok) {
       const uint8_t* rs = raw + stage * C::kRawStage;
 #pragma unroll
       for (int c = tid; c < kTileBlocks * C::kChunksPerBlock; c += kPfThreads) {
         const int jb = c / C::kChunksPerBlock, cc = c % C::kChunksPerBlock;
         uint4 w = make_uint4(0u, 0u, 0u, 0u);
-        if (jb < nb) {
-          w = lds128(rs + jb * C::kGran + kFp8Header + cc * 16);
+        if (jb < nb) w = lds128(rs + jb * C::kGran + kFp8Header + cc * 16);
+        uint8_t* dst;
+        uint32_t b0[4], b1[4];
+        if (cc < D) {
+          const int rg = cc / (D / 2), rem = cc % (D / 2), u = rem >> 3, n = rem & 7;   // token 8 rg + n, dims 16u..16u+15
+          dst = cv + jb * C::kConvBlock + (rg * (D / 64) + (u >> 2)) * 1024 + ((u & 3) >> 1) * 512 + (4 * n) * 16 + (u & 1) * 8;
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+          for (int q = 0; q < 4; ++q) { b0[q] = e4m3x2_to_f16x2_lo(ww[q]); b1[q] = e4m3x2_to_f16x2_hi(ww[q]); }
+        } else {
+          const int d = cc - D, j = d >> 3, n = d & 7;                                  // dim d, tokens 0..15
           const int tok0 = (tile * kTileBlocks + jb) * kBlockSize;
-          if (cc >= D && tok0 + kBlockSize > L) {
+          if (jb < nb && tok0 + kBlockSize > L) {
             // V codes of slots past the context are cleared so that stale bytes cannot reach P V
-            const int nvalid = L - tok0, c2 = 2 * (cc & 3);
-            const uint32_t vm = (c2 < nvalid ? 0x000000FFu : 0u) | (c2 + 1 < nvalid ? 0x0000FF00u : 0u) |
-                                (c2 + 8 < nvalid ? 0x00FF0000u : 0u) | (c2 + 9 < nvalid ? 0xFF000000u : 0u);
-            w.x &= vm; w.y &= vm; w.z &= vm; w.w &= vm;
+            const int keep = L - tok0;
+            uint32_t* wm = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const int left = keep - 4 * q;
+              wm[q] &= left >= 4 ? 0xFFFFFFFFu : (left <= 0 ? 0u : (1u << (8 * left)) - 1u);
+            }
           }
+          dst = cv + jb * C::kConvBlock + (D / 32) * 1024 + (j >> 2) * 1024 + ((j & 3) >> 1) * 512 + (4 * n) * 16 + (j & 1) * 8;
+          // lane c of the quad: b0 = tokens 2c, 2c+1, b1 = tokens 2c+8, 2c+9
+          b0[0] = e4m3x2_to_f16x2_lo(w.x); b0[1] = e4m3x2_to_f16x2_hi(w.x); b0[2] = e4m3x2_to_f16x2_lo(w.y); b0[3] = e4m3x2_to_f16x2_hi(w.y);
+          b1[0] = e4m3x2_to_f16x2_lo(w.z); b1[1] = e4m3x2_to_f16x2_hi(w.z); b1[2] = e4m3x2_to_f16x2_lo(w.w); b1[3] = e4m3x2_to_f16x2_hi(w.w);
         }
-        uint8_t* dst = cv + jb * C::kConvBlock + (cc >> 5) * 1024 + (cc & 31) * 16;
-        sts128(dst, make_uint4(e4m3x2_to_f16x2_lo(w.x), e4m3x2_to_f16x2_hi(w.x), e4m3x2_to_f16x2_lo(w.y), e4m3x2_to_f16x2_hi(w.y)));
-        sts128(dst + 512, make_uint4(e4m3x2_to_f16x2_lo(w.z), e4m3x2_to_f16x2_hi(w.z), e4m3x2_to_f16x2_lo(w.w), e4m3x2_to_f16x2_hi(w.w)));
+#pragma unroll
+        for (int q = 0; q < 4; ++q) *reinterpret_cast<uint2*>(dst + q * 16) = make_uint2(b0[q], b1[q]);
       }
       if (tid < kTileBlocks * 2) {
         const int jb = tid >> 1;

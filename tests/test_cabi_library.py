@@ -71,19 +71,28 @@ def test_layout_is_a_bijection_inside_each_granule(lib, head_dim, dtype):
     assert binding.cache_offset(c, 0, 0, 2, 0, 0) == -1 and binding.cache_offset(c, 0, 0, 0, 0, head_dim) == -1
 
 
-def test_fragment_order_serves_16_byte_loads(lib):
-    """A lane's operands for four k-steps (K) or four n-tiles (V) share one 16-byte chunk."""
-    c = _FakeCache(128, binding.KV_FP8_E4M3)
+def test_fp8_parts_are_tensor_core_operands_in_place(lib):
+    """FP8 granule: both parts are K-major operands made of 8-row x 16-byte core matrices, K with tokens
+    as rows (contraction over dims), V transposed with dims as rows (contraction over tokens)."""
+    for D in (64, 128):
+        c = _FakeCache(D, binding.KV_FP8_E4M3)
+        k0 = binding.cache_offset(c, 0, 0, 0, 0, 0)
+        v0 = binding.cache_offset(c, 0, 0, 1, 0, 0)
+        assert k0 == 32 and v0 == 32 + 16 * D
+        for t in (0, 5, 8, 15):
+            for d in (0, 1, 15, 16, 37, D - 1):
+                assert binding.cache_offset(c, 0, 0, 0, t, d) - k0 == (t // 8) * 8 * D + (d // 16) * 128 + (t % 8) * 16 + d % 16
+                assert binding.cache_offset(c, 0, 0, 1, t, d) - v0 == (d // 8) * 128 + (d % 8) * 16 + t
+
+
+def test_bf16_fragment_order_serves_16_byte_loads(lib):
+    """bf16 granule: a lane's operands for two k-steps (K) or two n-tiles (V) share one 16-byte chunk."""
+    c = _FakeCache(128, binding.KV_BF16)
     for token in (0, 5, 11):
         for quad in range(4):
-            dims = [16 * s + 2 * quad + e for s in range(4) for e in (0, 1, 8, 9)]
+            dims = [16 * s + 2 * quad + e for s in range(2) for e in (0, 1, 8, 9)]
             offs = [binding.cache_offset(c, 0, 0, 0, token, d) for d in dims]
-            assert offs == list(range(offs[0], offs[0] + 16)) and offs[0] % 16 == 0
-    for dim in (0, 7, 40):
-        for quad in range(4):
-            toks = [2 * quad, 2 * quad + 1, 2 * quad + 8, 2 * quad + 9]
-            offs = [binding.cache_offset(c, 0, 0, 1, t, dim) for t in toks]
-            assert offs == list(range(offs[0], offs[0] + 4)) and offs[0] % 4 == 0
+            assert offs == list(range(offs[0], offs[0] + 16, 2)) and offs[0] % 16 == 0
 
 
 def test_sizes_and_host_side_argument_checks(lib):

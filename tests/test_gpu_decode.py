@@ -91,6 +91,31 @@ def test_block_permutation_invariance_determinism_and_guard_bytes():
     assert torch.equal(padded[1:-1], out1) and (padded[0] == 7).all() and (padded[-1] == 7).all()
 
 
+def test_cold_l2_and_poisoned_workspace_do_not_change_the_result():
+    """Timing must not matter: evict L2 before the call (all loads come from HBM, so the copy ring runs
+    dry and the roles of the kernel meet in a different order) and fill the partials area of the
+    workspace with NaN patterns (a piece that is merged before it was written would show)."""
+    w = workloads.make_workload("cold", [700, 15, 2000], 8, 8, 64, seed=0)
+    cache = helpers.gpu_fill(w)
+    ref = _oracle_out(w)
+    q, table, lens = w.q.cuda(), w.block_table.cuda(), w.context_lens_tensor.cuda()
+    outs = []
+    for rep in range(3):
+        n = binding.workspace_bytes(w.batch, 8, 8, 64, w.block_table.shape[1])
+        ws = torch.empty(n, dtype=torch.uint8, device="cuda")
+        ws.view(torch.int32)[:] = 0x7FC00000
+        binding.workspace_init(ws)
+        junk = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+        junk.fill_(rep)                                    # larger than L2: evicts the cache and the queries
+        del junk
+        out = binding.paged_decode(cache, q, table, lens, w.sm_scale, ws)
+        torch.cuda.synchronize()
+        assert binding.workspace_status(ws) == 0
+        helpers.check_attention(out, ref, what=f"cold rep {rep}")
+        outs.append(out)
+    assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
+
+
 def test_llama13b_decode_full_size_sampled():
     """BASELINE configuration 2 at full size, in the launch configuration the benchmark times;
     the oracle recomputes a sample of (sequence, query head) outputs from its own cache."""
