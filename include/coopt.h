@@ -19,11 +19,11 @@
  * Cache layout (DEVICE memory, `coopt_cache.data`)
  *   The cache is an array of granules, one per (physical block, kv head):
  *       granule(blk, h) starts at byte (blk * num_kv_heads + h) * coopt_granule_bytes().
- *   block_size is 16 tokens.  FP8 E4M3 cache (COOPT_KV_FP8_E4M3):
- *       bytes  0..3   fp32 K scale of the granule     bytes 4..7  fp32 V scale
- *       bytes  8..31  zero
- *       bytes 32..32+16*D-1        K codes: token t, dim d at (t/8)*8D + (d/16)*128 + (t%8)*16 + d%16
- *       bytes 32+16*D..32+32*D-1   V codes, transposed: token t, dim d at (d/8)*128 + (d%8)*16 + t
+ *   block_size is 16 tokens.  FP8 E4M3 cache (COOPT_KV_FP8_E4M3), D = head_dim:
+ *       bytes 0..16*D-1        K codes: token t, dim d at (t/8)*8D + (d/16)*128 + (t%8)*16 + d%16
+ *       bytes 16*D..32*D-1     V codes, transposed: token t, dim d at (d/8)*128 + (d%8)*16 + t
+ *       bytes 32*D..32*D+3     fp32 K scale of the granule     bytes 32*D+4..32*D+7  fp32 V scale
+ *       bytes 32*D+8..32*D+31  zero
  *   A dequantised element is decode_e4m3(code) * scale (Eq. 6).  A scale of 0 marks a
  *   granule that holds only zeros.  Both parts are laid out as the tensor cores read matrix
  *   operands from shared memory (8 rows x 16 bytes form one contiguous 128-byte unit), so a part

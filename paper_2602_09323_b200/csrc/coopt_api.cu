@@ -111,7 +111,7 @@ int64_t coopt_cache_offset(const coopt_cache* c, int32_t block, int32_t kv_head,
 int64_t coopt_scale_offset(const coopt_cache* c, int32_t block, int32_t kv_head, int32_t which) {
   if (!c || !cache_shape_ok(c->head_dim, c->block_size, c->dtype) || c->dtype != COOPT_KV_FP8_E4M3) return -1;
   if (block < 0 || block >= c->num_blocks || kv_head < 0 || kv_head >= c->num_kv_heads || which < 0 || which > 1) return -1;
-  return (static_cast<int64_t>(block) * c->num_kv_heads + kv_head) * granule_bytes(c->head_dim, true) + 4 * which;
+  return (static_cast<int64_t>(block) * c->num_kv_heads + kv_head) * granule_bytes(c->head_dim, true) + header_offset(c->head_dim) + 4 * which;
 }
 
 int coopt_kv_write(const coopt_cache* cache, const void* k, const void* v, int64_t kv_token_stride,

@@ -11,13 +11,14 @@
 namespace coopt {
 
 constexpr int kBlockSize = 16;     // tokens per physical block
-constexpr int kFp8Header = 32;     // bytes in front of an FP8 granule: K scale, V scale, zeros
+constexpr int kFp8Header = 32;     // bytes behind the codes of an FP8 granule: K scale, V scale, zeros
 constexpr float kE4m3Max = 448.0f;
 
 // ---- cache layout ---------------------------------------------------------------------------
 // A granule holds 16 tokens x D of K and of V for one (block, kv head).
-// FP8 granule: the layout the tensor cores read from shared memory without any rearrangement, so
-// that one bulk copy per part is all the staging there is.  Both parts are "K-major, no swizzle"
+// FP8 granule: K part, V part, then the 32-byte header with the two scales (the V part and the header
+// travel in one copy).  The parts have the layout the tensor cores read from shared memory without any
+// rearrangement, so that a bulk copy is all the staging there is.  Both parts are "K-major, no swizzle"
 // operands of tcgen05.mma: 8 rows x 16 bytes form a contiguous 128-byte core matrix.
 //   K part (rows = tokens, contraction over dims): token t, dim d at
 //       (t / 8) * 8D + (d / 16) * 128 + (t % 8) * 16 + d % 16
@@ -33,9 +34,9 @@ __host__ __device__ constexpr int granule_bytes(int D, bool fp8) {
   return fp8 ? kFp8Header + 2 * kBlockSize * D : 2 * kBlockSize * D * 2;
 }
 __host__ __device__ constexpr int part_bytes(int D, bool fp8) { return kBlockSize * D * (fp8 ? 1 : 2); }
-__host__ __device__ constexpr int part_offset(int D, bool fp8, int which) {
-  return (fp8 ? kFp8Header : 0) + which * part_bytes(D, fp8);
-}
+__host__ __device__ constexpr int part_offset(int D, bool fp8, int which) { return which * part_bytes(D, fp8); }
+// FP8 granule: [K codes 16D][V codes 16D][fp32 K scale, fp32 V scale, 24 zero bytes]
+__host__ __device__ constexpr int header_offset(int D) { return 2 * kBlockSize * D; }
 
 // Byte offset of K element (token t, dim d) inside the K part.
 __host__ __device__ inline int k_elem_offset(int D, bool fp8, int t, int d) {

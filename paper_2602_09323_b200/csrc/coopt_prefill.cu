@@ -67,10 +67,6 @@ __device__ __forceinline__ float quad_sum(float x) {
   x += __shfl_xor_sync(0xffffffffu, x, 1);
   return x + __shfl_xor_sync(0xffffffffu, x, 2);
 }
-__device__ __forceinline__ void sts128(void* p, uint4 v) {
-  asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(smem_u32(p)), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
 template <int D>
 __global__ void __launch_bounds__(kPfThreads, 1) paged_prefill_kernel(const PrefillParams p) {
   using C = PfCfg<D>;
@@ -230,7 +226,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) paged_prefill_kernel(const Pref
       for (int c = tid; c < kTileBlocks * C::kChunksPerBlock; c += kPfThreads) {
         const int jb = c / C::kChunksPerBlock, cc = c % C::kChunksPerBlock;
         uint4 w = make_uint4(0u, 0u, 0u, 0u);
-        if (jb < nb) w = lds128(rs + jb * C::kGran + kFp8Header + cc * 16);
+        if (jb < nb) w = lds128(rs + jb * C::kGran + cc * 16);
         uint8_t* dst;
         uint32_t b0[4], b1[4];
         if (cc < D) {
@@ -263,7 +259,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) paged_prefill_kernel(const Pref
       if (tid < kTileBlocks * 2) {
         const int jb = tid >> 1;
         tile_scales[buf * kTileBlocks * 2 + tid] =
-            jb < nb ? reinterpret_cast<const float*>(rs + jb * C::kGran)[tid & 1] : 0.0f;
+            jb < nb ? reinterpret_cast<const float*>(rs + jb * C::kGran + header_offset(D))[tid & 1] : 0.0f;
       }
     }
     // operand tile complete, raw stage free again; a wait that ran out ends the walk for everyone

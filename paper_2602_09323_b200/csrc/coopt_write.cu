@@ -78,7 +78,7 @@ __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WritePar
   for (int t = 0; t < n; ++t) fresh |= (group.off[t] == 0);
 
   uint8_t* gran = p.cache + (static_cast<size_t>(group.blk) * p.num_kv_heads + h) * granule_bytes(D, true);
-  float* scales = reinterpret_cast<float*>(gran);
+  float* scales = reinterpret_cast<float*>(gran + header_offset(D));
   uint8_t* st = stage[warp];
 
 #pragma unroll 1

@@ -51,8 +51,8 @@ def test_layout_is_a_bijection_inside_each_granule(lib, head_dim, dtype):
     c = _FakeCache(head_dim, dtype)
     gran = lib.coopt_granule_bytes(head_dim, dtype)
     esize = 1 if dtype == binding.KV_FP8_E4M3 else 2
-    header = 32 if dtype == binding.KV_FP8_E4M3 else 0
-    assert gran == header + 2 * 16 * head_dim * esize
+    header = 0                                   # the FP8 header sits behind the codes
+    assert gran == (32 if dtype == binding.KV_FP8_E4M3 else 0) + 2 * 16 * head_dim * esize
     assert lib.coopt_cache_bytes(3, 2, head_dim, dtype) == 3 * 2 * gran
     for blk, h in [(0, 0), (2, 1)]:
         base = (blk * 2 + h) * gran
@@ -66,7 +66,7 @@ def test_layout_is_a_bijection_inside_each_granule(lib, head_dim, dtype):
                     seen.add(off)
         assert len(seen) == 2 * 16 * head_dim
         if dtype == binding.KV_FP8_E4M3:
-            assert binding.scale_offset(c, blk, h, 0) == base and binding.scale_offset(c, blk, h, 1) == base + 4
+            assert binding.scale_offset(c, blk, h, 0) == base + 32 * head_dim and binding.scale_offset(c, blk, h, 1) == base + 32 * head_dim + 4
     assert binding.cache_offset(c, 3, 0, 0, 0, 0) == -1 and binding.cache_offset(c, 0, 0, 0, 16, 0) == -1
     assert binding.cache_offset(c, 0, 0, 2, 0, 0) == -1 and binding.cache_offset(c, 0, 0, 0, 0, head_dim) == -1
 
@@ -78,7 +78,7 @@ def test_fp8_parts_are_tensor_core_operands_in_place(lib):
         c = _FakeCache(D, binding.KV_FP8_E4M3)
         k0 = binding.cache_offset(c, 0, 0, 0, 0, 0)
         v0 = binding.cache_offset(c, 0, 0, 1, 0, 0)
-        assert k0 == 32 and v0 == 32 + 16 * D
+        assert k0 == 0 and v0 == 16 * D and binding.scale_offset(c, 0, 0, 0) == 32 * D
         for t in (0, 5, 8, 15):
             for d in (0, 1, 15, 16, 37, D - 1):
                 assert binding.cache_offset(c, 0, 0, 0, t, d) - k0 == (t // 8) * 8 * D + (d // 16) * 128 + (t % 8) * 16 + d % 16
