@@ -156,7 +156,7 @@ int coopt_paged_decode_static(const coopt_cache* cache, const void* q, void* out
  *                 sequence; q/out are bf16 [cu_q_lens[batch]][num_q_heads][head_dim]
  *   context_lens  include the new tokens; the n query tokens of a sequence are its last n
  *                 positions and, when causal != 0, query i sees positions 0..len-n+i
- *   chunk_size    tokens per chunk, a multiple of 16, at most 32768
+ *   chunk_size    tokens per chunk, a multiple of 16, at most 16384
  *   total_q       cu_q_lens[batch] as known by the host (sizes the launch)
  * When every sequence has exactly one query token (total_q == batch) each chunk c of
  * (sequence b, query head h) produces m_c (max logit, natural-log units after sm_scale),

@@ -40,8 +40,8 @@ namespace {
 
 constexpr int kTeamThreads = 128;                     // four warps: one per 32 tensor-memory lanes
 constexpr int kSmThreads = 2 * kTeamThreads;          // warps 0-7
-constexpr int kProducerWarp = 8, kMmaWarp = 9;
-constexpr int kUmmaThreads = 320;
+constexpr int kProducerWarp = 8, kMmaWarp = 9, kEpilogueWarp = 10;
+constexpr int kUmmaThreads = 352;
 constexpr int kTileBlocks = 8;
 constexpr int kTileTokens = kTileBlocks * kBlockSize;  // 128
 constexpr float kLn2 = 0.6931471805599453f;
@@ -53,7 +53,7 @@ struct UCfg {
   static constexpr int kPart = kBlockSize * D;                 // K (or V) codes of one granule
   static constexpr int kVSlot = kPart + kFp8Header;            // V codes and the header of one granule: one copy
   static constexpr int kGMax = NP == 16 ? 5 : 8;               // head slots per probability term
-  static constexpr int kTmemCols = 128;                        // 4 x 16 logits columns + 2 x NP output columns
+  static constexpr int kTmemCols = NP == 16 ? 128 : 256;       // 4 x 16 logits columns + 4 x NP output columns
   static constexpr int kStages = D == 128 ? (NP == 16 ? 6 : 5) : 8;
   static constexpr int kKArea = kTileBlocks * kPart;
   static constexpr int kVArea = kTileBlocks * kVSlot + (D == 64 ? kPart : 0);   // D = 64: rows 64..127 of the 128-row operand read on
@@ -65,7 +65,7 @@ struct UCfg {
   static constexpr int kRingOff = 0;
   static constexpr int kQOff = kRingOff + kStages * kStageBytes;
   static constexpr int kPOff = kQOff + 2 * kQBytes;
-  static constexpr int kIdsOff = kPOff + 2 * kPBytes;
+  static constexpr int kIdsOff = kPOff + 4 * kPBytes;
   static constexpr int kPreBlkOff = kIdsOff + kCap * 4;
   static constexpr int kPreUnitOff = kPreBlkOff + (kMaxBatch + 4) * 4;
   static constexpr int kSegOff = kPreUnitOff + (kMaxBatch + 4) * 4;
@@ -74,7 +74,7 @@ struct UCfg {
   // int red_max [2 teams][4 warps][12], float red_sum [2][4][8], uint red_q [4][8], float qscale [2][8]
   static constexpr int kRedBytes = (2 * 4 * 12 + 2 * 4 * 8 + 4 * 8 + 2 * 8) * 4;
   static constexpr int kBarOff = kRedOff + kRedBytes;
-  static constexpr int kNumBars = 2 * kStages + 4 + 4 + 3 * 2;
+  static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kSmemBytes = kMiscOff + 64;
   static_assert(kStageBytes % 16 == 0 && kVSlot % 16 == 0, "bulk copies need 16-byte granularity");
@@ -128,22 +128,23 @@ __device__ __forceinline__ bool barrier_or(int id, int count, bool flag) {
                : "=r"(r) : "r"(id), "r"(count), "r"(static_cast<uint32_t>(flag)) : "memory");
   return r != 0;
 }
-// Non-blocking look at a phase of an mbarrier.  The waits of this kernel are short and sit on the
-// critical path between the roles, so they poll instead of letting the hardware park the thread.
+// Non-blocking look at a phase of an mbarrier: the instruction-issuing lane polls with it, because it
+// always has something else to look at.
 __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
   uint32_t ok;
   asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait that also gives up when another role has already given up.  The clock and the abort
-// flag are looked at once in 4096 unsuccessful polls, so the common short wait costs nothing extra.
+// Bounded wait that also gives up when another role has already given up.  try_wait lets the hardware
+// park the warp, so waiting warps do not take issue slots from the two single-lane roles that share
+// their schedulers.  The clock and the abort flag are looked at once in 256 unsuccessful tries.
 __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
   uint64_t t0 = 0;
 #pragma unroll 1
-  for (uint32_t polls = 1;; ++polls) {
-    if (mbar_test(bar, parity)) return true;
-    if ((polls & 0xFFFu) == 0) {
+  for (uint32_t tries = 1;; ++tries) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((tries & 0xFFu) == 0) {
       if (*abort_flag != 0) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
@@ -194,7 +195,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   plan.pre_blk = reinterpret_cast<int*>(smem + C::kPreBlkOff);
   plan.pre_unit = reinterpret_cast<int*>(smem + C::kPreUnitOff);
   plan.segs = reinterpret_cast<Segment*>(smem + C::kSegOff);
-  plan.misc = reinterpret_cast<int*>(smem + C::kMiscOff);          // [0..2] planner, [3] last-arriver flag
+  plan.misc = reinterpret_cast<int*>(smem + C::kMiscOff);          // [0..2] planner
   float* xch = reinterpret_cast<float*>(smem + C::kXchOff);         // [2 segment parities][kXchFloats]
   int* red_max = reinterpret_cast<int*>(smem + C::kRedOff);         // [2][4][12] per-warp maxima of a tile (ordered ints)
   float* red_sum = reinterpret_cast<float*>(red_max + 2 * 4 * 12);  // [2][4][8]
@@ -205,9 +206,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   uint64_t* bar_empty = bar_full + C::kStages;      // [kStages] the P V instructions of the tile in this stage are done
   uint64_t* bar_sfull = bar_empty + C::kStages;     // [4] logits of a tile are in tensor memory (buffer = tile & 3)
   uint64_t* bar_sfree = bar_sfull + 4;              // [4] the team's four warps have read them
-  uint64_t* bar_pfull = bar_sfree + 4;              // [2] probabilities of a tile are in shared memory
-  uint64_t* bar_ofree = bar_pfull + 2;              // [2] the team has folded the output buffer into its registers
-  uint64_t* bar_qfull = bar_ofree + 2;              // [2] query operand of a segment is in shared memory
+  uint64_t* bar_pfull = bar_sfree + 4;              // [4] probabilities of a tile are in shared memory (buffer = tile & 3)
+  uint64_t* bar_ofree = bar_pfull + 4;              // [4] the team has folded the output buffer into its registers
+  uint64_t* bar_qfull = bar_ofree + 4;              // [2] query operand of a segment is in shared memory
+  uint64_t* bar_efull = bar_qfull + 2;              // [2] merged result of a segment is in the exchange area
+  uint64_t* bar_efree = bar_efull + 2;              // [2] the epilogue warp has stored it
   volatile int* abort_flag = plan.misc + 4;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(plan.misc + 5);
 
@@ -221,12 +224,13 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
     reinterpret_cast<uint4*>(smem + C::kQOff)[i] = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) {
     for (int i = 0; i < C::kStages; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 1); }
-    for (int i = 0; i < 4; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 4); }
-    for (int i = 0; i < 2; ++i) {
+    for (int i = 0; i < 4; ++i) {
+      mbar_init(&bar_sfull[i], 1);
+      mbar_init(&bar_sfree[i], 4);
       mbar_init(&bar_pfull[i], kTeamThreads);
       mbar_init(&bar_ofree[i], 4);
-      mbar_init(&bar_qfull[i], kTeamThreads);
     }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bar_qfull[i], kTeamThreads); mbar_init(&bar_efull[i], kTeamThreads); mbar_init(&bar_efree[i], 1); }
     mbar_fence_init();
     *abort_flag = 0;
   }
@@ -245,7 +249,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_o[2] = {tmem + 64, tmem + 64 + NP};      // logits buffer b at column 16 b
+  const uint32_t tmem_o = tmem + 64;                           // logits buffer b at column 16 b, output buffer b at 64 + NP b
   const uint32_t lane_base = static_cast<uint32_t>(warp & 3) * 32u << 16;
 
   PlanSlice sl;
@@ -267,25 +271,29 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
 
     if (warp == kProducerWarp) {
       // ================= copies: per granule the K part, and the V part with the header ================
+      // Lane 2i copies the K part of granule i of the tile, lane 2i + 1 its V part and header.  The
+      // addresses of a tile are worked out before the lane that watches the ring looks at the stage, so
+      // that the copy engine's queue is refilled with as little of a gap as possible.
       bool ok = true;
+      const int gi = lane >> 1;
+      const uint32_t src_off = (lane & 1) ? C::kPart : 0u, bytes = (lane & 1) ? C::kVSlot : C::kPart;
+      const uint32_t dst_off = (lane & 1) ? C::kKArea + gi * C::kVSlot : gi * C::kPart;
       for (int si = 0; si < nseg && ok; ++si) {
-        const Segment sg = plan.segs[si];
-        for (int k0 = 0; k0 < sg.n && ok; k0 += kTileBlocks) {
-          const int nb = min(kTileBlocks, sg.n - k0);
+        const int n = plan.segs[si].n, g = plan.segs[si].g;
+        const int* seg_ids = plan.ids + plan.segs[si].list_off;
+        for (int k0 = 0; k0 < n; k0 += kTileBlocks) {
+          const int nb = min(kTileBlocks, n - k0);
+          const uint8_t* src = nullptr;
+          if (lane < 2 * nb) src = p.cache + (static_cast<size_t>(seg_ids[k0 + gi]) * Hkv + g) * C::kGran + src_off;
           const uint32_t stage = tile_no % C::kStages, use = tile_no / C::kStages;
-          if (use > 0) ok = wait_bar(&bar_empty[stage], (use - 1) & 1u, abort_flag);
-          ok = __all_sync(0xffffffffu, ok);
-          if (!ok) break;
           uint8_t* st = ring + stage * C::kStageBytes;
-          if (lane == 0) mbar_expect_tx(&bar_full[stage], nb * C::kGran);
-          __syncwarp();
-          if (lane < 2 * nb) {
-            const int i = lane >> 1;
-            const int id = plan.ids[sg.list_off + k0 + i];
-            const uint8_t* src = p.cache + (static_cast<size_t>(id) * Hkv + sg.g) * C::kGran;
-            if ((lane & 1) == 0) bulk_copy_g2s(st + i * C::kPart, src, C::kPart, &bar_full[stage]);
-            else bulk_copy_g2s(st + C::kKArea + i * C::kVSlot, src + C::kPart, C::kVSlot, &bar_full[stage]);
+          if (lane == 0) {
+            if (use > 0) ok = wait_bar(&bar_empty[stage], (use - 1) & 1u, abort_flag);
+            if (ok) mbar_expect_tx(&bar_full[stage], nb * C::kGran);
           }
+          ok = __shfl_sync(0xffffffffu, ok, 0);
+          if (!ok) break;
+          if (lane < 2 * nb) bulk_copy_g2s(st + dst_off, src, bytes, &bar_full[stage]);
           ++tile_no;
         }
       }
@@ -306,7 +314,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           bool progress = false;
           // ---- P V of tile `tile_no`
           {
-            const uint32_t buf = tile_no & 1u, use = tile_no >> 1;
+            const uint32_t buf = tile_no & 3u, use = tile_no >> 2;
             if (mbar_test(&bar_pfull[buf], use & 1u) && (use == 0 || mbar_test(&bar_ofree[buf], (use - 1) & 1u))) {
               const int n = plan.segs[v_si].n;
               const int nb = min(kTileBlocks, n - v_k0);
@@ -316,7 +324,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
               const uint32_t pa = smem_u32(pbuf + buf * C::kPBytes);
               const int nks = (nb + 1) >> 1;                  // 32 tokens (two granules) per instruction
               for (int ks = 0; ks < nks; ++ks)
-                umma_f8(tmem_o[buf], umma_desc(va + ks * 2 * C::kVSlot, C::kVSlot, 128), umma_desc(pa + ks * 256, 128, 1024), umma_idesc(NP),
+                umma_f8(tmem_o + NP * buf, umma_desc(va + ks * 2 * C::kVSlot, C::kVSlot, 128), umma_desc(pa + ks * 256, 128, 1024), umma_idesc(NP),
                         ks > 0 ? 1u : 0u);
               umma_commit(&bar_empty[stage]);     // the stage is free again and the tile's product is in its output buffer
               ++tile_no;
@@ -353,6 +361,116 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         }
         if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
       }
+    } else if (warp == kEpilogueWarp) {
+      // ================= stores, piece counting and the split-KV merge: off the teams' critical path ========
+      // Lane l owns dims 4l .. 4l+3 of every head.
+      bool ok = true;
+      const int d0 = lane * 4;
+      for (int si = 0; si < nseg; ++si, ++seg_no) {
+        const Segment sg = plan.segs[si];
+        const uint32_t par = seg_no & 1u;
+        ok = wait_bar(&bar_efull[par], (seg_no >> 1) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        const float* xs = xch + par * C::kXchFloats;
+        const int h0 = sg.g * G;
+        if (!sg.partial) {
+          if (d0 < D) {
+            for (int h = 0; h < G; ++h) {
+              const float4 v = *reinterpret_cast<const float4*>(xs + h * kTeamThreads + d0);
+              *reinterpret_cast<uint2*>(p.out + (static_cast<size_t>(sg.b) * Hq + h0 + h) * D + d0) =
+                  make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+            }
+          }
+        } else {
+          const size_t base = chunk_mode ? (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks + sg.slot
+                                         : static_cast<size_t>(sg.slot) * G;
+          const size_t pstride = chunk_mode ? static_cast<size_t>(p.max_chunks) : 1;
+          for (int h = 0; h < G; ++h) {
+            if (d0 < D) *reinterpret_cast<float4*>(p.part_o + (base + h * pstride) * D + d0) = *reinterpret_cast<const float4*>(xs + h * kTeamThreads + d0);
+            if (lane == 0) {
+              const float M = xs[kGMax * kTeamThreads + h];
+              p.part_m[base + h * pstride] = chunk_mode ? M * kLn2 : M;   // exported partials use natural-log units
+              p.part_l[base + h * pstride] = xs[kGMax * kTeamThreads + 8 + h];
+            }
+          }
+          __syncwarp();                         // every store of the piece has been issued
+          int last = 0;
+          if (lane == 0) {
+            // release (this CTA's piece is visible before the count moves) and acquire (the other pieces
+            // are visible before they are read) in one round trip
+            int* counter = p.counters + sg.b * Hkv + sg.g;
+            int old;
+            asm volatile("atom.add.acq_rel.gpu.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+            last = old == sg.expected - 1;
+            if (last) *counter = 0;             // ready for the next call
+          }
+          last = __shfl_sync(0xffffffffu, last, 0);
+          if (last && d0 < D) {
+            // this CTA delivered the last piece: log-sum-exp merge of all pieces (split-K merge).  Two
+            // pieces at a time: all their (m, l, o) are loaded before any is used, so a batch costs one
+            // trip to L2; the running (M, num, den) carries over from batch to batch.
+            int first_cta = 0;
+            if (!chunk_mode) {
+              const long long fs = static_cast<long long>(Hkv) * plan.pre_blk[sg.b] + static_cast<long long>(sg.g) * sg.seq_blocks;
+              first_cta = plan_cta_of(sl, fs);
+            }
+            const size_t cstride = chunk_mode ? 1 : static_cast<size_t>(2) * G;            // between pieces
+            const size_t base0 = chunk_mode ? (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks
+                                            : static_cast<size_t>(2 * first_cta) * G;
+            // decode mode: the first piece sits in the odd slot of its CTA, the others in the even slot
+            auto piece = [&](int c, int r) -> size_t {
+              return base0 + c * cstride + r * pstride + ((!chunk_mode && c == 0) ? static_cast<size_t>(G) : 0);
+            };
+            const float unit = chunk_mode ? kLog2eU : 1.0f;     // exported maxima of chunk mode are natural logs
+            float M[kGMax], den[kGMax];
+            float4 num[kGMax];
+#pragma unroll
+            for (int r = 0; r < kGMax; ++r) { M[r] = -INFINITY; den[r] = 0.0f; num[r] = make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+            for (int c0 = 0; c0 < sg.expected; c0 += 2) {
+              float mc[2][kGMax], lc[2][kGMax];
+              float4 oc[2][kGMax];
+#pragma unroll
+              for (int k = 0; k < 2; ++k)
+#pragma unroll
+                for (int r = 0; r < kGMax; ++r) {
+                  const bool on = r < G && c0 + k < sg.expected;
+                  const size_t at = on ? piece(c0 + k, r) : 0;
+                  mc[k][r] = on ? __ldcg(p.part_m + at) : 0.0f;
+                  lc[k][r] = on ? __ldcg(p.part_l + at) : 0.0f;
+                  oc[k][r] = on ? __ldcg(reinterpret_cast<const float4*>(p.part_o + at * D + d0)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+                }
+#pragma unroll
+              for (int k = 0; k < 2; ++k)
+#pragma unroll
+                for (int r = 0; r < kGMax; ++r) {
+                  if (lc[k][r] > 0.0f) {
+                    const float mk = mc[k][r] * unit;
+                    const float Mn = fmaxf(M[r], mk);
+                    const float keep = ex2(M[r] - Mn), wgt = lc[k][r] * ex2(mk - Mn);
+                    num[r].x = num[r].x * keep + wgt * oc[k][r].x;
+                    num[r].y = num[r].y * keep + wgt * oc[k][r].y;
+                    num[r].z = num[r].z * keep + wgt * oc[k][r].z;
+                    num[r].w = num[r].w * keep + wgt * oc[k][r].w;
+                    den[r] = den[r] * keep + wgt;
+                    M[r] = Mn;
+                  }
+                }
+            }
+#pragma unroll
+            for (int r = 0; r < kGMax; ++r) {
+              if (r < G) {
+                const float inv = den[r] > 0.0f ? 1.0f / den[r] : 0.0f;
+                *reinterpret_cast<uint2*>(p.out + (static_cast<size_t>(sg.b) * Hq + h0 + r) * D + d0) =
+                    make_uint2(pack_bf16x2(num[r].x * inv, num[r].y * inv), pack_bf16x2(num[r].z * inv, num[r].w * inv));
+              }
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_efree[par]);
+      }
+      if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     } else {
       // ================= softmax teams: thread t owns token t of its tiles and dim t of its output =====
       const int team = warp >> 2, wq = warp & 3;
@@ -425,7 +543,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         float vref = 0.0f;
         bool pending = false;       // a tile of this team whose P V product is not folded in yet
         uint32_t pend_tile = 0;
-        const uint32_t obuf = tmem_o[team] + lane_base;
 
         // O_tile -> registers: o = o * a + (term0 + term1 / 16 + term2 / 256)
         auto fold_issue = [&](uint32_t (&r)[NP]) {
@@ -434,6 +551,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           bad = bad || !ok;
           if (bad) return;
           tc_fence_after();
+          const uint32_t obuf = tmem_o + NP * (pend_tile & 3u) + lane_base;
 #pragma unroll
           for (int half = 0; half < NP / 16; ++half) tmem_ld16_issue(obuf + half * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[half * 16]));
         };
@@ -443,7 +561,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           for (int half = 0; half < NP / 16; ++half) tmem_ld_wait(*reinterpret_cast<uint32_t(*)[16]>(&r[half * 16]));
           tc_fence_before();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&bar_ofree[team]);
+          if (lane == 0) mbar_arrive(&bar_ofree[pend_tile & 3u]);
 #pragma unroll
           for (int h = 0; h < kGMax; ++h)
             o_reg[h] = o_reg[h] * a_prev[h] + (__uint_as_float(r[h]) + __uint_as_float(r[kGMax + h]) * 0.0625f +
@@ -455,7 +573,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           if (k0 == kTileBlocks && team == 0 && more) publish_q(seg_no + 1);   // after the segment's first tile, whoever had it
           if ((tile_no & 1u) != static_cast<uint32_t>(team)) continue;
           const int nb = min(kTileBlocks, sg.n - k0);
-          const uint32_t stage = tile_no % C::kStages, buf = team;
+          const uint32_t stage = tile_no % C::kStages, buf = tile_no & 3u;
           uint8_t* st = ring + stage * C::kStageBytes;
           // scales of the granule that holds token t: the header travels behind the granule's V codes
           const float* hdr = reinterpret_cast<const float*>(st + C::kKArea + (t >> 4) * C::kVSlot + C::kPart);
@@ -494,11 +612,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           }
           bad = barrier_or(team_bar, kTeamThreads, bad);
           if (bad) break;
-          // the product of the team's previous tile is on its way into registers while this tile's
-          // probabilities are computed
-          uint32_t o_raw[NP];
-          const bool folding = pending;
-          if (folding) fold_issue(o_raw);
           const int* rmx = my_red_max;
           // reference V scale: the largest met so far by the team in the segment (uniform over the team)
           const float vmax = __int_as_float(max(max(rmx[8], rmx[20]), max(rmx[32], rmx[44])));
@@ -552,7 +665,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             fence_proxy_async();
             mbar_arrive(&bar_pfull[buf]);
           }
-          if (folding) fold_finish(o_raw);
+          // the product of the team's previous tile (its own buffers, so nothing above had to wait for it)
+          if (pending) {
+            uint32_t o_raw[NP];
+            fold_issue(o_raw);
+            fold_finish(o_raw);
+          }
 #pragma unroll
           for (int h = 0; h < kGMax; ++h) a_prev[h] = a_o[h];
           pending = true;
@@ -573,11 +691,17 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           if (lane == 0) my_red_sum[wq * 8 + h] = ws;
         }
         bad = barrier_or(team_bar, kTeamThreads, bad);
-        float lsum[kGMax];
+        float lsum[kGMax], acc_m[kGMax], acc_l[kGMax];
 #pragma unroll
         for (int h = 0; h < kGMax; ++h) lsum[h] = (my_red_sum[h] + my_red_sum[8 + h]) + (my_red_sum[16 + h] + my_red_sum[24 + h]);
         float* xs = xch + (seg_no & 1u) * C::kXchFloats;
         if (team == 1) {
+          // the area was last used two segments ago; the epilogue warp must be done with it
+          if (seg_no >= 2) {
+            bool ok = !bad && wait_bar(&bar_efree[seg_no & 1u], ((seg_no >> 1) - 1) & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            bad = bad || !ok;
+          }
 #pragma unroll
           for (int h = 0; h < kGMax; ++h) {
             xs[h * kTeamThreads + t] = o_reg[h] * vref;
@@ -587,94 +711,26 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         bad = barrier_or(3, kSmThreads, bad);
         if (bad) break;
         if (team == 0) {
-          const int h0 = sg.g * G;
-          float* po = nullptr; float* pm = nullptr; float* pl = nullptr;
-          size_t pstride = 1;
-          if (sg.partial) {
-            const size_t base = chunk_mode ? (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks + sg.slot
-                                           : static_cast<size_t>(sg.slot) * G;
-            po = p.part_o + base * D; pm = p.part_m + base; pl = p.part_l + base;
-            pstride = chunk_mode ? static_cast<size_t>(p.max_chunks) : 1;
-          }
+          // the other team's running softmax is one more piece of the same segment; the merged, normalised
+          // result goes back into the exchange area, from where the epilogue warp stores it
 #pragma unroll
           for (int h = 0; h < kGMax; ++h) {
-            if (h < G) {
-              // the other team's running softmax is one more piece of the same segment
-              const float m1 = xs[kGMax * kTeamThreads + h], l1 = xs[kGMax * kTeamThreads + 8 + h];
-              const float M = fmaxf(m_run[h], m1);
-              const float mu = M == -INFINITY ? 0.0f : M;
-              const float w0 = ex2(m_run[h] - mu), w1 = ex2(m1 - mu);
-              const float den = lsum[h] * w0 + l1 * w1;
-              const float num = o_reg[h] * vref * w0 + xs[h * kTeamThreads + t] * w1;
-              const float val = den > 0.0f ? num * (1.0f / 256.0f) / den : 0.0f;
-              if (!sg.partial) {
-                if (t < D) p.out[(static_cast<size_t>(sg.b) * Hq + h0 + h) * D + t] = __float2bfloat16(val);
-              } else {
-                if (t < D) po[h * pstride * D + t] = val;
-                if (t == 0) {
-                  pm[h * pstride] = chunk_mode ? M * kLn2 : M;   // exported partials use natural-log units
-                  pl[h * pstride] = den;
-                }
-              }
-            }
+            const float m1 = xs[kGMax * kTeamThreads + h], l1 = xs[kGMax * kTeamThreads + 8 + h];
+            const float M = fmaxf(m_run[h], m1);
+            const float mu = M == -INFINITY ? 0.0f : M;
+            const float w0 = ex2(m_run[h] - mu), w1 = ex2(m1 - mu);
+            const float den = lsum[h] * w0 + l1 * w1;
+            const float num = o_reg[h] * vref * w0 + xs[h * kTeamThreads + t] * w1;
+            xs[h * kTeamThreads + t] = den > 0.0f ? num * (1.0f / 256.0f) / den : 0.0f;
+            acc_m[h] = M;
+            acc_l[h] = den;
           }
-          if (sg.partial) {
-            bad = barrier_or(team_bar, kTeamThreads, bad);      // every store of the piece has been issued
-            int* counter = p.counters + sg.b * Hkv + sg.g;
-            if (t == 0) {
-              // release (this CTA's piece is visible before the count moves) and acquire (the other pieces
-              // are visible before they are read) in one round trip
-              int old;
-              asm volatile("atom.add.acq_rel.gpu.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
-              const int last = old == sg.expected - 1;
-              if (last) *counter = 0;             // ready for the next call
-              plan.misc[3] = last;
-            }
-            bad = barrier_or(team_bar, kTeamThreads, bad);
-            if (plan.misc[3] && t < D) {
-              // this CTA delivered the last piece: log-sum-exp merge of all pieces (split-K merge), dim t.
-              // All heads advance together so that the loads of one pass are in flight at the same time.
-              int first_cta = 0;
-              if (!chunk_mode) {
-                const long long fs = static_cast<long long>(Hkv) * plan.pre_blk[sg.b] + static_cast<long long>(sg.g) * sg.seq_blocks;
-                first_cta = plan_cta_of(sl, fs);
-              }
-              const size_t cstride = chunk_mode ? 1 : static_cast<size_t>(2) * G;            // between pieces
-              const size_t rstride = chunk_mode ? static_cast<size_t>(p.max_chunks) : 1;     // between heads
-              const size_t base0 = chunk_mode ? (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks
-                                              : static_cast<size_t>(2 * first_cta) * G;
-              // decode mode: the first piece sits in the odd slot of its CTA, the others in the even slot
-              auto piece = [&](int c, int r) -> size_t {
-                return base0 + c * cstride + r * rstride + ((!chunk_mode && c == 0) ? static_cast<size_t>(G) : 0);
-              };
-              float M[kGMax], num[kGMax], den[kGMax];
+          bad = barrier_or(team_bar, kTeamThreads, bad);     // every thread has read the other team's maxima and sums
+          if (t == 0) {
 #pragma unroll
-              for (int r = 0; r < kGMax; ++r) { M[r] = -INFINITY; num[r] = 0.0f; den[r] = 0.0f; }
-#pragma unroll 2
-              for (int c = 0; c < sg.expected; ++c) {
-#pragma unroll
-                for (int r = 0; r < kGMax; ++r)
-                  if (r < G) M[r] = fmaxf(M[r], __ldcg(p.part_m + piece(c, r)));
-              }
-#pragma unroll 2
-              for (int c = 0; c < sg.expected; ++c) {
-#pragma unroll
-                for (int r = 0; r < kGMax; ++r) {
-                  if (r < G) {
-                    const size_t at = piece(c, r);
-                    const float mc = __ldcg(p.part_m + at), lc = __ldcg(p.part_l + at), oc = __ldcg(p.part_o + at * D + t);
-                    const float wgt = lc > 0.0f ? lc * (chunk_mode ? ex2((mc - M[r]) * kLog2eU) : ex2(mc - M[r])) : 0.0f;
-                    num[r] += wgt * oc;
-                    den[r] += wgt;
-                  }
-                }
-              }
-#pragma unroll
-              for (int r = 0; r < kGMax; ++r)
-                if (r < G) p.out[(static_cast<size_t>(sg.b) * Hq + h0 + r) * D + t] = __float2bfloat16(den[r] > 0.0f ? num[r] / den[r] : 0.0f);
-            }
-            bad = barrier_or(team_bar, kTeamThreads, bad);     // misc[3] is reused by the next segment
+            for (int h = 0; h < kGMax; ++h) { xs[kGMax * kTeamThreads + h] = acc_m[h]; xs[kGMax * kTeamThreads + 8 + h] = acc_l[h]; }
           }
+          mbar_arrive(&bar_efull[seg_no & 1u]);
         }
         ++seg_no;
       }

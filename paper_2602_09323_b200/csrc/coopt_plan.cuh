@@ -10,7 +10,7 @@
 
 namespace coopt {
 
-constexpr int kCap = 2048;            // block ids staged in shared memory per round
+constexpr int kCap = 1024;            // block ids staged in shared memory per round
 constexpr int kMaxSeg = 32;           // segments planned per round
 constexpr int kMaxBatch = 1024;
 constexpr int kMinBlocksPerCta = 16;
@@ -164,7 +164,7 @@ __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, cons
     Segment sg;
     sg.b = cb; sg.g = cg; sg.j0 = cj; sg.n = static_cast<int>(n); sg.list_off = used;
     sg.seq_blocks = nb;
-    sg.ctx_len = max(0, min(p.context_lens[cb], p.max_blocks_per_seq * kBlockSize));
+    sg.ctx_len = 0;     // filled in by plan_stage_ids, off this thread's serial path
     if (chunk_mode) {
       sg.partial = 1;
       sg.slot = cj / p.chunk_blocks;
@@ -194,8 +194,10 @@ __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, cons
 }
 
 // Physical block ids of every planned segment -> shared memory (range-checked: a bad id is
-// reported in the status word and replaced by block 0, never dereferenced).
+// reported in the status word and replaced by block 0, never dereferenced), and the context length
+// of every segment's sequence.
 __device__ inline void plan_stage_ids(const DecodeParams& p, const PlanSmem& s, int nseg, int tid, int nthreads) {
+  if (tid < nseg) s.segs[tid].ctx_len = max(0, min(p.context_lens[s.segs[tid].b], p.max_blocks_per_seq * kBlockSize));
   for (int i = 0; i < nseg; ++i) {
     const Segment& sg = s.segs[i];
     const int* trow = p.block_table + static_cast<size_t>(sg.b) * p.max_blocks_per_seq + sg.j0;
