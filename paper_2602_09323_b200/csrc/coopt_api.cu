@@ -76,6 +76,8 @@ int check_attention_args(const coopt_cache* c, const void* q, void* out, const i
   if (group < 1 || group > 8) return COOPT_ERR_UNSUPPORTED;
   if (batch > decode_max_batch() || static_cast<long long>(batch) * c->num_kv_heads > decode_counter_slots())
     return COOPT_ERR_UNSUPPORTED;
+  // the planner indexes (sequence, kv head, block) triples with 31 bits
+  if (static_cast<long long>(batch) * c->num_kv_heads * max_blocks_per_seq >= (1ll << 31)) return COOPT_ERR_UNSUPPORTED;
   return COOPT_OK;
 }
 

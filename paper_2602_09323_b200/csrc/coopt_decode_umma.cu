@@ -542,6 +542,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         for (int h = 0; h < kGMax; ++h) { m_run[h] = -INFINITY; l_run[h] = 0.0f; o_reg[h] = 0.0f; a_prev[h] = 0.0f; }
         float vref = 0.0f;
         bool pending = false;       // a tile of this team whose P V product is not folded in yet
+        bool q_due = team == 0 && more;   // the next segment's query is published behind this team's first tile
         uint32_t pend_tile = 0;
 
         // O_tile -> registers: o = o * a + (term0 + term1 / 16 + term2 / 256)
@@ -570,7 +571,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         };
 
         for (int k0 = 0; k0 < sg.n; k0 += kTileBlocks, ++tile_no) {
-          if (k0 == kTileBlocks && team == 0 && more) publish_q(seg_no + 1);   // after the segment's first tile, whoever had it
           if ((tile_no & 1u) != static_cast<uint32_t>(team)) continue;
           const int nb = min(kTileBlocks, sg.n - k0);
           const uint32_t stage = tile_no % C::kStages, buf = tile_no & 3u;
@@ -675,9 +675,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           for (int h = 0; h < kGMax; ++h) a_prev[h] = a_o[h];
           pending = true;
           pend_tile = tile_no;
+          if (q_due) { publish_q(seg_no + 1); q_due = false; }
         }
         // (a team whose wait ran out keeps company until the next barrier makes it known to everybody)
-        if (team == 0 && more && sg.n <= kTileBlocks) publish_q(seg_no + 1);   // a one-tile segment
+        if (q_due) publish_q(seg_no + 1);   // the segment had no tile for this team
 
         // ---- end of segment: fold the last product, reduce the sums, merge the two teams ---------------
         if (pending) {

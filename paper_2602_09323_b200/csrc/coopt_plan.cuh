@@ -60,6 +60,15 @@ struct PlanSmem {
   int* misc;         // [4]: nseg, next x (lo, hi), scratch flag
 };
 
+// floor(a / b) for 0 <= a < 2^52, 0 < b < 2^31: one double division and a fix-up instead of the
+// generic 64-bit routine (the planner is one thread's serial work at the head of every CTA).
+__device__ __forceinline__ long long plan_div(long long a, int b) {
+  long long q = static_cast<long long>(static_cast<double>(a) / static_cast<double>(b));
+  const long long r = a - q * b;
+  if (r < 0) --q; else if (r >= b) ++q;
+  return q;
+}
+
 __device__ __forceinline__ int plan_find_seq(const int* pre, int batch, long long x, int heads) {
   // largest b in [0, batch) with heads * pre[b] <= x
   int lo = 0, hi = batch - 1;
@@ -114,20 +123,20 @@ __device__ inline bool plan_slice(const DecodeParams& p, const PlanSmem& s, Plan
   if (p.chunk_blocks == 0) {
     sl.P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), max(1ll, sl.N / kMinBlocksPerCta)));
     if (static_cast<int>(blockIdx.x) >= sl.P) return false;
-    sl.lo = blockIdx.x * sl.N / sl.P;
-    sl.hi = (blockIdx.x + 1ll) * sl.N / sl.P;
+    sl.lo = plan_div(blockIdx.x * sl.N, sl.P);
+    sl.hi = plan_div((blockIdx.x + 1ll) * sl.N, sl.P);
     return true;
   }
   const long long U = static_cast<long long>(Hkv) * s.pre_unit[B];
   sl.P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), U));
   if (static_cast<int>(blockIdx.x) >= sl.P) return false;
-  const long long ulo = blockIdx.x * U / sl.P, uhi = (blockIdx.x + 1ll) * U / sl.P;
+  const long long ulo = plan_div(blockIdx.x * U, sl.P), uhi = plan_div((blockIdx.x + 1ll) * U, sl.P);
   auto unit_to_block = [&](long long u) -> long long {
     if (u >= U) return sl.N;
     const int b = plan_find_seq(s.pre_unit, B, u, Hkv);
     const int nch = s.pre_unit[b + 1] - s.pre_unit[b], nb = s.pre_blk[b + 1] - s.pre_blk[b];
     const long long rem = u - static_cast<long long>(Hkv) * s.pre_unit[b];
-    const int g = static_cast<int>(rem / nch), c = static_cast<int>(rem % nch);
+    const int g = static_cast<int>(plan_div(rem, nch)), c = static_cast<int>(rem - static_cast<long long>(g) * nch);
     return static_cast<long long>(Hkv) * s.pre_blk[b] + static_cast<long long>(g) * nb + static_cast<long long>(c) * p.chunk_blocks;
   };
   sl.lo = unit_to_block(ulo);
@@ -136,7 +145,7 @@ __device__ inline bool plan_slice(const DecodeParams& p, const PlanSmem& s, Plan
 }
 // CTA that owns flat block index x (decode mode).
 __device__ __forceinline__ int plan_cta_of(const PlanSlice& sl, long long x) {
-  return static_cast<int>(((x + 1) * sl.P - 1) / sl.N);
+  return static_cast<int>(plan_div((x + 1) * sl.P - 1, static_cast<int>(sl.N)));
 }
 
 // One thread plans the next round starting at flat index x: fills segs, misc[0] = number of
@@ -150,8 +159,8 @@ __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, cons
   {
     const int nb = s.pre_blk[cb + 1] - s.pre_blk[cb];
     const long long rem = xx - static_cast<long long>(Hkv) * s.pre_blk[cb];
-    cg = static_cast<int>(rem / nb);
-    cj = static_cast<int>(rem % nb);
+    cg = static_cast<int>(plan_div(rem, nb));
+    cj = static_cast<int>(rem - static_cast<long long>(cg) * nb);
   }
   while (xx < sl.hi && nseg < kMaxSeg) {
     const int nb = s.pre_blk[cb + 1] - s.pre_blk[cb];
