@@ -42,6 +42,23 @@ def algorithmic_bytes(batch=BATCH, context=CONTEXT):
     return kv + scales + q_out + table
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks of the default process group (the
+    identity without one).  Every rank's timing enters the job's number: the slowest rank decides."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def job_tokens_per_second(world: int, batch_per_rank: int, steps: int, ms: float) -> float:
+    """Whole-job throughput: the path shards by sequence with no exchange, so every rank runs its own
+    batch (weak scaling) and the job's tokens are the sum over ranks, timed by the slowest rank."""
+    return world * batch_per_rank * steps / (ms * 1e-3)
+
+
 class ClockSampler(threading.Thread):
     """SM clock and throttle reasons of one GPU, sampled through NVML while the timed region runs."""
 
@@ -250,11 +267,8 @@ def main():
     ms = start.elapsed_time(stop)
     kernel_ms = sum(a.elapsed_time(b) for a, b in kernel_events) / len(kernel_events)
     assert binding.workspace_status(ws) == 0
-    t = torch.tensor([ms, kernel_ms], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms, kernel_ms = float(t[0]), float(t[1])
-    value = world * BATCH * args.steps / (ms * 1e-3)
+    ms, kernel_ms = max_over_ranks([ms, kernel_ms], device="cuda")
+    value = job_tokens_per_second(world, BATCH, args.steps, ms)
 
     # ---- end to end: host buffers in, host result out, through coopt_decode_step_host ----------
     e2e = None
@@ -278,11 +292,9 @@ def main():
         for i in range(n_e2e):
             host_step(i)
         el = time.perf_counter() - t0
-        te = torch.tensor([el], device="cuda", dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
+        el = max_over_ranks([el], device="cuda")[0]
         h2d = hq_.numel() * 2 + hk_.numel() * 2 + hv_.numel() * 2 + BATCH * 8 + BATCH * max_blocks * 4 + BATCH * 4
-        e2e = {"value": world * BATCH * n_e2e / float(te[0]), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        e2e = {"value": job_tokens_per_second(world, BATCH, n_e2e, el * 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                "d2h_bytes_per_step": ho_.numel() * 2, "steps": n_e2e}
         assert torch.equal(ho_.cuda(), out)
 

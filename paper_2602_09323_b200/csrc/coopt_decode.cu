@@ -1,21 +1,18 @@
-// Paged GQA decode over the FP8 (or bf16) cache: Algorithm 1 phase 2 (Eq. 6 dequantisation on
-// load), Algorithm 2 (Eq. 7-8: the G query heads of a group consume one K/V stream),
-// Algorithm 3 (Eq. 9 valid blocks only, Eq. 10 max-subtracted softmax) and the Opt-Pa
-// chunk-and-merge reduction.
+// Paged decode over the bf16 ablation cache (the un-quantised layout the method is compared with):
+// Eq. 1, Eq. 7-8 (the G query heads of a group consume one K/V stream), Eq. 9 (valid blocks only),
+// Eq. 10 (max-subtracted softmax) and the Opt-Pa chunk-and-merge reduction, on mma.sync.  The FP8
+// cache has its own kernel on the 5th-generation tensor cores; this file also holds the host launcher
+// and the workspace arithmetic that both share.
 //
-// Work decomposition.  All (sequence, kv head, block) triples form one flat list.  In decode
-// mode CTA i takes the i-th of P equal slices of that list (split-KV balanced by bytes); in
-// chunk mode it takes a contiguous run of fixed-size chunks.  A slice is cut into segments at
-// (sequence, kv head) boundaries (and chunk boundaries).  Inside a segment the CTA's warps take
-// blocks round-robin; each warp streams its granules through a private ring of shared-memory
-// stages filled by bulk async copies (one elected lane issues, an mbarrier per stage counts the
-// bytes), runs both contractions on mma.sync with the G query heads padded to the 16 rows of
-// the instruction, and keeps an online softmax per query head (warp shuffles inside the quad
-// that owns a head, one shared-memory step across warps at the end of the segment).  A segment
-// that does not cover its whole sequence leaves (m, l, o) in the workspace; the CTA that
-// delivers the last piece of a (sequence, kv head) merges them by log-sum-exp and writes the
-// bf16 output.  The K scale of a granule factors out of the dot product and is applied to the
-// logits; the V scale is folded into the probabilities.
+// The work decomposition is the shared planner's.  Inside a segment the CTA's warps take blocks
+// round-robin; each warp streams its granules through a private ring of shared-memory stages filled
+// by bulk async copies (one elected lane issues, an mbarrier per stage counts the bytes), runs both
+// contractions with the G query heads in the top rows of the 16-row instruction tile (the
+// probabilities split into a bf16 high and low half, the low halves in rows 8..15), and keeps an
+// online softmax per query head (warp shuffles inside the quad that owns a head, one shared-memory
+// step across warps at the end of the segment).  A segment that does not cover its whole sequence
+// leaves (m, l, o) in the workspace; the CTA that delivers the last piece of a (sequence, kv head)
+// merges them by log-sum-exp and writes the bf16 output.
 #include "coopt_plan.cuh"
 
 namespace coopt {
@@ -27,13 +24,13 @@ constexpr int kThreads = kWarps * 32;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-template <int D, bool FP8>
+template <int D>
 struct Cfg {
-  static constexpr int kGran = granule_bytes(D, FP8);
-  static constexpr int kStages = FP8 ? 4 : 2;
+  static constexpr int kGran = granule_bytes(D, false);
+  static constexpr int kStages = 2;
   static constexpr int kKSteps = D / 16;
   static constexpr int kNTiles = D / 8;
-  static constexpr int kOAcc = FP8 ? 2 : 4;     // accumulator registers kept per n-tile
+  static constexpr int kOAcc = 4;               // accumulator registers kept per n-tile
   // shared memory carve-up (bytes)
   static constexpr int kRingOff = 0;
   static constexpr int kRingBytes = kWarps * kStages * kGran;
@@ -57,24 +54,19 @@ __device__ __forceinline__ float quad_sum(float x) {
   return x + __shfl_xor_sync(0xffffffffu, x, 2);
 }
 
-// mma with only the top 8 rows of A in use (rows 8..15 are zero): two live accumulators.
-template <bool F16>
+// bf16 mma with only the top 8 rows of A in use (rows 8..15 are zero): two live accumulators.
 __device__ __forceinline__ void mma_top(float& d0, float& d1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
   float t2, t3;
-  if constexpr (F16) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
-                 : "+f"(d0), "+f"(d1), "=f"(t2), "=f"(t3)
-                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.0f));
-  } else {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
-                 : "+f"(d0), "+f"(d1), "=f"(t2), "=f"(t3)
-                 : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.0f));
-  }
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
+               : "+f"(d0), "+f"(d1), "=f"(t2), "=f"(t3)
+               : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.0f));
+  (void)t2;
+  (void)t3;
 }
 
-template <int D, bool FP8>
+template <int D>
 __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeParams p) {
-  using C = Cfg<D, FP8>;
+  using C = Cfg<D>;
   extern __shared__ __align__(128) uint8_t smem[];
   uint8_t* ring = smem + C::kRingOff;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
@@ -165,36 +157,14 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
     for (int si = 0; si < nseg; ++si) {
       const Segment sg = segs[si];
 
-      // ---- query fragments (A operand), converted for the tensor-core input type ------------
+      // ---- query fragments (A operand): bf16 as loaded ---------------------------------------
       uint32_t qa[C::kKSteps][2];
-      float qscale = p.sm_scale_log2;
-      if constexpr (FP8) {
-        float amax = 0.0f;
 #pragma unroll
-        for (int s = 0; s < C::kKSteps; ++s)
-#pragma unroll
-          for (int e = 0; e < 2; ++e)
-            amax = fmaxf(amax, fmaxf(fabsf(bf16_lo(qraw[s][e])), fabsf(bf16_hi(qraw[s][e]))));
-        amax = quad_max(amax);
-        // power-of-two scaling into f16's comfortable range: exact, undone on the logits
-        int k2 = 0;
-        if (amax > 0.0f) k2 = max(-64, min(64, 134 - static_cast<int>((__float_as_uint(amax) >> 23) & 0xFF)));
-        const float up = __uint_as_float(static_cast<uint32_t>(k2 + 127) << 23);
-        const float down = __uint_as_float(static_cast<uint32_t>(127 - k2) << 23);
-        qscale *= down;
-#pragma unroll
-        for (int s = 0; s < C::kKSteps; ++s)
-#pragma unroll
-          for (int e = 0; e < 2; ++e)
-            qa[s][e] = pack_f16x2(bf16_lo(qraw[s][e]) * up, bf16_hi(qraw[s][e]) * up);
-      } else {
-#pragma unroll
-        for (int s = 0; s < C::kKSteps; ++s) { qa[s][0] = qraw[s][0]; qa[s][1] = qraw[s][1]; }
-      }
+      for (int s = 0; s < C::kKSteps; ++s) { qa[s][0] = qraw[s][0]; qa[s][1] = qraw[s][1]; }
       if (si + 1 < nseg) load_q_raw(segs[si + 1]);
 
       // ---- online softmax state of this warp for the segment ---------------------------------
-      float m_run = -INFINITY, l_run = 0.0f, vref = 0.0f;
+      float m_run = -INFINITY, l_run = 0.0f;
       float o[C::kNTiles][C::kOAcc];
 #pragma unroll
       for (int t = 0; t < C::kNTiles; ++t)
@@ -214,42 +184,21 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
         const uint8_t* st = my_ring + stage * C::kGran;
         const int nvalid = min(kBlockSize, sg.ctx_len - (sg.j0 + k) * kBlockSize);   // Eq. 9 tail
 
-        float sK = 1.0f, sV = 1.0f;
-        if constexpr (FP8) {
-          sK = reinterpret_cast<const float*>(st)[0];
-          sV = reinterpret_cast<const float*>(st)[1];
-        }
-
         // ---- S = Q K^T for 16 tokens (two n-tiles of 8) ---------------------------------------
         float s0[2] = {0.0f, 0.0f}, s1[2] = {0.0f, 0.0f};
-        const uint8_t* kp = st + part_offset(D, FP8, 0) + lane * 16;
-        if constexpr (FP8) {
+        const uint8_t* kp = st + part_offset(D, false, 0) + lane * 16;
 #pragma unroll
-          for (int i = 0; i < D / 64; ++i) {
-            const uint4 w0 = lds128(kp + (0 * (D / 64) + i) * 512);
-            const uint4 w1 = lds128(kp + (1 * (D / 64) + i) * 512);
-            const uint32_t a[4] = {w0.x, w0.y, w0.z, w0.w}, c[4] = {w1.x, w1.y, w1.z, w1.w};
-#pragma unroll
-            for (int ss = 0; ss < 4; ++ss) {
-              const int s = 4 * i + ss;
-              mma_top<true>(s0[0], s0[1], qa[s][0], qa[s][1], e4m3x2_to_f16x2_lo(a[ss]), e4m3x2_to_f16x2_hi(a[ss]));
-              mma_top<true>(s1[0], s1[1], qa[s][0], qa[s][1], e4m3x2_to_f16x2_lo(c[ss]), e4m3x2_to_f16x2_hi(c[ss]));
-            }
-          }
-        } else {
-#pragma unroll
-          for (int i = 0; i < D / 32; ++i) {
-            const uint4 w0 = lds128(kp + (0 * (D / 32) + i) * 512);
-            const uint4 w1 = lds128(kp + (1 * (D / 32) + i) * 512);
-            mma_top<false>(s0[0], s0[1], qa[2 * i][0], qa[2 * i][1], w0.x, w0.y);
-            mma_top<false>(s0[0], s0[1], qa[2 * i + 1][0], qa[2 * i + 1][1], w0.z, w0.w);
-            mma_top<false>(s1[0], s1[1], qa[2 * i][0], qa[2 * i][1], w1.x, w1.y);
-            mma_top<false>(s1[0], s1[1], qa[2 * i + 1][0], qa[2 * i + 1][1], w1.z, w1.w);
-          }
+        for (int i = 0; i < D / 32; ++i) {
+          const uint4 w0 = lds128(kp + (0 * (D / 32) + i) * 512);
+          const uint4 w1 = lds128(kp + (1 * (D / 32) + i) * 512);
+          mma_top(s0[0], s0[1], qa[2 * i][0], qa[2 * i][1], w0.x, w0.y);
+          mma_top(s0[0], s0[1], qa[2 * i + 1][0], qa[2 * i + 1][1], w0.z, w0.w);
+          mma_top(s1[0], s1[1], qa[2 * i][0], qa[2 * i][1], w1.x, w1.y);
+          mma_top(s1[0], s1[1], qa[2 * i + 1][0], qa[2 * i + 1][1], w1.z, w1.w);
         }
 
         // ---- online softmax (Eq. 10), log2 units ---------------------------------------------------
-        const float ks = qscale * sK;
+        const float ks = p.sm_scale_log2;
         float sc[4] = {s0[0] * ks, s0[1] * ks, s1[0] * ks, s1[1] * ks};
         const int tok[4] = {2 * quad, 2 * quad + 1, 2 * quad + 8, 2 * quad + 9};
         if (nvalid < kBlockSize) {
@@ -259,47 +208,21 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
         const float m_blk = quad_max(fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3])));
         const float m_new = fmaxf(m_run, m_blk);
         const float a_m = ex2(m_run - m_new);
-        float a_o = a_m, pv = 1.0f;
-        if constexpr (FP8) {
-          // o accumulates sum p * (sV / vref) * codes with vref the largest V scale seen so far
-          const float vnew = fmaxf(vref, sV);
-          if (vnew > 0.0f) {
-            a_o = a_m * __fdividef(vref, vnew);
-            pv = __fdividef(sV, vnew);
-          }
-          vref = vnew;
-        }
         float pr[4];
 #pragma unroll
         for (int e = 0; e < 4; ++e) pr[e] = ex2(sc[e] - m_new);
         l_run = l_run * a_m + (pr[0] + pr[1]) + (pr[2] + pr[3]);
         m_run = m_new;
-        if (__any_sync(0xffffffffu, a_o != 1.0f)) {
+        if (__any_sync(0xffffffffu, a_m != 1.0f)) {
 #pragma unroll
           for (int t = 0; t < C::kNTiles; ++t)
 #pragma unroll
-            for (int e = 0; e < C::kOAcc; ++e) o[t][e] *= a_o;
+            for (int e = 0; e < C::kOAcc; ++e) o[t][e] *= a_m;
         }
 
         // ---- O += P V -----------------------------------------------------------------------------
-        const uint8_t* vp = st + part_offset(D, FP8, 1) + lane * 16;
-        if constexpr (FP8) {
-          const uint32_t pa0 = pack_f16x2(pr[0] * pv, pr[1] * pv), pa2 = pack_f16x2(pr[2] * pv, pr[3] * pv);
-          uint32_t vmask = 0xffffffffu;
-          if (nvalid < kBlockSize) {
-            vmask = 0u;
-#pragma unroll
-            for (int e = 0; e < 4; ++e) vmask |= tok[e] < nvalid ? (0xFFu << (8 * e)) : 0u;
-          }
-#pragma unroll
-          for (int qd = 0; qd < D / 32; ++qd) {
-            const uint4 w = lds128(vp + qd * 512);
-            const uint32_t a[4] = {w.x & vmask, w.y & vmask, w.z & vmask, w.w & vmask};
-#pragma unroll
-            for (int u = 0; u < 4; ++u)
-              mma_top<true>(o[4 * qd + u][0], o[4 * qd + u][1], pa0, pa2, e4m3x2_to_f16x2_lo(a[u]), e4m3x2_to_f16x2_hi(a[u]));
-          }
-        } else {
+        const uint8_t* vp = st + part_offset(D, false, 1) + lane * 16;
+        {
           // bf16 probabilities split into high and low halves; the low halves ride in rows 8..15
           uint32_t hi0 = pack_bf16x2(pr[0], pr[1]), hi2 = pack_bf16x2(pr[2], pr[3]);
           const uint32_t lo0 = pack_bf16x2(pr[0] - bf16_lo(hi0), pr[1] - bf16_hi(hi0));
@@ -330,13 +253,9 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
       l_run = quad_sum(l_run);
       if (row < G) {
         float* mr = merge + (warp * kMaxGroup + row) * C::kMergeStride;
-        const float os = FP8 ? vref : 1.0f;
 #pragma unroll
-        for (int t = 0; t < C::kNTiles; ++t) {
-          float v0 = o[t][0], v1 = o[t][1];
-          if constexpr (!FP8) { v0 += o[t][2]; v1 += o[t][3]; }
-          *reinterpret_cast<float2*>(mr + 8 * t + 2 * quad) = make_float2(v0 * os, v1 * os);
-        }
+        for (int t = 0; t < C::kNTiles; ++t)   // high and low halves of the probabilities were accumulated apart
+          *reinterpret_cast<float2*>(mr + 8 * t + 2 * quad) = make_float2(o[t][0] + o[t][2], o[t][1] + o[t][3]);
         if (quad == 0) { mr[D] = m_run; mr[D + 1] = l_run; }
       }
       __syncthreads();
@@ -464,18 +383,18 @@ void chunk_partial_offsets(int batch, int num_q_heads, int head_dim, int max_chu
   *l = *m + rows * 4;
 }
 
-template <int D, bool FP8>
+template <int D>
 static int launch_one(const DecodeParams& p, int grid, cudaStream_t stream) {
-  using C = Cfg<D, FP8>;
+  using C = Cfg<D>;
   static bool configured[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
   if (dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(paged_decode_kernel<D, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(paged_decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
       return COOPT_ERR_CUDA;
     configured[dev] = true;
   }
-  paged_decode_kernel<D, FP8><<<grid, kThreads, C::kSmemBytes, stream>>>(p);
+  paged_decode_kernel<D><<<grid, kThreads, C::kSmemBytes, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
 
@@ -518,7 +437,7 @@ int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const in
   }
   // FP8 cache: the tcgen05 kernel; bf16 ablation cache: the mma.sync kernel of this file
   if (c->dtype == COOPT_KV_FP8_E4M3) return launch_paged_decode_umma(p, c->head_dim, planned_ctas, stream);
-  return c->head_dim == 128 ? launch_one<128, false>(p, planned_ctas, stream) : launch_one<64, false>(p, planned_ctas, stream);
+  return c->head_dim == 128 ? launch_one<128>(p, planned_ctas, stream) : launch_one<64>(p, planned_ctas, stream);
 }
 
 }  // namespace coopt

@@ -150,3 +150,71 @@ def test_chunked_decode_partials_and_merge(chunk):
         assert np.allclose(m_c[b, h, :n].cpu().numpy(), m, rtol=1e-4, atol=1e-3)
         assert np.allclose(l_c[b, h, :n].cpu().numpy(), l, rtol=5e-3, atol=1e-4)
         assert np.allclose(o_c[b, h, :n].cpu().numpy(), o, rtol=5e-3, atol=2e-2)
+
+
+def _oracle_sequence_cache(w, b, g, calls):
+    """Oracle cache of one sequence and kv head, written by the given (start, stop) row ranges."""
+    k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
+    codes, scales = kv_cache.new_cache(w.num_blocks, w.num_kv_heads, w.head_dim)
+    off = w.kv_offsets[b]
+    for a, z in calls:
+        kv_cache.kv_write(codes, scales, k[off + a:off + z], v[off + a:off + z], slots[off + a:off + z], heads=[g])
+    return codes, scales
+
+
+def test_mixed_length_serving_step_full_size_sampled():
+    """BASELINE configuration 3 at full size: 64 sequences with contexts uniform in [128, 8192]; the
+    history is filled in bulk, then one token per sequence is appended with coopt_kv_write (which may
+    grow a block's scale and re-express its resident codes) and the decode runs over the updated cache.
+    The oracle replays the same two writes for a sample of (sequence, query head) pairs."""
+    w = workloads.config_mixed_serving()
+    B, L = w.batch, w.context_lens
+    k, v, slots = w.k.cuda(), w.v.cuda(), w.slot_mapping.cuda()
+    last = torch.tensor([w.kv_offsets[b] + L[b] - 1 for b in range(B)])
+    hist = torch.ones(k.shape[0], dtype=torch.bool)
+    hist[last] = False
+    hist_idx, new_idx = hist.nonzero().squeeze(1).cuda(), last.cuda()
+    cache = binding.Cache(w.num_blocks, 8, 128)
+    binding.kv_write(cache, k[hist_idx], v[hist_idx], slots[hist_idx])
+    binding.kv_write(cache, k[new_idx].contiguous(), v[new_idx].contiguous(), slots[new_idx].contiguous())
+    out, _ = helpers.gpu_decode(w, cache)
+    assert torch.isfinite(out.float()).all()
+    rng = np.random.default_rng(3)
+    order = np.argsort(L)
+    picks = [(int(order[0]), 3), (int(order[-1]), 38), (int(rng.integers(0, B)), int(rng.integers(0, 40))),
+             (int(rng.integers(0, B)), int(rng.integers(0, 40)))]
+    ref = np.full((B, 40, 128), np.nan)
+    g_codes, g_scales, _ = helpers.cache_to_logical(cache)
+    for b, h in picks:
+        g = h // 5
+        codes, scales = _oracle_sequence_cache(w, b, g, [(0, L[b] - 1), (L[b] - 1, L[b])])
+        blks = w.block_table[b, :(L[b] + 15) // 16].numpy()
+        assert np.array_equal(g_codes[blks, g], codes[blks, g]) and np.array_equal(g_scales[blks, g], scales[blks, g])
+        ref[b, h] = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), L,
+                                              pairs=[(b, h)])[b, h]
+    helpers.check_attention(out, ref, what="mixed serving step")
+
+
+def test_long_context_chunked_full_size_sampled():
+    """BASELINE configuration 4 at full size: contexts of 32768 .. 131072 tokens, chunk size 2048, per-chunk
+    (m, l, o) exported and merged by log-sum-exp; the oracle recomputes two (sequence, query head) pairs."""
+    w = workloads.config_long_context()
+    cache = helpers.gpu_fill(w)
+    out, ws = helpers.gpu_decode(w, cache, chunk_size=2048)
+    assert torch.isfinite(out.float()).all()
+    o_c, m_c, l_c = binding.chunk_partials(ws, w.batch, 40, 128, w.block_table.shape[1], 2048)
+    q = w.q.float().numpy()
+    ref = np.full((4, 40, 128), np.nan)
+    for b, h in [(0, 7), (3, 21)]:
+        L = w.context_lens[b]
+        codes, scales = _oracle_sequence_cache(w, b, h // 5, [(0, L)])
+        res, partials = attention.paged_attention_chunked(q, (codes, scales), w.block_table.numpy(), w.context_lens, 2048,
+                                                          pairs=[(b, h)])
+        ref[b, h] = res[b, h]
+        m, l, o = partials[(b, h)]
+        n = len(m)
+        assert n == L // 2048
+        assert np.allclose(m_c[b, h, :n].cpu().numpy(), m, rtol=1e-4, atol=1e-3)
+        assert np.allclose(l_c[b, h, :n].cpu().numpy(), l, rtol=5e-3, atol=1e-4)
+        assert np.allclose(o_c[b, h, :n].cpu().numpy(), o, rtol=5e-3, atol=2e-2)
+    helpers.check_attention(out, ref, what="long context chunked")
