@@ -8,7 +8,8 @@ namespace coopt {
 
 namespace {
 
-constexpr int kWriteWarps = 4;
+constexpr int kWriteHeads = 4;                 // kv heads per CTA
+constexpr int kWriteWarps = 2 * kWriteHeads;   // FP8: one warp per (kv head, K | V)
 
 struct WriteParams {
   uint8_t* cache;
@@ -57,8 +58,45 @@ __device__ __forceinline__ void find_group(const WriteParams& p, int i, Group& g
   }
 }
 
-// FP8 path.  Each warp stages the K (then V) part of its granule in shared memory, applies the
-// scale rule, and writes the part back with 16-byte stores.
+// The same discovery by one warp in a single trip to memory: 32 slots before token i and 32 from it
+// on are looked at together.  Neighbourhoods that the two windows do not settle (long runs of skipped
+// tokens) fall back to the serial walk.
+__device__ __forceinline__ void find_group_warp(const WriteParams& p, int i, Group& g, int lane) {
+  const int jb = i - 32 + lane, jf = i + lane;
+  const int64_t sb = jb >= 0 ? p.slot_mapping[jb] : -1;
+  const int64_t sf = jf < p.num_tokens ? p.slot_mapping[jf] : -1;
+  const int64_t slot = __shfl_sync(0xffffffffu, sf, 0);
+  if (lane == 0) g.n = 0;
+  if (slot < 0) return;                                   // Eq. 5: skipped token
+  const int64_t blk = slot / kBlockSize;
+  if (blk >= p.num_blocks) return;
+  const unsigned before = __ballot_sync(0xffffffffu, sb >= 0);
+  const unsigned same = __ballot_sync(0xffffffffu, sf >= 0 && sf / kBlockSize == blk);
+  const unsigned other = __ballot_sync(0xffffffffu, sf >= 0 && sf / kBlockSize != blk);
+  const unsigned mem = same & (other ? (1u << (__ffs(other) - 1)) - 1u : 0xffffffffu);
+  const bool back_known = before != 0 || i <= 32;
+  const bool fwd_known = other != 0 || i + 32 >= p.num_tokens || __popc(mem) >= kBlockSize;
+  if (!back_known || !fwd_known) {
+    if (lane == 0) find_group(p, i, g);
+    return;
+  }
+  if (before != 0) {
+    const int64_t sp = __shfl_sync(0xffffffffu, sb, 31 - __clz(before));
+    if (sp / kBlockSize == blk) return;                   // not the leader of its group
+  }
+  const int rank = __popc(mem & ((1u << lane) - 1u));
+  if (((mem >> lane) & 1u) && rank < kBlockSize) {
+    g.tok[rank] = jf;
+    g.off[rank] = static_cast<int>(sf % kBlockSize);
+  }
+  if (lane == 0) {
+    g.blk = static_cast<int>(blk);
+    g.n = min(__popc(mem), kBlockSize);
+  }
+}
+
+// FP8 path.  One warp per (kv head, K | V): it stages that part of its granule in shared memory,
+// applies the scale rule, and writes the part back with 16-byte stores.
 template <int D>
 __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WriteParams p) {
   constexpr int kPart = part_bytes(D, true);          // 16 * D bytes
@@ -66,12 +104,13 @@ __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WritePar
   __shared__ __align__(16) uint8_t stage[kWriteWarps][kPart];
   __shared__ Group group;
 
-  if (threadIdx.x == 0) find_group(p, blockIdx.x, group);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp == 0) find_group_warp(p, blockIdx.x, group, lane);
   __syncthreads();
   const int n = group.n;
   if (n == 0) return;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int h = blockIdx.y * kWriteWarps + warp;
+  const int h = blockIdx.y * kWriteHeads + (warp >> 1);
+  const int which = warp & 1;
   if (h >= p.num_kv_heads) return;
 
   bool fresh = false;
@@ -81,8 +120,7 @@ __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WritePar
   float* scales = reinterpret_cast<float*>(gran + header_offset(D));
   uint8_t* st = stage[warp];
 
-#pragma unroll 1
-  for (int which = 0; which < 2; ++which) {
+  {
     const __nv_bfloat16* src = which == 0 ? p.k : p.v;
     uint8_t* part = gran + part_offset(D, true, which);
 
@@ -143,7 +181,7 @@ __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WritePar
     if (lane == 0) scales[which] = s_new;
     __syncwarp();
   }
-  if (fresh && lane < 6) scales[2 + lane] = 0.0f;       // rest of the header
+  if (which == 0 && fresh && lane < 6) scales[2 + lane] = 0.0f;       // rest of the header
 }
 
 // bf16 ablation cache: store the values unchanged at their permuted places.
@@ -186,9 +224,11 @@ int launch_kv_write(const coopt_cache* c, const void* k, const void* v, int64_t 
   p.num_tokens = num_tokens;
   p.num_kv_heads = c->num_kv_heads;
   p.num_blocks = c->num_blocks;
-  const dim3 grid(num_tokens, (c->num_kv_heads + kWriteWarps - 1) / kWriteWarps);
   const dim3 block(kWriteWarps * 32);
   const bool fp8 = c->dtype == COOPT_KV_FP8_E4M3;
+  // FP8: a CTA serves kWriteHeads kv heads (two warps each); bf16: kWriteWarps heads (one warp each)
+  const int heads_per_cta = fp8 ? kWriteHeads : kWriteWarps;
+  const dim3 grid(num_tokens, (c->num_kv_heads + heads_per_cta - 1) / heads_per_cta);
   if (c->head_dim == 128) {
     if (fp8) kv_write_fp8_kernel<128><<<grid, block, 0, stream>>>(p);
     else kv_write_bf16_kernel<128><<<grid, block, 0, stream>>>(p);
