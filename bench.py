@@ -170,6 +170,110 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_other_workload(args):
+    """The other configurations, one GPU: a step is the configuration's whole pass (cache write of the
+    step's new tokens where it has any, then the attention call); the attention kernel is timed with
+    an event pair on a sample of steps.  Steps rotate over layer caches so that loads come from HBM."""
+    import torch
+    from paper_2602_09323_b200 import binding, build, workloads
+    torch.cuda.set_device(0)
+    build.build()
+    binding.load_library()
+    name = args.workload
+    steps, warmup = min(args.steps, 2000), max(3, min(args.warmup, 20))
+    if name == "mha_bf16_ablation":
+        w, dtype, n_layers, chunk, new_per_seq = workloads.config_llama13b_mha_ablation(), binding.KV_BF16, 2, 0, 1
+    elif name == "mixed_serving":
+        w, dtype, n_layers, chunk, new_per_seq = workloads.config_mixed_serving(), binding.KV_FP8_E4M3, 2, 0, 1
+    elif name == "long_context":
+        w, dtype, n_layers, chunk, new_per_seq = workloads.config_long_context(), binding.KV_FP8_E4M3, 2, 2048, 0
+    else:
+        w, dtype, n_layers, chunk, new_per_seq = workloads.config_chunked_prefill(), binding.KV_FP8_E4M3, 4, 2048, 512
+    Hq, Hkv, Dh, B = w.num_q_heads, w.num_kv_heads, w.head_dim, w.batch
+    k, v, q = w.k.cuda(), w.v.cuda(), w.q.cuda()
+    is_new = torch.zeros(k.shape[0], dtype=torch.bool)
+    for b in range(B):
+        end = w.kv_offsets[b] + w.context_lens[b]
+        is_new[end - new_per_seq:end] = new_per_seq > 0
+    hist_idx, new_idx = (~is_new).nonzero().squeeze(1).cuda(), is_new.nonzero().squeeze(1).cuda()
+    k_new, v_new = k[new_idx].contiguous(), v[new_idx].contiguous()
+    layers = []
+    for l in range(n_layers):
+        wl = w if l == 0 else workloads.relayout(w, seed=77 + l)
+        cache = binding.Cache(wl.num_blocks, Hkv, Dh, dtype)
+        slots = wl.slot_mapping.cuda()
+        binding.kv_write(cache, k[hist_idx], v[hist_idx], slots[hist_idx])
+        layers.append((cache, wl.block_table.clamp(min=0).cuda(), slots[new_idx].contiguous()))
+    lens, cu = w.context_lens_tensor.cuda(), w.cu_q_lens.cuda()
+    total_q = sum(w.q_lens)
+    ws = binding.new_workspace(B, Hq, Hkv, Dh, w.block_table.shape[1], chunk, total_q)
+    out = torch.empty_like(q)
+
+    def step(i, ev=None):
+        cache, table, slots_new = layers[i % n_layers]
+        if new_per_seq:
+            binding.kv_write(cache, k_new, v_new, slots_new)
+        if ev:
+            ev[0].record()
+        if chunk:
+            binding.paged_chunked(cache, q, cu, table, lens, chunk, True, w.sm_scale, ws, out=out)
+        else:
+            binding.paged_decode(cache, q, table, lens, w.sm_scale, ws, out=out)
+        if ev:
+            ev[1].record()
+
+    for i in range(warmup):
+        step(i)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    stride = max(1, steps // 200)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range((steps + stride - 1) // stride)]
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(torch.cuda.current_device())
+    sampler.start()
+    start.record()
+    for i in range(steps):
+        step(i, evs[i // stride] if i % stride == 0 else None)
+    stop.record()
+    torch.cuda.synchronize()
+    sampler.stop_flag = True
+    assert binding.workspace_status(ws) == 0
+    ms = start.elapsed_time(stop) / steps
+    kernel_ms = sum(a.elapsed_time(b) for a, b in evs) / len(evs)
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peaks = json.load(open(peaks_path)) if os.path.exists(peaks_path) else None
+    esize = 1 if dtype == binding.KV_FP8_E4M3 else 2
+    tokens = sum(w.context_lens)
+    blocks = sum((L + 15) // 16 for L in w.context_lens)
+    kv_bytes = tokens * Hkv * Dh * 2 * esize + (blocks * Hkv * 8 if esize == 1 else 0)
+    if name == "chunked_prefill":
+        pairs = sum(n * (L - n) + n * (n + 1) // 2 for L, n in zip(w.context_lens, w.q_lens))
+        flops = 4.0 * Dh * Hq * pairs
+        peak = peaks["bf16_tflops_sustained"] if peaks else 1400.0
+        achieved = flops / (kernel_ms * 1e-3) / 1e12
+        roofline = {"bound": "tensor", "kernel": "paged_prefill_kernel<128>", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                    "frac": achieved / peak, "peak_source": "measured sustained bf16 (f16 mma has the same nominal rate)" if peaks else "fallback",
+                    "flops_per_launch": flops, "kernel_us": kernel_ms * 1e3, "traffic": None}
+        metric, unit, value = "chunked prefill query tokens/s", "attention-layer query tokens/s", total_q / (ms * 1e-3)
+    else:
+        algo = kv_bytes + 2 * q.numel() * 2 + blocks * 4 + B * 4
+        peak = peaks["hbm_gbs"] if peaks else FALLBACK_HBM_GBS
+        achieved = algo / (kernel_ms * 1e-3) / 1e9
+        kern = "paged_decode_kernel<128> (bf16, mma.sync)" if esize == 2 else "paged_decode_umma_kernel<128,16>"
+        roofline = {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                    "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)" if peaks else "fallback",
+                    "algorithmic_bytes_per_launch": algo, "kernel_us": kernel_ms * 1e3, "traffic": None}
+        metric, unit, value = METRIC, UNIT, B / (ms * 1e-3)
+    line = {"metric": metric, "value": value, "unit": unit, "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if esize == 2 else "fp8_e4m3 cache, fp32 accumulate", "data": "synthetic",
+            "config": {"workload": name, "batch": B, "context_tokens": tokens, "layers_rotated": n_layers,
+                       "l2": "layer caches visited round-robin"},
+            "gpu_launches": steps * (2 if new_per_seq else 1), "clocks": sampler.summary(), "e2e": None, "roofline": roofline,
+            "cpu_baseline": None}
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -179,9 +283,15 @@ def main():
     ap.add_argument("--layers", type=int, default=8, help="layer caches the steps rotate over")
     ap.add_argument("--cpu-seconds", type=float, default=12.0, help="budget of the CPU-baseline leg")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--workload", default="llama13b_decode",
+                    choices=["llama13b_decode", "mha_bf16_ablation", "mixed_serving", "long_context", "chunked_prefill"],
+                    help="llama13b_decode is the benchmark; the others time the remaining configurations (1 GPU, "
+                         "kernel-level line without the end-to-end and CPU legs)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload != "llama13b_decode":
+        return run_other_workload(args)
 
     import torch
     import torch.distributed as dist

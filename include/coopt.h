@@ -115,7 +115,7 @@ int coopt_kv_write(const coopt_cache* cache, const void* k, const void* v, int64
  * The context of every (sequence, kv head) is cut into byte-balanced pieces across the SMs;
  * pieces are merged by a log-sum-exp reduction inside the same launch.
  * Errors: INVALID_ARG, UNSUPPORTED (group size num_q_heads/num_kv_heads not in 1..8 or not
- * integral, batch > 1024, head_dim/block_size/dtype as above), WORKSPACE, CUDA.
+ * integral, batch > 512, head_dim/block_size/dtype as above), WORKSPACE, CUDA.
  */
 int coopt_paged_decode(const coopt_cache* cache, const void* q, void* out, const int32_t* block_table,
                        int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch,
@@ -156,7 +156,7 @@ int coopt_paged_decode_static(const coopt_cache* cache, const void* q, void* out
  *                 sequence; q/out are bf16 [cu_q_lens[batch]][num_q_heads][head_dim]
  *   context_lens  include the new tokens; the n query tokens of a sequence are its last n
  *                 positions and, when causal != 0, query i sees positions 0..len-n+i
- *   chunk_size    tokens per chunk, a multiple of 16, at most 16384
+ *   chunk_size    tokens per chunk, a multiple of 16, at most 32768
  *   total_q       cu_q_lens[batch] as known by the host (sizes the launch)
  * When every sequence has exactly one query token (total_q == batch) each chunk c of
  * (sequence b, query head h) produces m_c (max logit, natural-log units after sm_scale),

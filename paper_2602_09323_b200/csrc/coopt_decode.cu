@@ -369,7 +369,9 @@ size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int bat
 size_t workspace_control_bytes() { return kWsHeaderBytes + static_cast<size_t>(kCounterSlots) * 4; }
 
 int decode_planned_ctas(int num_sms, long long upper_blocks) {
-  const long long need = (upper_blocks + kCap / 2 - 1) / (kCap / 2);
+  // a CTA's slice must fit one round of staged block ids, so that no (sequence, kv head) is cut twice
+  // inside one CTA; slices differ by at most one block from the mean
+  const long long need = (upper_blocks + (kCap - 16) - 1) / (kCap - 16);
   return static_cast<int>(need > num_sms ? need : num_sms);
 }
 int decode_max_batch() { return kMaxBatch; }

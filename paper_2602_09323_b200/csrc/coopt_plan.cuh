@@ -10,9 +10,9 @@
 
 namespace coopt {
 
-constexpr int kCap = 1024;            // block ids staged in shared memory per round
+constexpr int kCap = 2048;            // block ids staged in shared memory per round
 constexpr int kMaxSeg = 32;           // segments planned per round
-constexpr int kMaxBatch = 1024;
+constexpr int kMaxBatch = 512;
 constexpr int kMinBlocksPerCta = 16;
 constexpr int kMaxGroup = 8;
 constexpr int kCounterSlots = 16384;
