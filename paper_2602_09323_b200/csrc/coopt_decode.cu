@@ -60,8 +60,7 @@ __device__ __forceinline__ void mma_top(float& d0, float& d1, uint32_t a0, uint3
   asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%10,%10};"
                : "+f"(d0), "+f"(d1), "=f"(t2), "=f"(t3)
                : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(0.0f));
-  (void)t2;
-  (void)t3;
+  static_cast<void>(t2 + t3);
 }
 
 template <int D>

@@ -88,6 +88,67 @@ def test_skips_growth_and_block_reuse(head_dim, heads):
     assert not codes[4].any()                       # a block nobody wrote stays zero on both sides
 
 
+@pytest.mark.parametrize("head_dim", [64, 128])
+def test_extreme_magnitudes_divide_exactly(head_dim):
+    """Scales from 2^-110 to 2^80 and values down to bf16's subnormals inside one group: the stored
+    code is the encoding of the IEEE fp32 quotient x / s whatever route the kernel takes to it.
+    Whole blocks and partial groups, first writes and growth with re-expression."""
+    rng = np.random.default_rng(7 + head_dim)
+    H, NB = 2, 24
+    cache = binding.Cache(NB, H, head_dim)
+    codes, scales = kv_cache.new_cache(NB, H, head_dim)
+    exps = [-118, -60, -41, -40, -39, -12, 0, 9, 30, 31, 32, 70]          # amax of block b is about 2^exps[b % 12]
+    for call in range(3):
+        slots, ks, vs = [], [], []
+        for b in range(NB):
+            whole = b % 2 == 0
+            offs = list(range(16)) if (whole and call == 0) else ([] if whole else list(range(5 * call, 5 * call + 5)))
+            for o in offs:
+                slots.append(b * 16 + o)
+                mag = 2.0 ** (exps[b % 12] + 2 * call)
+                x = rng.standard_normal((2, H, head_dim)) * mag
+                spread = 2.0 ** rng.integers(-100, 1, size=x.shape)           # mostly far below the block's amax
+                x = np.where(rng.random(x.shape) < 0.5, x * spread, x)
+                x.flat[rng.integers(0, x.size, 4)] = 2.0 ** -133              # bf16 subnormal
+                x.flat[rng.integers(0, x.size, 2)] = -0.0
+                ks.append(x[0]); vs.append(x[1])
+        k = torch.from_numpy(np.stack(ks)).to(torch.bfloat16)
+        v = torch.from_numpy(np.stack(vs)).to(torch.bfloat16)
+        s = torch.tensor(slots, dtype=torch.int64)
+        assert torch.isfinite(k.float()).all() and torch.isfinite(v.float()).all()
+        binding.kv_write(cache, k.cuda(), v.cuda(), s.cuda())
+        kv_cache.kv_write(codes, scales, k.float().numpy(), v.float().numpy(), s.numpy())
+        _compare_fp8(cache, codes, scales, f"call {call}")
+    assert scales.min() < 2.0 ** -100 and scales.max() > 2.0 ** 60
+
+
+def test_long_call_of_scattered_and_contiguous_tokens():
+    """More tokens than the per-token launch takes: runs of a whole block, runs that straddle the
+    tokens one CTA looks at, single tokens in blocks of their own, and skipped tokens between."""
+    rng = np.random.default_rng(11)
+    H, D, NB = 5, 128, 400
+    order = rng.permutation(NB)
+    slots = []
+    for i, b in enumerate(order):
+        kind = i % 4
+        if kind == 0: slots += [b * 16 + o for o in range(16)]
+        elif kind == 1: slots += [b * 16 + o for o in range(3, 14)] + [-1]
+        elif kind == 2: slots += [b * 16 + 7]
+        else: slots += [-1, -1] + [b * 16 + o for o in (0, 1, 2)] + [-5] + [b * 16 + o for o in (9, 4)]
+    T = len(slots)
+    assert T > 512
+    k = torch.from_numpy(rng.standard_normal((T, H, D))).to(torch.bfloat16)
+    v = torch.from_numpy(rng.standard_normal((T, H, D)) * 3).to(torch.bfloat16)
+    s = torch.tensor(slots, dtype=torch.int64)
+    cache = binding.Cache(NB, H, D)
+    codes, scales = kv_cache.new_cache(NB, H, D)
+    for rep in range(2):                       # the second pass meets resident codes and old scales
+        kk = k if rep == 0 else (k * 1.5).to(torch.bfloat16)
+        binding.kv_write(cache, kk.cuda(), v.cuda(), s.cuda())
+        kv_cache.kv_write(codes, scales, kk.float().numpy(), v.float().numpy(), s.numpy())
+        _compare_fp8(cache, codes, scales, f"pass {rep}")
+
+
 def test_strided_token_rows_and_out_of_range_blocks_are_ignored():
     w = workloads.make_workload("strided", [40], 4, 2, 128, seed=3)
     kv = torch.zeros(40, 3, 2, 128, dtype=torch.bfloat16)     # k and v interleaved with padding
