@@ -363,7 +363,8 @@ size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int bat
   size_t bytes = kWsHeaderBytes + static_cast<size_t>(kCounterSlots) * 4;
   const size_t dec = static_cast<size_t>(2) * planned_ctas * group * (head_dim + 2) * 4;
   const size_t chk = static_cast<size_t>(batch) * num_q_heads * max_chunks * (head_dim + 2) * 4;
-  return bytes + (dec > chk ? dec : chk) + 256;
+  // chunk mode holds both: the per-chunk partials it exports and the merged pieces of the CTAs' runs
+  return bytes + (max_chunks > 0 ? chk + dec + 256 : dec) + 256;
 }
 size_t workspace_control_bytes() { return kWsHeaderBytes + static_cast<size_t>(kCounterSlots) * 4; }
 
@@ -430,11 +431,20 @@ int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const in
     p.part_o = reinterpret_cast<float*>(ws + o);
     p.part_m = reinterpret_cast<float*>(ws + m);
     p.part_l = reinterpret_cast<float*>(ws + l);
+    const size_t chunk_rows = static_cast<size_t>(batch) * num_q_heads * p.max_chunks;
+    const size_t run_at = (l + chunk_rows * 4 + 255) / 256 * 256;
+    const size_t rows = static_cast<size_t>(2) * planned_ctas * p.group;
+    p.run_o = reinterpret_cast<float*>(ws + run_at);
+    p.run_m = p.run_o + rows * c->head_dim;
+    p.run_l = p.run_m + rows;
   } else {
     const size_t rows = static_cast<size_t>(2) * planned_ctas * p.group;
     p.part_o = reinterpret_cast<float*>(parts);
     p.part_m = p.part_o + rows * c->head_dim;
     p.part_l = p.part_m + rows;
+    p.run_o = p.part_o;
+    p.run_m = p.part_m;
+    p.run_l = p.part_l;
   }
   // FP8 cache: the tcgen05 kernel; bf16 ablation cache: the mma.sync kernel of this file
   if (c->dtype == COOPT_KV_FP8_E4M3) return launch_paged_decode_umma(p, c->head_dim, planned_ctas, stream);

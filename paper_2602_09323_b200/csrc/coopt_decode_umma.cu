@@ -45,7 +45,6 @@ constexpr int kUmmaThreads = 352;
 constexpr int kTileBlocks = 8;
 constexpr int kTileTokens = kTileBlocks * kBlockSize;  // 128
 constexpr float kLn2 = 0.6931471805599453f;
-constexpr float kLog2eU = 1.4426950408889634f;
 
 template <int D, int NP>
 struct UCfg {
@@ -60,7 +59,8 @@ struct UCfg {
   static constexpr int kStageBytes = kKArea + kVArea;
   static constexpr int kQBytes = 2 * 8 * D;                    // 16 rows x D codes
   static constexpr int kPBytes = NP * kTileTokens;             // NP rows x 128 codes
-  static constexpr int kXchFloats = kGMax * kTeamThreads + 2 * 8;   // team 1's output, maxima and sums of a segment
+  static constexpr int kXchFloats = kGMax * kTeamThreads;            // one team's output of a segment: [head][dim]
+  static constexpr int kMlFloats = 4 * 8 + 8;                       // one team's sums (per warp) and maxima of a segment
   // shared memory carve-up (bytes)
   static constexpr int kRingOff = 0;
   static constexpr int kQOff = kRingOff + kStages * kStageBytes;
@@ -70,9 +70,10 @@ struct UCfg {
   static constexpr int kPreUnitOff = kPreBlkOff + (kMaxBatch + 4) * 4;
   static constexpr int kSegOff = kPreUnitOff + (kMaxBatch + 4) * 4;
   static constexpr int kXchOff = kSegOff + kMaxSeg * static_cast<int>(sizeof(Segment));
-  static constexpr int kRedOff = kXchOff + 2 * kXchFloats * 4;
-  // int red_max [2 teams][4 warps][12], float red_sum [2][4][8], uint red_q [4][8], float qscale [2][8]
-  static constexpr int kRedBytes = (2 * 4 * 12 + 2 * 4 * 8 + 4 * 8 + 2 * 8) * 4;
+  static constexpr int kMlOff = kXchOff + 2 * kXchFloats * 4;       // [2 segment parities][2 teams][kMlFloats]
+  static constexpr int kRedOff = kMlOff + 2 * 2 * kMlFloats * 4;
+  // int red_max [2 teams][4 warps][12], uint red_q [4][8], float qscale [2][8]
+  static constexpr int kRedBytes = (2 * 4 * 12 + 4 * 8 + 2 * 8) * 4;
   static constexpr int kBarOff = kRedOff + kRedBytes;
   static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
@@ -180,6 +181,58 @@ __device__ __forceinline__ uint32_t e4m3_term(uint32_t& h2, float gain) {
   return codes;
 }
 
+// The CTA that delivered the last piece of a (sequence, kv head) merges all pieces by log-sum-exp (the
+// split-KV merge) and writes the bf16 output rows.  One warp; lane l owns dims d0 = 4l .. 4l+3 of every
+// head.  Two pieces at a time: all their (m, l, o) are loaded before any is used, so a batch costs one
+// trip to L2; the running (M, num, den) carries over from batch to batch.  The first piece of a
+// (sequence, kv head) sits in the odd slot of its CTA, the others in the even slot.
+template <int D, int kGMax>
+__device__ __forceinline__ void merge_run_pieces(const float* run_o, const float* run_m, const float* run_l, __nv_bfloat16* out_rows,
+                                              int first_cta, int pieces, int G, int d0) {
+  auto piece = [&](int c, int r) -> size_t { return (static_cast<size_t>(2 * (first_cta + c)) + (c == 0 ? 1 : 0)) * G + r; };
+  float M[kGMax], den[kGMax];
+  float4 nm[kGMax];
+#pragma unroll
+  for (int r = 0; r < kGMax; ++r) { M[r] = -INFINITY; den[r] = 0.0f; nm[r] = make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
+  for (int c0 = 0; c0 < pieces; c0 += 2) {
+    float mc[2][kGMax], lc[2][kGMax];
+    float4 oc[2][kGMax];
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+#pragma unroll
+      for (int r = 0; r < kGMax; ++r) {
+        const bool on = r < G && c0 + k < pieces;
+        const size_t at = on ? piece(c0 + k, r) : 0;
+        mc[k][r] = on ? __ldcg(run_m + at) : 0.0f;
+        lc[k][r] = on ? __ldcg(run_l + at) : 0.0f;
+        oc[k][r] = on ? __ldcg(reinterpret_cast<const float4*>(run_o + at * D + d0)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      }
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+#pragma unroll
+      for (int r = 0; r < kGMax; ++r) {
+        if (lc[k][r] > 0.0f) {
+          const float Mn = fmaxf(M[r], mc[k][r]);
+          const float keep = ex2(M[r] - Mn), wgt = lc[k][r] * ex2(mc[k][r] - Mn);
+          nm[r].x = nm[r].x * keep + wgt * oc[k][r].x;
+          nm[r].y = nm[r].y * keep + wgt * oc[k][r].y;
+          nm[r].z = nm[r].z * keep + wgt * oc[k][r].z;
+          nm[r].w = nm[r].w * keep + wgt * oc[k][r].w;
+          den[r] = den[r] * keep + wgt;
+          M[r] = Mn;
+        }
+      }
+  }
+#pragma unroll
+  for (int r = 0; r < kGMax; ++r) {
+    if (r < G) {
+      const float inv = den[r] > 0.0f ? 1.0f / den[r] : 0.0f;
+      *reinterpret_cast<uint2*>(out_rows + static_cast<size_t>(r) * D + d0) =
+          make_uint2(pack_bf16x2(nm[r].x * inv, nm[r].y * inv), pack_bf16x2(nm[r].z * inv, nm[r].w * inv));
+    }
+  }
+}
+
 template <int D, int NP>
 __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(const DecodeParams p) {
   using C = UCfg<D, NP>;
@@ -196,10 +249,10 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   plan.pre_unit = reinterpret_cast<int*>(smem + C::kPreUnitOff);
   plan.segs = reinterpret_cast<Segment*>(smem + C::kSegOff);
   plan.misc = reinterpret_cast<int*>(smem + C::kMiscOff);          // [0..2] planner
-  float* xch = reinterpret_cast<float*>(smem + C::kXchOff);         // [2 segment parities][kXchFloats]
+  float* xch = reinterpret_cast<float*>(smem + C::kXchOff);         // [2 teams][kXchFloats]
+  float* mlbuf = reinterpret_cast<float*>(smem + C::kMlOff);        // [2 segment parities][2 teams][kMlFloats]
   int* red_max = reinterpret_cast<int*>(smem + C::kRedOff);         // [2][4][12] per-warp maxima of a tile (ordered ints)
-  float* red_sum = reinterpret_cast<float*>(red_max + 2 * 4 * 12);  // [2][4][8]
-  uint32_t* red_q = reinterpret_cast<uint32_t*>(red_sum + 2 * 4 * 8);   // [4][8]
+  uint32_t* red_q = reinterpret_cast<uint32_t*>(red_max + 2 * 4 * 12);   // [4][8]
   float* qscale = reinterpret_cast<float*>(red_q + 4 * 8);          // [2 segment parities][8] logit scale per head
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
   uint64_t* bar_full = bars;                        // [kStages] copies of a tile landed
@@ -209,8 +262,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   uint64_t* bar_pfull = bar_sfree + 4;              // [4] probabilities of a tile are in shared memory (buffer = tile & 3)
   uint64_t* bar_ofree = bar_pfull + 4;              // [4] the team has folded the output buffer into its registers
   uint64_t* bar_qfull = bar_ofree + 4;              // [2] query operand of a segment is in shared memory
-  uint64_t* bar_efull = bar_qfull + 2;              // [2] merged result of a segment is in the exchange area
-  uint64_t* bar_efree = bar_efull + 2;              // [2] the epilogue warp has stored it
+  uint64_t* bar_efull = bar_qfull + 2;              // [2] both teams' pieces of a segment are in the exchange area
+  uint64_t* bar_efree = bar_efull + 2;              // [2] the epilogue warp has read them
   volatile int* abort_flag = plan.misc + 4;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(plan.misc + 5);
 
@@ -230,7 +283,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       mbar_init(&bar_pfull[i], kTeamThreads);
       mbar_init(&bar_ofree[i], 4);
     }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bar_qfull[i], kTeamThreads); mbar_init(&bar_efull[i], kTeamThreads); mbar_init(&bar_efree[i], 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bar_qfull[i], kTeamThreads); mbar_init(&bar_efull[i], kSmThreads); mbar_init(&bar_efree[i], 1); }
     mbar_fence_init();
     *abort_flag = 0;
   }
@@ -363,112 +416,140 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       }
     } else if (warp == kEpilogueWarp) {
       // ================= stores, piece counting and the split-KV merge: off the teams' critical path ========
-      // Lane l owns dims 4l .. 4l+3 of every head.
+      // Lane l owns dims 4l .. 4l+3 of every head.  A run (what this CTA holds of one (sequence, kv head):
+      // one segment in decode mode, several consecutive chunks in chunk mode) is merged in registers; only
+      // runs that do not cover their whole sequence go through the workspace and the piece counter.
       bool ok = true;
       const int d0 = lane * 4;
+      float4 acc[kGMax];                    // the run so far: sum of weight * o, relative to acc_m
+      float acc_m[kGMax], acc_l[kGMax];
+#pragma unroll
+      for (int h = 0; h < kGMax; ++h) { acc[h] = make_float4(0.0f, 0.0f, 0.0f, 0.0f); acc_m[h] = -INFINITY; acc_l[h] = 0.0f; }
       for (int si = 0; si < nseg; ++si, ++seg_no) {
         const Segment sg = plan.segs[si];
         const uint32_t par = seg_no & 1u;
         ok = wait_bar(&bar_efull[par], (seg_no >> 1) & 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        const float* xs = xch + par * C::kXchFloats;
         const int h0 = sg.g * G;
-        if (!sg.partial) {
-          if (d0 < D) {
-            for (int h = 0; h < G; ++h) {
-              const float4 v = *reinterpret_cast<const float4*>(xs + h * kTeamThreads + d0);
-              *reinterpret_cast<uint2*>(p.out + (static_cast<size_t>(sg.b) * Hq + h0 + h) * D + d0) =
-                  make_uint2(pack_bf16x2(v.x, v.y), pack_bf16x2(v.z, v.w));
+        const size_t run_base = static_cast<size_t>(sg.run_slot) * G;
+        // a run that an earlier round of this CTA began: its state was parked in the run's workspace slot
+        if (si == 0 && !(sg.run_flags & kRunFirst)) {
+#pragma unroll
+          for (int h = 0; h < kGMax; ++h) {
+            if (h < G) {
+              if (d0 < D) acc[h] = *reinterpret_cast<const float4*>(p.run_o + (run_base + h) * D + d0);
+              acc_m[h] = p.run_m[run_base + h];
+              acc_l[h] = p.run_l[run_base + h];
             }
           }
-        } else {
-          const size_t base = chunk_mode ? (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks + sg.slot
-                                         : static_cast<size_t>(sg.slot) * G;
-          const size_t pstride = chunk_mode ? static_cast<size_t>(p.max_chunks) : 1;
-          for (int h = 0; h < G; ++h) {
-            if (d0 < D) *reinterpret_cast<float4*>(p.part_o + (base + h * pstride) * D + d0) = *reinterpret_cast<const float4*>(xs + h * kTeamThreads + d0);
-            if (lane == 0) {
-              const float M = xs[kGMax * kTeamThreads + h];
-              p.part_m[base + h * pstride] = chunk_mode ? M * kLn2 : M;   // exported partials use natural-log units
-              p.part_l[base + h * pstride] = xs[kGMax * kTeamThreads + 8 + h];
-            }
-          }
-          __syncwarp();                         // every store of the piece has been issued
-          int last = 0;
-          if (lane == 0) {
-            // release (this CTA's piece is visible before the count moves) and acquire (the other pieces
-            // are visible before they are read) in one round trip
-            int* counter = p.counters + sg.b * Hkv + sg.g;
-            int old;
-            asm volatile("atom.add.acq_rel.gpu.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
-            last = old == sg.expected - 1;
-            if (last) *counter = 0;             // ready for the next call
-          }
-          last = __shfl_sync(0xffffffffu, last, 0);
-          if (last && d0 < D) {
-            // this CTA delivered the last piece: log-sum-exp merge of all pieces (split-K merge).  Two
-            // pieces at a time: all their (m, l, o) are loaded before any is used, so a batch costs one
-            // trip to L2; the running (M, num, den) carries over from batch to batch.
-            int first_cta = 0;
-            if (!chunk_mode) {
-              const long long fs = static_cast<long long>(Hkv) * plan.pre_blk[sg.b] + static_cast<long long>(sg.g) * sg.seq_blocks;
-              first_cta = plan_cta_of(sl, fs);
-            }
-            const size_t cstride = chunk_mode ? 1 : static_cast<size_t>(2) * G;            // between pieces
-            const size_t base0 = chunk_mode ? (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks
-                                            : static_cast<size_t>(2 * first_cta) * G;
-            // decode mode: the first piece sits in the odd slot of its CTA, the others in the even slot
-            auto piece = [&](int c, int r) -> size_t {
-              return base0 + c * cstride + r * pstride + ((!chunk_mode && c == 0) ? static_cast<size_t>(G) : 0);
-            };
-            const float unit = chunk_mode ? kLog2eU : 1.0f;     // exported maxima of chunk mode are natural logs
-            float M[kGMax], den[kGMax];
-            float4 num[kGMax];
+        }
+        // The two teams' running softmaxes are two pieces of the same segment.
+        const float* ml = mlbuf + par * 2 * C::kMlFloats;
+        float4 num[kGMax];
+        float Mh[kGMax], denh[kGMax];
 #pragma unroll
-            for (int r = 0; r < kGMax; ++r) { M[r] = -INFINITY; den[r] = 0.0f; num[r] = make_float4(0.0f, 0.0f, 0.0f, 0.0f); }
-            for (int c0 = 0; c0 < sg.expected; c0 += 2) {
-              float mc[2][kGMax], lc[2][kGMax];
-              float4 oc[2][kGMax];
-#pragma unroll
-              for (int k = 0; k < 2; ++k)
-#pragma unroll
-                for (int r = 0; r < kGMax; ++r) {
-                  const bool on = r < G && c0 + k < sg.expected;
-                  const size_t at = on ? piece(c0 + k, r) : 0;
-                  mc[k][r] = on ? __ldcg(p.part_m + at) : 0.0f;
-                  lc[k][r] = on ? __ldcg(p.part_l + at) : 0.0f;
-                  oc[k][r] = on ? __ldcg(reinterpret_cast<const float4*>(p.part_o + at * D + d0)) : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
-                }
-#pragma unroll
-              for (int k = 0; k < 2; ++k)
-#pragma unroll
-                for (int r = 0; r < kGMax; ++r) {
-                  if (lc[k][r] > 0.0f) {
-                    const float mk = mc[k][r] * unit;
-                    const float Mn = fmaxf(M[r], mk);
-                    const float keep = ex2(M[r] - Mn), wgt = lc[k][r] * ex2(mk - Mn);
-                    num[r].x = num[r].x * keep + wgt * oc[k][r].x;
-                    num[r].y = num[r].y * keep + wgt * oc[k][r].y;
-                    num[r].z = num[r].z * keep + wgt * oc[k][r].z;
-                    num[r].w = num[r].w * keep + wgt * oc[k][r].w;
-                    den[r] = den[r] * keep + wgt;
-                    M[r] = Mn;
-                  }
-                }
-            }
-#pragma unroll
-            for (int r = 0; r < kGMax; ++r) {
-              if (r < G) {
-                const float inv = den[r] > 0.0f ? 1.0f / den[r] : 0.0f;
-                *reinterpret_cast<uint2*>(p.out + (static_cast<size_t>(sg.b) * Hq + h0 + r) * D + d0) =
-                    make_uint2(pack_bf16x2(num[r].x * inv, num[r].y * inv), pack_bf16x2(num[r].z * inv, num[r].w * inv));
-              }
+        for (int h = 0; h < kGMax; ++h) {
+          num[h] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+          Mh[h] = -INFINITY;
+          denh[h] = 0.0f;
+          if (h < G) {
+            const float* a0 = ml, *a1 = ml + C::kMlFloats;
+            const float m0 = a0[32 + h], m1 = a1[32 + h];
+            const float l0 = (a0[h] + a0[8 + h]) + (a0[16 + h] + a0[24 + h]), l1 = (a1[h] + a1[8 + h]) + (a1[16 + h] + a1[24 + h]);
+            const float M = fmaxf(m0, m1);
+            const float mu = M == -INFINITY ? 0.0f : M;
+            const float w0 = ex2(m0 - mu) * (1.0f / 256.0f), w1 = ex2(m1 - mu) * (1.0f / 256.0f);   // outputs are carried times 2^8
+            Mh[h] = M;
+            denh[h] = (l0 * w0 + l1 * w1) * 256.0f;
+            if (d0 < D) {
+              const float4 v0 = *reinterpret_cast<const float4*>(xch + h * kTeamThreads + d0);
+              const float4 v1 = *reinterpret_cast<const float4*>(xch + C::kXchFloats + h * kTeamThreads + d0);
+              num[h] = make_float4(v0.x * w0 + v1.x * w1, v0.y * w0 + v1.y * w1, v0.z * w0 + v1.z * w1, v0.w * w0 + v1.w * w1);
             }
           }
         }
         __syncwarp();
-        if (lane == 0) mbar_arrive(&bar_efree[par]);
+        if (lane == 0) mbar_arrive(&bar_efree[par]);      // the exchange area may take the next segment
+
+        if (chunk_mode) {
+          // Opt-Pa: the chunk's own (m, l, o) is exported, in natural-log units, o normalised
+          const size_t base = (static_cast<size_t>(sg.b) * Hq + h0) * p.max_chunks + sg.slot;
+#pragma unroll
+          for (int h = 0; h < kGMax; ++h) {
+            if (h < G) {
+              const float inv = denh[h] > 0.0f ? 1.0f / denh[h] : 0.0f;
+              const size_t at = base + static_cast<size_t>(h) * p.max_chunks;
+              if (d0 < D) *reinterpret_cast<float4*>(p.part_o + at * D + d0) = make_float4(num[h].x * inv, num[h].y * inv, num[h].z * inv, num[h].w * inv);
+              if (lane == 0) { p.part_m[at] = Mh[h] * kLn2; p.part_l[at] = denh[h]; }
+            }
+          }
+        }
+        // fold the segment into the run
+#pragma unroll
+        for (int h = 0; h < kGMax; ++h) {
+          const float Mn = fmaxf(acc_m[h], Mh[h]);
+          const float mu = Mn == -INFINITY ? 0.0f : Mn;
+          const float ka = ex2(acc_m[h] - mu), kc = ex2(Mh[h] - mu);
+          acc[h] = make_float4(acc[h].x * ka + num[h].x * kc, acc[h].y * ka + num[h].y * kc, acc[h].z * ka + num[h].z * kc, acc[h].w * ka + num[h].w * kc);
+          acc_l[h] = acc_l[h] * ka + denh[h] * kc;
+          acc_m[h] = Mn;
+        }
+        if (!(sg.run_flags & kRunLast)) {
+          // the run goes on; if the round ends here, park it where its merged piece will go later (a run that
+          // covers its whole sequence has no such slot: the CTA's second slot is free until a later run ends)
+          if (si == nseg - 1) {
+#pragma unroll
+            for (int h = 0; h < kGMax; ++h) {
+              if (h < G) {
+                if (d0 < D) *reinterpret_cast<float4*>(p.run_o + (run_base + h) * D + d0) = acc[h];
+                if (lane == 0) { p.run_m[run_base + h] = acc_m[h]; p.run_l[run_base + h] = acc_l[h]; }
+              }
+            }
+            __syncwarp();
+          }
+          continue;
+        }
+        if (sg.run_flags & kRunWhole) {
+          if (d0 < D) {
+#pragma unroll
+            for (int h = 0; h < kGMax; ++h) {
+              if (h < G) {
+                const float inv = acc_l[h] > 0.0f ? 1.0f / acc_l[h] : 0.0f;
+                *reinterpret_cast<uint2*>(p.out + (static_cast<size_t>(sg.b) * Hq + h0 + h) * D + d0) =
+                    make_uint2(pack_bf16x2(acc[h].x * inv, acc[h].y * inv), pack_bf16x2(acc[h].z * inv, acc[h].w * inv));
+              }
+            }
+          }
+#pragma unroll
+          for (int h = 0; h < kGMax; ++h) { acc[h] = make_float4(0.0f, 0.0f, 0.0f, 0.0f); acc_m[h] = -INFINITY; acc_l[h] = 0.0f; }
+          continue;
+        }
+        // the run is one piece of its (sequence, kv head): normalised o, maximum (base-2 units) and sum
+#pragma unroll
+        for (int h = 0; h < kGMax; ++h) {
+          if (h < G) {
+            const float inv = acc_l[h] > 0.0f ? 1.0f / acc_l[h] : 0.0f;
+            if (d0 < D) *reinterpret_cast<float4*>(p.run_o + (run_base + h) * D + d0) = make_float4(acc[h].x * inv, acc[h].y * inv, acc[h].z * inv, acc[h].w * inv);
+            if (lane == 0) { p.run_m[run_base + h] = acc_m[h]; p.run_l[run_base + h] = acc_l[h]; }
+          }
+        }
+#pragma unroll
+        for (int h = 0; h < kGMax; ++h) { acc[h] = make_float4(0.0f, 0.0f, 0.0f, 0.0f); acc_m[h] = -INFINITY; acc_l[h] = 0.0f; }
+        __syncwarp();                         // every store of the piece has been issued
+        int last = 0;
+        if (lane == 0) {
+          // release (this CTA's piece is visible before the count moves) and acquire (the other pieces
+          // are visible before they are read) in one round trip
+          int* counter = p.counters + sg.b * Hkv + sg.g;
+          int old;
+          asm volatile("atom.add.acq_rel.gpu.s32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+          last = old == sg.run_expected - 1;
+          if (last) *counter = 0;             // ready for the next call
+        }
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last && d0 < D)
+          merge_run_pieces<D, kGMax>(p.run_o, p.run_m, p.run_l, p.out + (static_cast<size_t>(sg.b) * Hq + h0) * D, sg.first_cta, sg.run_expected, G, d0);
       }
       if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     } else {
@@ -477,8 +558,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       const int t = tid & (kTeamThreads - 1);
       const int team_bar = 1 + team;
       bool bad = false;     // warp-uniform until a barrier makes it uniform over the team
+      bool team_bad = false;   // uniform over the team: set only behind such a barrier
       int* my_red_max = red_max + team * 48;
-      float* my_red_sum = red_sum + team * 32;
 
       // query operand of a segment (team 0): E4M3 lead term in rows 0..7, remainder term in rows 8..15.
       // The global loads are started a segment ahead (load_q) and consumed after a tile (publish_q).
@@ -528,6 +609,44 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         bad = barrier_or(team_bar, kTeamThreads, bad);   // every thread has read the exchange words before the next query reuses them
         fence_proxy_async();
         mbar_arrive(&bar_qfull[segc & 1u]);
+      };
+
+      // The piece of the segment before: its last product is folded in, and the piece handed to the
+      // epilogue warp, behind the team's first tile of the next segment (flush_old), so that the end of a
+      // segment does not wait for the tensor core.
+      bool old_open = false, old_has_tile = false;
+      uint32_t old_tile = 0, old_seg = 0;
+      float o_old[kGMax], vref_old = 0.0f;
+#pragma unroll
+      for (int h = 0; h < kGMax; ++h) o_old[h] = 0.0f;
+      auto flush_old = [&]() {
+        bool ok = !bad;
+        if (ok && old_has_tile) ok = wait_bar(&bar_empty[old_tile % C::kStages], (old_tile / C::kStages) & 1u, abort_flag);
+        // the exchange area was last read by the epilogue warp for the segment before that one
+        if (ok && old_seg >= 1) ok = wait_bar(&bar_efree[(old_seg - 1) & 1u], ((old_seg - 1) >> 1) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok);
+        bad = bad || !ok;
+        old_open = false;
+        if (bad) return;
+        if (old_has_tile) {
+          uint32_t r[NP];
+          tc_fence_after();
+          const uint32_t obuf = tmem_o + NP * (old_tile & 3u) + lane_base;
+#pragma unroll
+          for (int half = 0; half < NP / 16; ++half) tmem_ld16_issue(obuf + half * 16, *reinterpret_cast<uint32_t(*)[16]>(&r[half * 16]));
+#pragma unroll
+          for (int half = 0; half < NP / 16; ++half) tmem_ld_wait(*reinterpret_cast<uint32_t(*)[16]>(&r[half * 16]));
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bar_ofree[old_tile & 3u]);
+#pragma unroll
+          for (int h = 0; h < kGMax; ++h)
+            o_old[h] += __uint_as_float(r[h]) + __uint_as_float(r[kGMax + h]) * 0.0625f + __uint_as_float(r[2 * kGMax + h]) * 0.00390625f;
+        }
+        float* xo = xch + team * C::kXchFloats;
+#pragma unroll
+        for (int h = 0; h < kGMax; ++h) xo[h * kTeamThreads + t] = o_old[h] * vref_old;
+        mbar_arrive(&bar_efull[old_seg & 1u]);
       };
 
       if (team == 0 && nseg > 0) { load_q(plan.segs[0]); publish_q(seg_no); }
@@ -611,7 +730,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             if (lane == 0) rw[8] = wv;
           }
           bad = barrier_or(team_bar, kTeamThreads, bad);
-          if (bad) break;
+          if (bad) { team_bad = true; break; }
           const int* rmx = my_red_max;
           // reference V scale: the largest met so far by the team in the segment (uniform over the team)
           const float vmax = __int_as_float(max(max(rmx[8], rmx[20]), max(rmx[32], rmx[44])));
@@ -676,65 +795,36 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           pending = true;
           pend_tile = tile_no;
           if (q_due) { publish_q(seg_no + 1); q_due = false; }
+          if (old_open) flush_old();
         }
         // (a team whose wait ran out keeps company until the next barrier makes it known to everybody)
         if (q_due) publish_q(seg_no + 1);   // the segment had no tile for this team
 
-        // ---- end of segment: fold the last product, reduce the sums, merge the two teams ---------------
-        if (pending) {
-          uint32_t o_raw[NP];
-          fold_issue(o_raw);
-          fold_finish(o_raw);
-        }
-#pragma unroll
-        for (int h = 0; h < kGMax; ++h) {
-          const float ws = warp_sum(l_run[h]);
-          if (lane == 0) my_red_sum[wq * 8 + h] = ws;
-        }
-        bad = barrier_or(team_bar, kTeamThreads, bad);
-        float lsum[kGMax], acc_m[kGMax], acc_l[kGMax];
-#pragma unroll
-        for (int h = 0; h < kGMax; ++h) lsum[h] = (my_red_sum[h] + my_red_sum[8 + h]) + (my_red_sum[16 + h] + my_red_sum[24 + h]);
-        float* xs = xch + (seg_no & 1u) * C::kXchFloats;
-        if (team == 1) {
-          // the area was last used two segments ago; the epilogue warp must be done with it
-          if (seg_no >= 2) {
-            bool ok = !bad && wait_bar(&bar_efree[seg_no & 1u], ((seg_no >> 1) - 1) & 1u, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            bad = bad || !ok;
-          }
+        // ---- end of segment: the team's sums and maxima go to the epilogue warp now, its output follows
+        // once the last product has been folded in (flush_old, behind the next segment's first tile)
+        if (team_bad) break;
+        if (old_open) flush_old();            // the segment gave this team no tile
+        {
+          // (the area of this parity was last read for segment seg_no - 2, which the flush of segment
+          // seg_no - 1 has waited for)
+          float* mls = mlbuf + ((seg_no & 1u) * 2 + team) * C::kMlFloats;
 #pragma unroll
           for (int h = 0; h < kGMax; ++h) {
-            xs[h * kTeamThreads + t] = o_reg[h] * vref;
-            if (t == 0) { xs[kGMax * kTeamThreads + h] = m_run[h]; xs[kGMax * kTeamThreads + 8 + h] = lsum[h]; }
+            const float ws = warp_sum(l_run[h]);
+            if (lane == 0) mls[wq * 8 + h] = ws;
+            if (t == 0) mls[32 + h] = m_run[h];
           }
         }
-        bad = barrier_or(3, kSmThreads, bad);
-        if (bad) break;
-        if (team == 0) {
-          // the other team's running softmax is one more piece of the same segment; the merged, normalised
-          // result goes back into the exchange area, from where the epilogue warp stores it
+        old_open = true;
+        old_has_tile = pending;
+        old_tile = pend_tile;
+        old_seg = seg_no;
+        vref_old = vref;
 #pragma unroll
-          for (int h = 0; h < kGMax; ++h) {
-            const float m1 = xs[kGMax * kTeamThreads + h], l1 = xs[kGMax * kTeamThreads + 8 + h];
-            const float M = fmaxf(m_run[h], m1);
-            const float mu = M == -INFINITY ? 0.0f : M;
-            const float w0 = ex2(m_run[h] - mu), w1 = ex2(m1 - mu);
-            const float den = lsum[h] * w0 + l1 * w1;
-            const float num = o_reg[h] * vref * w0 + xs[h * kTeamThreads + t] * w1;
-            xs[h * kTeamThreads + t] = den > 0.0f ? num * (1.0f / 256.0f) / den : 0.0f;
-            acc_m[h] = M;
-            acc_l[h] = den;
-          }
-          bad = barrier_or(team_bar, kTeamThreads, bad);     // every thread has read the other team's maxima and sums
-          if (t == 0) {
-#pragma unroll
-            for (int h = 0; h < kGMax; ++h) { xs[kGMax * kTeamThreads + h] = acc_m[h]; xs[kGMax * kTeamThreads + 8 + h] = acc_l[h]; }
-          }
-          mbar_arrive(&bar_efull[seg_no & 1u]);
-        }
+        for (int h = 0; h < kGMax; ++h) o_old[h] = pending ? o_reg[h] * a_prev[h] : 0.0f;
         ++seg_no;
       }
+      if (old_open) flush_old();              // the round's last segment
       if (bad && t == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     }
 

@@ -27,7 +27,14 @@ struct Segment {
   int expected;      // partial: number of pieces the (sequence, kv head) is cut into
   int seq_blocks;    // blocks of the whole sequence
   int ctx_len;       // tokens of the whole sequence
+  // A run is what one CTA holds of one (sequence, kv head): in chunk mode several consecutive chunks,
+  // which the tcgen05 kernel merges on chip before anything is counted; in decode mode the segment itself.
+  int run_flags;     // kRunFirst | kRunLast | kRunWhole
+  int run_slot;      // workspace slot of the run's merged piece (two per CTA)
+  int run_expected;  // number of CTAs that hold a run of this (sequence, kv head)
+  int first_cta;     // the first of them
 };
+constexpr int kRunFirst = 1, kRunLast = 2, kRunWhole = 4;
 
 struct DecodeParams {
   const uint8_t* cache;
@@ -47,6 +54,9 @@ struct DecodeParams {
   float* part_o;           // decode: [2P][G][D]        chunk: [B][Hq][max_chunks][D]
   float* part_m;           // decode: [2P][G]           chunk: [B][Hq][max_chunks]
   float* part_l;
+  float* run_o;            // merged pieces of runs, [2P][G][D] (decode mode: the same arrays as part_*)
+  float* run_m;            // [2P][G], base-2 logarithm units
+  float* run_l;
 };
 
 #ifdef __CUDACC__
@@ -114,11 +124,13 @@ __device__ inline void plan_prefix(const DecodeParams& p, const PlanSmem& s, int
 // The slice [lo, hi) of the flat block list that belongs to this CTA; false if it has none.
 struct PlanSlice {
   long long lo, hi, N;
+  long long ulo, uhi, U;     // chunk mode: the same slice in units of (sequence, kv head, chunk)
   int P;
 };
 __device__ inline bool plan_slice(const DecodeParams& p, const PlanSmem& s, PlanSlice& sl) {
   const int B = p.batch, Hkv = p.num_kv_heads;
   sl.N = static_cast<long long>(Hkv) * s.pre_blk[B];
+  sl.ulo = sl.uhi = sl.U = 0;
   if (sl.N == 0) return false;
   if (p.chunk_blocks == 0) {
     sl.P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), max(1ll, sl.N / kMinBlocksPerCta)));
@@ -141,6 +153,7 @@ __device__ inline bool plan_slice(const DecodeParams& p, const PlanSmem& s, Plan
   };
   sl.lo = unit_to_block(ulo);
   sl.hi = unit_to_block(uhi);
+  sl.ulo = ulo; sl.uhi = uhi; sl.U = U;
   return true;
 }
 // CTA that owns flat block index x (decode mode).
@@ -175,14 +188,28 @@ __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, cons
     sg.seq_blocks = nb;
     sg.ctx_len = 0;     // filled in by plan_stage_ids, off this thread's serial path
     if (chunk_mode) {
+      const int nch = s.pre_unit[cb + 1] - s.pre_unit[cb], c = cj / p.chunk_blocks;
       sg.partial = 1;
-      sg.slot = cj / p.chunk_blocks;
-      sg.expected = s.pre_unit[cb + 1] - s.pre_unit[cb];
+      sg.slot = c;
+      sg.expected = nch;
+      // the CTA's run of this (sequence, kv head): units [max(fu, ulo), min(fu + nch, uhi))
+      const long long fu = static_cast<long long>(Hkv) * s.pre_unit[cb] + static_cast<long long>(cg) * nch, u = fu + c;
+      const int Un = static_cast<int>(sl.U);
+      const int cta_f = static_cast<int>(plan_div((fu + 1) * sl.P - 1, Un)), cta_l = static_cast<int>(plan_div((fu + nch) * sl.P - 1, Un));
+      sg.first_cta = cta_f;
+      sg.run_expected = cta_l - cta_f + 1;
+      sg.run_slot = 2 * blockIdx.x + (cta_f < static_cast<int>(blockIdx.x) ? 0 : 1);
+      sg.run_flags = ((c == 0 || u == sl.ulo) ? kRunFirst : 0) | ((c == nch - 1 || u == sl.uhi - 1) ? kRunLast : 0) |
+                     (cta_l == cta_f ? kRunWhole : 0);
     } else {
       sg.partial = !(cj == 0 && n == nb);
       sg.slot = 2 * blockIdx.x + (cj > 0 ? 0 : 1);
       const long long fs = static_cast<long long>(Hkv) * s.pre_blk[cb] + static_cast<long long>(cg) * nb;
-      sg.expected = plan_cta_of(sl, fs + nb - 1) - plan_cta_of(sl, fs) + 1;
+      sg.first_cta = plan_cta_of(sl, fs);
+      sg.expected = plan_cta_of(sl, fs + nb - 1) - sg.first_cta + 1;
+      sg.run_flags = kRunFirst | kRunLast | (sg.partial ? 0 : kRunWhole);
+      sg.run_slot = sg.slot;
+      sg.run_expected = sg.expected;
     }
     s.segs[nseg++] = sg;
     used += static_cast<int>(n);
