@@ -152,6 +152,24 @@ def test_chunked_decode_partials_and_merge(chunk):
         assert np.allclose(o_c[b, h, :n].cpu().numpy(), o, rtol=5e-3, atol=2e-2)
 
 
+@pytest.mark.parametrize("lens,hq,hkv", [([100000], 2, 1), ([640] * 220 + [37, 1300], 2, 1), ([3000] * 70, 4, 2)])
+def test_chunked_decode_runs_that_span_planning_rounds(lens, hq, hkv):
+    """Chunks of one block: a CTA holds more chunks of one (sequence, kv head) than one planning round
+    lists, so the run it merges on chip is parked in the workspace between rounds, both for runs that
+    are one piece of their sequence and for runs that cover their sequence whole.  Run twice on the same
+    workspace: the piece counters must have been left ready."""
+    w = workloads.make_workload("rounds", lens, hq, hkv, 64, seed=21)
+    cache = helpers.gpu_fill(w)
+    ref = _oracle_out(w)
+    ws = binding.new_workspace(w.batch, hq, hkv, 64, w.block_table.shape[1], 16, w.batch)
+    q, table, lens_t, cu = w.q.cuda(), w.block_table.cuda(), w.context_lens_tensor.cuda(), w.cu_q_lens.cuda()
+    for rep in range(2):
+        out = binding.paged_chunked(cache, q, cu, table, lens_t, 16, True, w.sm_scale, ws)
+        torch.cuda.synchronize()
+        assert binding.workspace_status(ws) == 0
+        helpers.check_attention(out, ref, what=f"rounds rep {rep}")
+
+
 def _oracle_sequence_cache(w, b, g, calls):
     """Oracle cache of one sequence and kv head, written by the given (start, stop) row ranges."""
     k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
