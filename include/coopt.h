@@ -172,6 +172,22 @@ int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, cons
                         float sm_scale, void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * coopt_decode_step — one serving step with DEVICE inputs (Algorithm 1: phase 1, the new token of
+ * every sequence is written to the cache; phase 2 and Algorithms 2-3, attention over the updated
+ * cache): coopt_kv_write(k_new, v_new, slot_mapping, num_tokens = batch) followed by
+ * coopt_paged_decode, with the same arguments, results and errors as those two calls made one after
+ * the other, in one call.
+ *   k_new, v_new   DEVICE bf16 [batch][num_kv_heads][head_dim], kv_token_stride elements apart
+ *   slot_mapping   DEVICE int64 [batch]
+ *   context_lens   DEVICE int32 [batch], counting the new token
+ * All arguments are checked before anything is launched.
+ */
+int coopt_decode_step(const coopt_cache* cache, const void* k_new, const void* v_new, int64_t kv_token_stride,
+                      const int64_t* slot_mapping, const void* q, void* out, const int32_t* block_table,
+                      int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                      float sm_scale, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * coopt_decode_step_host — one serving step for callers whose step inputs live in HOST memory
  * (Section 2's token-insertion phase followed by the attention phase): copies the step's
  * inputs to the device, runs coopt_kv_write for the one new token of every sequence and

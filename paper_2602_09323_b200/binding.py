@@ -59,6 +59,10 @@ _SIGNATURES = {
                                + [ctypes.c_void_p] * 2 + [ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
                                                           ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
                                                           ctypes.c_size_t, ctypes.c_void_p]),
+    "coopt_decode_step": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
+                                         ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                                         ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_void_p,
+                                         ctypes.c_size_t, ctypes.c_void_p]),
     "coopt_step_staging_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 5),
     "coopt_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "coopt_version": (ctypes.c_int, []),
@@ -172,6 +176,22 @@ def paged_decode(cache: Cache, q: torch.Tensor, block_table: torch.Tensor, conte
                                            _ptr(context_lens), q.shape[0], q.shape[1], float(sm_scale),
                                            _ptr(workspace), workspace.numel(), _stream())
     _check(st, "coopt_paged_decode")
+    return out
+
+
+def decode_step(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, slot_mapping: torch.Tensor, q: torch.Tensor,
+                block_table: torch.Tensor, context_lens: torch.Tensor, sm_scale: float, workspace: torch.Tensor,
+                out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """coopt_decode_step: the new token of every sequence written, then decode attention, as one call."""
+    assert q.dtype == torch.bfloat16 and q.is_contiguous() and block_table.dtype == torch.int32 and block_table.is_contiguous()
+    assert k_new.dtype == torch.bfloat16 and v_new.dtype == torch.bfloat16 and k_new.is_contiguous() and v_new.is_contiguous()
+    assert slot_mapping.dtype == torch.int64 and context_lens.dtype == torch.int32
+    if out is None:
+        out = torch.empty_like(q)
+    st = load_library().coopt_decode_step(cache.ref(), _ptr(k_new), _ptr(v_new), k_new.shape[1] * k_new.shape[2], _ptr(slot_mapping),
+                                          _ptr(q), _ptr(out), _ptr(block_table), block_table.shape[1], _ptr(context_lens),
+                                          q.shape[0], q.shape[1], float(sm_scale), _ptr(workspace), workspace.numel(), _stream())
+    _check(st, "coopt_decode_step")
     return out
 
 

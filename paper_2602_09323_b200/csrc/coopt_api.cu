@@ -169,6 +169,26 @@ int coopt_paged_decode(const coopt_cache* cache, const void* q, void* out, const
                              0, workspace, P, static_cast<cudaStream_t>(stream));
 }
 
+int coopt_decode_step(const coopt_cache* cache, const void* k_new, const void* v_new, int64_t kv_token_stride,
+                      const int64_t* slot_mapping, const void* q, void* out, const int32_t* block_table,
+                      int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                      float sm_scale, void* workspace, size_t workspace_bytes, void* stream) {
+  // every check of both halves before anything is launched
+  int rc = check_attention_args(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads);
+  if (rc != COOPT_OK) return rc;
+  if (!k_new || !v_new || !slot_mapping || kv_token_stride < static_cast<int64_t>(cache->num_kv_heads) * cache->head_dim)
+    return COOPT_ERR_INVALID_ARG;
+  if (batch == 0) return COOPT_OK;
+  if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, cache->num_kv_heads, cache->head_dim,
+                                                            max_blocks_per_seq, 0, batch))
+    return COOPT_ERR_WORKSPACE;
+  rc = launch_kv_write(cache, k_new, v_new, kv_token_stride, slot_mapping, batch, static_cast<cudaStream_t>(stream));
+  if (rc != COOPT_OK) return rc;
+  const int P = planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq);
+  return launch_paged_decode(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads, sm_scale,
+                             0, workspace, P, static_cast<cudaStream_t>(stream));
+}
+
 int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, const int32_t* cu_q_lens,
                         const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
                         int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t chunk_size, int32_t causal,
@@ -244,12 +264,10 @@ int coopt_decode_step_host(const coopt_cache* cache, const void* q_host, const v
   ok &= cudaMemcpyAsync(dev + s.table, block_table_host, static_cast<size_t>(batch) * max_blocks_per_seq * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
   ok &= cudaMemcpyAsync(dev + s.lens, context_lens_host, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
   if (!ok) return COOPT_ERR_CUDA;
-  rc = coopt_kv_write(cache, dev + s.k, dev + s.v, static_cast<int64_t>(hkv) * d,
-                      reinterpret_cast<const int64_t*>(dev + s.slots), batch, stream);
-  if (rc != COOPT_OK) return rc;
-  rc = coopt_paged_decode(cache, dev + s.q, dev + s.out, reinterpret_cast<const int32_t*>(dev + s.table),
-                          max_blocks_per_seq, reinterpret_cast<const int32_t*>(dev + s.lens), batch, num_q_heads,
-                          sm_scale, workspace, workspace_bytes, stream);
+  rc = coopt_decode_step(cache, dev + s.k, dev + s.v, static_cast<int64_t>(hkv) * d, reinterpret_cast<const int64_t*>(dev + s.slots),
+                         dev + s.q, dev + s.out, reinterpret_cast<const int32_t*>(dev + s.table), max_blocks_per_seq,
+                         reinterpret_cast<const int32_t*>(dev + s.lens), batch, num_q_heads, sm_scale, workspace,
+                         workspace_bytes, stream);
   if (rc != COOPT_OK) return rc;
   return cudaMemcpyAsync(out_host, dev + s.out, qb, cudaMemcpyDeviceToHost, st) == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }

@@ -866,7 +866,8 @@ int launch_umma_one(const DecodeParams& p, int grid, cudaStream_t stream) {
 
 // FP8 cache: group sizes 1..5 use 16 probability rows, 6..8 use 32.
 int launch_paged_decode_umma(const DecodeParams& p, int head_dim, int grid, cudaStream_t stream) {
-  if (p.group <= 5) return head_dim == 128 ? launch_umma_one<128, 16>(p, grid, stream) : launch_umma_one<64, 16>(p, grid, stream);
+  if (p.group <= 5)
+    return head_dim == 128 ? launch_umma_one<128, 16>(p, grid, stream) : launch_umma_one<64, 16>(p, grid, stream);
   return head_dim == 128 ? launch_umma_one<128, 32>(p, grid, stream) : launch_umma_one<64, 32>(p, grid, stream);
 }
 

@@ -170,6 +170,44 @@ def test_chunked_decode_runs_that_span_planning_rounds(lens, hq, hkv):
         helpers.check_attention(out, ref, what=f"rounds rep {rep}")
 
 
+def test_decode_step_equals_write_then_decode_bit_for_bit():
+    """Token by token over the last 40 positions of every sequence, the one-call step and the two
+    separate calls must leave identical cache bytes and identical outputs, and the outputs must match
+    the oracle at the end."""
+    w = workloads.make_workload("step", [300, 64, 2048, 1500, 47, 900], 10, 2, 128, seed=17)
+    rows = np.concatenate([np.arange(w.kv_offsets[b], w.kv_offsets[b] + L - 40) for b, L in enumerate(w.context_lens)])
+    rows_t = torch.from_numpy(rows).cuda()
+    k, v, slots = w.k.cuda(), w.v.cuda(), w.slot_mapping.cuda()
+    table, q = w.block_table.cuda(), w.q.cuda()
+    caches = []
+    for _ in range(2):
+        c = binding.Cache(w.num_blocks, 2, 128)
+        binding.kv_write(c, k[rows_t], v[rows_t], slots[rows_t])
+        caches.append(c)
+    ws = [binding.new_workspace(w.batch, 10, 2, 128, w.block_table.shape[1]) for _ in range(2)]
+    outs = [None, None]
+    for step in range(40):
+        new = torch.tensor([w.kv_offsets[b] + L - 40 + step for b, L in enumerate(w.context_lens)]).cuda()
+        lens = torch.tensor([L - 40 + step + 1 for L in w.context_lens], dtype=torch.int32).cuda()
+        k_new, v_new, s_new = k[new].contiguous(), v[new].contiguous(), slots[new].contiguous()
+        outs[0] = binding.decode_step(caches[0], k_new, v_new, s_new, q, table, lens, w.sm_scale, ws[0])
+        binding.kv_write(caches[1], k_new, v_new, s_new)
+        outs[1] = binding.paged_decode(caches[1], q, table, lens, w.sm_scale, ws[1])
+        torch.cuda.synchronize()
+        assert binding.workspace_status(ws[0]) == 0 and binding.workspace_status(ws[1]) == 0
+        assert torch.equal(outs[0], outs[1]), f"step {step}: outputs differ"
+        assert torch.equal(caches[0].data, caches[1].data), f"step {step}: cache bytes differ"
+    # the oracle fills the same way: the history of every sequence in one call, then 40 single-token calls
+    codes, scales = kv_cache.new_cache(w.num_blocks, 2, 128)
+    kf, vf, sf = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
+    kv_cache.kv_write(codes, scales, kf[rows], vf[rows], sf[rows])
+    for step in range(40):
+        new = np.array([w.kv_offsets[b] + L - 40 + step for b, L in enumerate(w.context_lens)])
+        kv_cache.kv_write(codes, scales, kf[new], vf[new], sf[new])
+    ref = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), w.context_lens)
+    helpers.check_attention(outs[0], ref, what="decode step")
+
+
 def _oracle_sequence_cache(w, b, g, calls):
     """Oracle cache of one sequence and kv head, written by the given (start, stop) row ranges."""
     k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
