@@ -17,9 +17,12 @@
 //
 // One CTA per SM walks its slice of the flat (sequence, kv head, block) list in tiles of eight
 // cache blocks (128 tokens).  Warp roles:
-//   warp 8      issues the copies of a tile (per granule: the K part, and the V part with the header)
-//               into a ring of stages; an mbarrier per stage counts the bytes;
-//   warp 9      one lane issues the matrix instructions and commits them to mbarriers;
+//   warp 8      issues the copies of a tile into a ring of stages, an mbarrier per stage counting the
+//               bytes.  The cache is one 2-D tensor (row = granule) to the copy engine; one gather
+//               request fetches the same columns of four granules (their K parts, their V parts, or
+//               their headers), so a tile of eight granules costs six requests;
+//   warps 9, 11 one lane each issues the matrix instructions of the logits (warp 9) and of the outputs
+//               (warp 11) and commits them to mbarriers;
 //   warps 0-3, 4-7   two softmax teams; even tiles go to team 0, odd tiles to team 1, so two tiles are
 //               always in flight.  Thread t of a team reads the logits of token t from tensor memory,
 //               takes part in the per-head maximum (one redux per head, then a shared-memory step
@@ -32,6 +35,8 @@
 // delivers the last piece merges all pieces by log-sum-exp and writes the bf16 output.
 // Every wait is bounded; a wait that runs out is reported in the workspace status word and all roles
 // leave through the common exit, which frees the tensor memory.
+#include <cuda.h>
+
 #include "coopt_plan.cuh"
 
 namespace coopt {
@@ -40,8 +45,8 @@ namespace {
 
 constexpr int kTeamThreads = 128;                     // four warps: one per 32 tensor-memory lanes
 constexpr int kSmThreads = 2 * kTeamThreads;          // warps 0-7
-constexpr int kProducerWarp = 8, kMmaWarp = 9, kEpilogueWarp = 10;
-constexpr int kUmmaThreads = 352;
+constexpr int kProducerWarp = 8, kMmaWarp = 9, kEpilogueWarp = 10, kPvWarp = 11;
+constexpr int kUmmaThreads = 384;
 constexpr int kTileBlocks = 8;
 constexpr int kTileTokens = kTileBlocks * kBlockSize;  // 128
 constexpr float kLn2 = 0.6931471805599453f;
@@ -50,13 +55,15 @@ template <int D, int NP>
 struct UCfg {
   static constexpr int kGran = granule_bytes(D, true);
   static constexpr int kPart = kBlockSize * D;                 // K (or V) codes of one granule
-  static constexpr int kVSlot = kPart + kFp8Header;            // V codes and the header of one granule: one copy
+  static constexpr int kGatherRows = 4;                        // granules per gather request
   static constexpr int kGMax = NP == 16 ? 5 : 8;               // head slots per probability term
   static constexpr int kTmemCols = NP == 16 ? 128 : 256;       // 4 x 16 logits columns + 4 x NP output columns
   static constexpr int kStages = D == 128 ? (NP == 16 ? 6 : 5) : 8;
   static constexpr int kKArea = kTileBlocks * kPart;
-  static constexpr int kVArea = kTileBlocks * kVSlot + (D == 64 ? kPart : 0);   // D = 64: rows 64..127 of the 128-row operand read on
-  static constexpr int kStageBytes = kKArea + kVArea;
+  static constexpr int kVArea = kTileBlocks * kPart + (D == 64 ? kPart : 0);   // D = 64: rows 64..127 of the 128-row operand read on
+  static constexpr int kHdrOff = kKArea + kVArea;               // the eight headers (scales) of the tile
+  static constexpr int kStageBytes = kHdrOff + kTileBlocks * kFp8Header;
+  static constexpr int kGroupBytes = kGatherRows * (2 * kPart + kFp8Header);   // what the three requests of four granules bring
   static constexpr int kQBytes = 2 * 8 * D;                    // 16 rows x D codes
   static constexpr int kPBytes = NP * kTileTokens;             // NP rows x 128 codes
   static constexpr int kXchFloats = kGMax * kTeamThreads;            // one team's output of a segment: [head][dim]
@@ -78,7 +85,9 @@ struct UCfg {
   static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kSmemBytes = kMiscOff + 64;
-  static_assert(kStageBytes % 16 == 0 && kVSlot % 16 == 0, "bulk copies need 16-byte granularity");
+  static_assert(kStageBytes % 128 == 0 && kKArea % 128 == 0 && kHdrOff % 128 == 0 && (kGatherRows * kPart) % 128 == 0 &&
+                    (kGatherRows * kFp8Header) % 128 == 0, "tensor copies land on 128-byte boundaries");
+  static_assert(kPart / 8 <= 256 && kGran % 16 == 0, "one box row is at most 256 eight-byte elements");
   static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
 };
 
@@ -119,6 +128,13 @@ __device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[16]) {
                :: "memory");
 }
 
+// One request: columns [x, x + box width) (in 8-byte elements) of the four rows r0..r3 of the 2-D tensor,
+// landing as four consecutive box rows in shared memory; completes on the mbarrier with its byte count.
+__device__ __forceinline__ void gather4_g2s(void* dst, const CUtensorMap* map, int x, int r0, int r1, int r2, int r3, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar)) : "memory");
+}
+
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
@@ -128,14 +144,6 @@ __device__ __forceinline__ bool barrier_or(int id, int count, bool flag) {
   asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %3, 0;\n barrier.cta.red.or.pred q, %1, %2, p;\n selp.u32 %0, 1, 0, q;\n}"
                : "=r"(r) : "r"(id), "r"(count), "r"(static_cast<uint32_t>(flag)) : "memory");
   return r != 0;
-}
-// Non-blocking look at a phase of an mbarrier: the instruction-issuing lane polls with it, because it
-// always has something else to look at.
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
-               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
 }
 // Bounded wait that also gives up when another role has already given up.  try_wait lets the hardware
 // park the warp, so waiting warps do not take issue slots from the two single-lane roles that share
@@ -234,7 +242,8 @@ __device__ __forceinline__ void merge_run_pieces(const float* run_o, const float
 }
 
 template <int D, int NP>
-__global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(const DecodeParams p) {
+__global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(const DecodeParams p, const __grid_constant__ CUtensorMap map_part,
+                                                                            const __grid_constant__ CUtensorMap map_hdr) {
   using C = UCfg<D, NP>;
   constexpr int kGMax = C::kGMax;
   constexpr int kKSteps = D / 32;                 // 32 codes per instruction along the contraction
@@ -323,93 +332,90 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
     __syncthreads();
 
     if (warp == kProducerWarp) {
-      // ================= copies: per granule the K part, and the V part with the header ================
-      // Lane 2i copies the K part of granule i of the tile, lane 2i + 1 its V part and header.  The
-      // addresses of a tile are worked out before the lane that watches the ring looks at the stage, so
-      // that the copy engine's queue is refilled with as little of a gap as possible.
+      // ================= copies: six gather requests per tile ==================================================
+      // Lane 3 q + w (q = 0, 1; w = 0, 1, 2) fetches the K parts (w = 0), the V parts (w = 1) or the headers
+      // (w = 2) of granules 4 q .. 4 q + 3 of the tile.  Rows past the tile's last granule repeat its first
+      // one: their tokens are masked out of the softmax.  The rows of a tile are worked out before the lane
+      // that watches the ring looks at the stage, so that the copy engine's queue is refilled with as little
+      // of a gap as possible.
       bool ok = true;
-      const int gi = lane >> 1;
-      const uint32_t src_off = (lane & 1) ? C::kPart : 0u, bytes = (lane & 1) ? C::kVSlot : C::kPart;
-      const uint32_t dst_off = (lane & 1) ? C::kKArea + gi * C::kVSlot : gi * C::kPart;
+      const int q4 = lane / 3, what = lane - 3 * q4;
+      const int x = what * (C::kPart / 8);                    // first column, in 8-byte elements
+      const uint32_t dst_off = what == 0 ? q4 * C::kGatherRows * C::kPart
+                             : what == 1 ? C::kKArea + q4 * C::kGatherRows * C::kPart
+                                         : C::kHdrOff + q4 * C::kGatherRows * kFp8Header;
+      const CUtensorMap* map = what == 2 ? &map_hdr : &map_part;
       for (int si = 0; si < nseg && ok; ++si) {
         const int n = plan.segs[si].n, g = plan.segs[si].g;
         const int* seg_ids = plan.ids + plan.segs[si].list_off;
         for (int k0 = 0; k0 < n; k0 += kTileBlocks) {
           const int nb = min(kTileBlocks, n - k0);
-          const uint8_t* src = nullptr;
-          if (lane < 2 * nb) src = p.cache + (static_cast<size_t>(seg_ids[k0 + gi]) * Hkv + g) * C::kGran + src_off;
+          const int ngroups = (nb + C::kGatherRows - 1) / C::kGatherRows;
+          int rows[C::kGatherRows] = {0, 0, 0, 0};
+          if (lane < 3 * ngroups) {
+#pragma unroll
+            for (int i = 0; i < C::kGatherRows; ++i) {
+              const int j = q4 * C::kGatherRows + i;
+              rows[i] = seg_ids[k0 + (j < nb ? j : 0)] * Hkv + g;
+            }
+          }
           const uint32_t stage = tile_no % C::kStages, use = tile_no / C::kStages;
           uint8_t* st = ring + stage * C::kStageBytes;
           if (lane == 0) {
             if (use > 0) ok = wait_bar(&bar_empty[stage], (use - 1) & 1u, abort_flag);
-            if (ok) mbar_expect_tx(&bar_full[stage], nb * C::kGran);
+            if (ok) mbar_expect_tx(&bar_full[stage], ngroups * C::kGroupBytes);
           }
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) break;
-          if (lane < 2 * nb) bulk_copy_g2s(st + dst_off, src, bytes, &bar_full[stage]);
+          if (lane < 3 * ngroups) gather4_g2s(st + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[stage]);
           ++tile_no;
         }
       }
       if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     } else if (warp == kMmaWarp) {
-      // ================= matrix instructions (one lane) ====================================================
+      // ================= logits: S^T = Ktile . Qg^T (one lane) ================================================
+      // Runs ahead of the softmax teams by up to four tiles (four logits buffers).  A single thread issues
+      // few instructions per cycle, so the two kinds of matrix instruction have a lane (and a warp
+      // scheduler) each, and the operand descriptors of a tile are one addition away from constants.
       if (lane == 0) {
-        // Two cursors over the round's tiles.  The logits cursor (a_*) runs ahead of the P V cursor by at
-        // most four tiles (four logits buffers) and at most into the segment after the one whose P V is
-        // due (the query of a later segment is published only once that one has begun).  Neither kind of
-        // instruction waits for the other: whichever has its inputs ready is issued, P V first.
         bool ok = true;
-        int a_si = 0, a_k0 = 0, v_si = 0, v_k0 = 0;
-        uint32_t a_tile = tile_no, a_seg = seg_no;
-        uint64_t t0 = 0;
-        uint32_t idle = 0;
-        while (ok && v_si < nseg) {
-          bool progress = false;
-          // ---- P V of tile `tile_no`
-          {
-            const uint32_t buf = tile_no & 3u, use = tile_no >> 2;
-            if (mbar_test(&bar_pfull[buf], use & 1u) && (use == 0 || mbar_test(&bar_ofree[buf], (use - 1) & 1u))) {
-              const int n = plan.segs[v_si].n;
-              const int nb = min(kTileBlocks, n - v_k0);
-              const uint32_t stage = tile_no % C::kStages;
-              tc_fence_after();
-              const uint32_t va = smem_u32(ring + stage * C::kStageBytes + C::kKArea);
-              const uint32_t pa = smem_u32(pbuf + buf * C::kPBytes);
-              const int nks = (nb + 1) >> 1;                  // 32 tokens (two granules) per instruction
-              for (int ks = 0; ks < nks; ++ks)
-                umma_f8(tmem_o + NP * buf, umma_desc(va + ks * 2 * C::kVSlot, C::kVSlot, 128), umma_desc(pa + ks * 256, 128, 1024), umma_idesc(NP),
-                        ks > 0 ? 1u : 0u);
-              umma_commit(&bar_empty[stage]);     // the stage is free again and the tile's product is in its output buffer
-              ++tile_no;
-              v_k0 += kTileBlocks;
-              if (v_k0 >= n) { v_k0 = 0; ++v_si; ++seg_no; }
-              progress = true;
-            }
-          }
-          // ---- logits of tile `a_tile`
-          if (a_si < nseg && a_tile < tile_no + 4 && a_seg <= seg_no + 1) {
-            const uint32_t stage = a_tile % C::kStages, buf = a_tile & 3u, use = a_tile >> 2;
-            if (mbar_test(&bar_full[stage], (a_tile / C::kStages) & 1u) && (use == 0 || mbar_test(&bar_sfree[buf], (use - 1) & 1u)) &&
-                (a_k0 > 0 || mbar_test(&bar_qfull[a_seg & 1u], (a_seg >> 1) & 1u))) {
-              tc_fence_after();
-              const uint32_t ka = smem_u32(ring + stage * C::kStageBytes);
-              const uint32_t qa = smem_u32(qbuf + (a_seg & 1u) * C::kQBytes);
+        const uint64_t desc_k = umma_desc(smem_u32(ring), 128, kSboRows), desc_q = umma_desc(smem_u32(qbuf), 128, kSboRows);
+        for (int si = 0; si < nseg && ok; ++si, ++seg_no) {
+          const int n = plan.segs[si].n;
+          ok = wait_bar(&bar_qfull[seg_no & 1u], (seg_no >> 1) & 1u, abort_flag);
+          const uint64_t dq = desc_q + (((seg_no & 1u) * C::kQBytes) >> 4);
+          for (int k0 = 0; k0 < n && ok; k0 += kTileBlocks, ++tile_no) {
+            const uint32_t stage = tile_no % C::kStages, buf = tile_no & 3u, use = tile_no >> 2;
+            ok = wait_bar(&bar_full[stage], (tile_no / C::kStages) & 1u, abort_flag);
+            if (ok && use > 0) ok = wait_bar(&bar_sfree[buf], (use - 1) & 1u, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t dk = desc_k + ((stage * C::kStageBytes) >> 4);
 #pragma unroll
-              for (int ks = 0; ks < kKSteps; ++ks)
-                umma_f8(tmem + 16 * buf, umma_desc(ka + ks * 256, 128, kSboRows), umma_desc(qa + ks * 256, 128, kSboRows), umma_idesc(16), ks > 0);
-              umma_commit(&bar_sfull[buf]);
-              ++a_tile;
-              a_k0 += kTileBlocks;
-              if (a_k0 >= plan.segs[a_si].n) { a_k0 = 0; ++a_si; ++a_seg; }
-              progress = true;
-            }
+            for (int ks = 0; ks < kKSteps; ++ks) umma_f8(tmem + 16 * buf, dk + ks * 16, dq + ks * 16, umma_idesc(16), ks > 0);
+            umma_commit(&bar_sfull[buf]);
           }
-          if (progress) { idle = 0; t0 = 0; continue; }
-          if ((++idle & 0xFFFu) == 0) {      // bounded: nothing became ready for a long time
-            if (*abort_flag != 0) ok = false;
-            const uint64_t now = global_timer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; ok = false; }
+        }
+        if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+      }
+    } else if (warp == kPvWarp) {
+      // ================= outputs: O^T = V^T . Pg^T of a tile into its own buffer (one lane) ==================
+      if (lane == 0) {
+        bool ok = true;
+        const uint64_t desc_v = umma_desc(smem_u32(ring + C::kKArea), C::kPart, 128), desc_p = umma_desc(smem_u32(pbuf), 128, 1024);
+        for (int si = 0; si < nseg && ok; ++si) {
+          const int n = plan.segs[si].n;
+          for (int k0 = 0; k0 < n && ok; k0 += kTileBlocks, ++tile_no) {
+            const uint32_t stage = tile_no % C::kStages, buf = tile_no & 3u, use = tile_no >> 2;
+            ok = wait_bar(&bar_pfull[buf], use & 1u, abort_flag);
+            if (ok && use > 0) ok = wait_bar(&bar_ofree[buf], (use - 1) & 1u, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint64_t dv = desc_v + ((stage * C::kStageBytes) >> 4), dp = desc_p + ((buf * C::kPBytes) >> 4);
+            const int nks = (min(kTileBlocks, n - k0) + 1) >> 1;      // 32 tokens (two granules) per instruction
+            for (int ks = 0; ks < nks; ++ks)
+              umma_f8(tmem_o + NP * buf, dv + ks * ((2 * C::kPart) >> 4), dp + ks * 16, umma_idesc(NP), ks > 0 ? 1u : 0u);
+            umma_commit(&bar_empty[stage]);     // the stage is free again and the tile's product is in its output buffer
           }
         }
         if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
@@ -694,8 +700,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           const int nb = min(kTileBlocks, sg.n - k0);
           const uint32_t stage = tile_no % C::kStages, buf = tile_no & 3u;
           uint8_t* st = ring + stage * C::kStageBytes;
-          // scales of the granule that holds token t: the header travels behind the granule's V codes
-          const float* hdr = reinterpret_cast<const float*>(st + C::kKArea + (t >> 4) * C::kVSlot + C::kPart);
+          // scales of the granule that holds token t
+          const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + (t >> 4) * kFp8Header);
           const int tok0 = (sg.j0 + k0) * kBlockSize;
           const int ntok = min(nb * kBlockSize, sg.ctx_len - tok0);            // Eq. 9: tail of the context
           const uint32_t sbuf = tile_no & 3u;
@@ -767,7 +773,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             }
             // V codes of slots past the context inside the last block are cleared (row t = dim t of V^T)
             if ((ntok & 15) != 0 && t < D) {
-              uint4* row = reinterpret_cast<uint4*>(st + C::kKArea + (ntok >> 4) * C::kVSlot + (t >> 3) * 128 + (t & 7) * 16);
+              uint4* row = reinterpret_cast<uint4*>(st + C::kKArea + (ntok >> 4) * C::kPart + (t >> 3) * 128 + (t & 7) * 16);
               const int keep = ntok & 15;
               uint4 w = *row;
               uint32_t* ww = reinterpret_cast<uint32_t*>(&w);
@@ -780,7 +786,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             }
             // an odd number of blocks: the last instruction also reads the slot behind them
             if ((nb & 1) != 0 && t < D)
-              *reinterpret_cast<uint4*>(st + C::kKArea + nb * C::kVSlot + (t >> 3) * 128 + (t & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+              *reinterpret_cast<uint4*>(st + C::kKArea + nb * C::kPart + (t >> 3) * 128 + (t & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
             fence_proxy_async();
             mbar_arrive(&bar_pfull[buf]);
           }
@@ -847,9 +853,35 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   if (warp == kMmaWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
 }
 
+// The cache as the copy engine sees it: [granules][granule bytes / 8] 8-byte elements, one box row of
+// `box_elems` elements per gathered granule.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+bool encode_cache_map(CUtensorMap* map, const void* cache, long long granules, int gran_bytes, int box_elems) {
+  static TensorMapEncodeFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult res;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess || !fn) return false;
+    encode = reinterpret_cast<TensorMapEncodeFn>(fn);
+  }
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(gran_bytes / 8), static_cast<cuuint64_t>(granules)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(gran_bytes)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_elems), 1}, elem_strides[2] = {1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(cache), dims, strides, box, elem_strides,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int D, int NP>
 int launch_umma_one(const DecodeParams& p, int grid, cudaStream_t stream) {
   using C = UCfg<D, NP>;
+  CUtensorMap map_part, map_hdr;
+  const long long granules = static_cast<long long>(p.num_blocks) * p.num_kv_heads;
+  if (!encode_cache_map(&map_part, p.cache, granules, C::kGran, C::kPart / 8) ||
+      !encode_cache_map(&map_hdr, p.cache, granules, C::kGran, kFp8Header / 8))
+    return COOPT_ERR_CUDA;
   static bool configured[64] = {};
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
@@ -858,7 +890,7 @@ int launch_umma_one(const DecodeParams& p, int grid, cudaStream_t stream) {
       return COOPT_ERR_CUDA;
     configured[dev] = true;
   }
-  paged_decode_umma_kernel<D, NP><<<grid, kUmmaThreads, C::kSmemBytes, stream>>>(p);
+  paged_decode_umma_kernel<D, NP><<<grid, kUmmaThreads, C::kSmemBytes, stream>>>(p, map_part, map_hdr);
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
 
