@@ -457,7 +457,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch on this workload, from the
 # ncu capture summarised under profiles/ (None while the kernel is newer than the capture).
-DRAM_TRAFFIC_PER_LAUNCH = 136.14e6 + 3.74e6
+DRAM_TRAFFIC_PER_LAUNCH = 136.18e6 + 4.16e6
 
 if __name__ == "__main__":
     main()
