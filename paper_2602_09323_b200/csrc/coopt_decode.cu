@@ -42,7 +42,7 @@ struct Cfg {
   static constexpr int kMergeOff = kSegOff + kMaxSeg * static_cast<int>(sizeof(Segment));
   static constexpr int kMergeStride = D + 4;    // floats per (warp, row): o[D], m, l, pad
   static constexpr int kMiscOff = kMergeOff + kWarps * kMaxGroup * kMergeStride * 4;
-  static constexpr int kSmemBytes = kMiscOff + 64;
+  static constexpr int kSmemBytes = kMiscOff + 128;
 };
 
 __device__ __forceinline__ float quad_max(float x) {
@@ -84,11 +84,16 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
   // ---- plan: blocks (and chunks) per sequence, this CTA's slice of the flat block list ---------
   PlanSmem plan;
   plan.pre_blk = pre_blk; plan.pre_unit = pre_unit; plan.segs = segs; plan.ids = ids; plan.misc = misc;
+  plan.slice = reinterpret_cast<long long*>(smem + C::kMiscOff + 64);
+  int ctx_early[2];
+  plan_prefix_load(p, tid, kThreads, ctx_early);
   if (tid == 0) {
     for (int i = 0; i < kWarps * C::kStages; ++i) mbar_init(&bars[i], 1);
     mbar_fence_init();
   }
-  plan_prefix(p, plan, tid, kThreads);
+  plan_prefix(p, plan, tid, kThreads, ctx_early);
+  if (tid == 0) plan_slice_publish(p, plan);
+  __syncthreads();
 
   // sequences with an empty context: all-zero output rows
   for (int b = blockIdx.x; b < B; b += gridDim.x) {
@@ -97,7 +102,7 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
   }
 
   PlanSlice sl;
-  if (!plan_slice(p, plan, sl)) return;
+  if (!plan_slice_fetch(plan, sl)) return;
   const long long lo = sl.lo, hi = sl.hi;
   auto cta_of = [&](long long x) -> int { return plan_cta_of(sl, x); };
 
@@ -114,6 +119,7 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
     __syncthreads();
     const int nseg = misc[0];
     const long long x_next = (static_cast<long long>(misc[2]) << 32) | static_cast<unsigned int>(misc[1]);
+    if (tid < nseg) plan_round_finish(p, plan, sl, tid);
     plan_stage_ids(p, plan, nseg, tid, kThreads);
     __syncthreads();
 

@@ -31,7 +31,10 @@
 //               P V product of each tile lands in a buffer of its own and is folded in one tile later,
 //               so the tensor memory is never rescaled.  Each team keeps its own running maximum and
 //               sum; at the end of a segment the two are merged like two split-KV pieces.
-// A segment that does not cover its whole sequence leaves (m, l, o) in the workspace; the CTA that
+//   warp 10     the epilogue: merges the two teams' pieces of a segment, folds the consecutive segments of one
+//               (sequence, kv head) that this CTA holds into a run (chunk mode: consecutive chunks, each also
+//               exported as its own (m, l, o)), and writes a run that covers its sequence straight to the output.
+// A run that does not cover its whole sequence leaves (m, l, o) in the workspace; the CTA that
 // delivers the last piece merges all pieces by log-sum-exp and writes the bf16 output.
 // Every wait is bounded; a wait that runs out is reported in the workspace status word and all roles
 // leave through the common exit, which frees the tensor memory.
@@ -84,7 +87,7 @@ struct UCfg {
   static constexpr int kBarOff = kRedOff + kRedBytes;
   static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2;
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kSmemBytes = kMiscOff + 64;
+  static constexpr int kSmemBytes = kMiscOff + 128;            // 64 bytes of planner words and flags, 64 of the published slice
   static_assert(kStageBytes % 128 == 0 && kKArea % 128 == 0 && kHdrOff % 128 == 0 && (kGatherRows * kPart) % 128 == 0 &&
                     (kGatherRows * kFp8Header) % 128 == 0, "tensor copies land on 128-byte boundaries");
   static_assert(kPart / 8 <= 256 && kGran % 16 == 0, "one box row is at most 256 eight-byte elements");
@@ -258,6 +261,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   plan.pre_unit = reinterpret_cast<int*>(smem + C::kPreUnitOff);
   plan.segs = reinterpret_cast<Segment*>(smem + C::kSegOff);
   plan.misc = reinterpret_cast<int*>(smem + C::kMiscOff);          // [0..2] planner
+  plan.slice = reinterpret_cast<long long*>(smem + C::kMiscOff + 64);
   float* xch = reinterpret_cast<float*>(smem + C::kXchOff);         // [2 teams][kXchFloats]
   float* mlbuf = reinterpret_cast<float*>(smem + C::kMlOff);        // [2 segment parities][2 teams][kMlFloats]
   int* red_max = reinterpret_cast<int*>(smem + C::kRedOff);         // [2][4][12] per-warp maxima of a tile (ordered ints)
@@ -281,6 +285,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   const bool chunk_mode = p.chunk_blocks > 0;
 
   // ---- set-up ---------------------------------------------------------------------------------------
+  // two trips to memory start before anything else: the context lengths for the planner, and the copy
+  // engine's view of the cache (fetched on first use otherwise, in front of the first tile)
+  int ctx_early[2];
+  plan_prefix_load(p, tid, kUmmaThreads, ctx_early);
+  if (tid == kProducerWarp * 32) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_part) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hdr) : "memory");
+  }
   // rows of Qg / Pg that no head uses must hold zero codes
   for (int i = tid; i < (C::kIdsOff - C::kQOff) / 16; i += kUmmaThreads)
     reinterpret_cast<uint4*>(smem + C::kQOff)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -300,7 +312,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  plan_prefix(p, plan, tid, kUmmaThreads);
+  plan_prefix(p, plan, tid, kUmmaThreads, ctx_early);
+  if (tid == 0) plan_slice_publish(p, plan);
   // sequences with an empty context: all-zero output rows
   for (int b = blockIdx.x; b < B; b += gridDim.x) {
     if (plan.pre_blk[b + 1] == plan.pre_blk[b])
@@ -315,7 +328,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   const uint32_t lane_base = static_cast<uint32_t>(warp & 3) * 32u << 16;
 
   PlanSlice sl;
-  const bool active = plan_slice(p, plan, sl);
+  const bool active = plan_slice_fetch(plan, sl);
 
   // counters that persist across rounds (every role advances its own copy identically)
   uint32_t tile_no = 0;     // tiles so far: ring stage, and team / buffer = tile_no & 1
@@ -328,6 +341,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
     __syncthreads();
     const int nseg = plan.misc[0];
     const long long x_next = (static_cast<long long>(plan.misc[2]) << 32) | static_cast<unsigned int>(plan.misc[1]);
+    if (tid < nseg) plan_round_finish(p, plan, sl, tid);
     plan_stage_ids(p, plan, nseg, tid, kUmmaThreads);
     __syncthreads();
 

@@ -68,6 +68,7 @@ struct PlanSmem {
   Segment* segs;     // [kMaxSeg]
   int* ids;          // [kCap]
   int* misc;         // [4]: nseg, next x (lo, hi), scratch flag
+  long long* slice;  // [8]: the CTA's slice as one thread worked it out (plan_slice_publish)
 };
 
 // floor(a / b) for 0 <= a < 2^52, 0 < b < 2^31: one double division and a fix-up instead of the
@@ -89,12 +90,25 @@ __device__ __forceinline__ int plan_find_seq(const int* pre, int batch, long lon
   return lo;
 }
 
+// The context lengths this thread will turn into block counts: loaded as early as the kernel can, so
+// that the trip to memory overlaps the rest of the set-up.  (kMaxBatch <= 2 * the smallest CTA.)
+__device__ __forceinline__ void plan_prefix_load(const DecodeParams& p, int tid, int nthreads, int (&L)[2]) {
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int b = tid + k * nthreads;
+    L[k] = b < p.batch ? p.context_lens[b] : 0;
+  }
+}
+
 // Blocks (and chunks) per sequence and their prefix sums.  Every thread of the CTA calls this.
-__device__ inline void plan_prefix(const DecodeParams& p, const PlanSmem& s, int tid, int nthreads) {
+__device__ inline void plan_prefix(const DecodeParams& p, const PlanSmem& s, int tid, int nthreads, const int (&Lin)[2]) {
   const int B = p.batch;
   const bool chunk_mode = p.chunk_blocks > 0;
-  for (int b = tid; b < B; b += nthreads) {
-    int L = p.context_lens[b];
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const int b = tid + k * nthreads;
+    if (b >= B) break;
+    int L = Lin[k];
     L = max(0, min(L, p.max_blocks_per_seq * kBlockSize));
     const int nb = (L + kBlockSize - 1) / kBlockSize;
     s.pre_blk[b + 1] = nb;
@@ -156,13 +170,26 @@ __device__ inline bool plan_slice(const DecodeParams& p, const PlanSmem& s, Plan
   sl.ulo = ulo; sl.uhi = uhi; sl.U = U;
   return true;
 }
+// One thread works the slice out (its divisions are double-precision: a whole CTA doing them at once
+// queues on the few units an SM has) and leaves it in shared memory; after a barrier everybody fetches it.
+__device__ inline void plan_slice_publish(const DecodeParams& p, const PlanSmem& s) {
+  PlanSlice sl;
+  const bool active = plan_slice(p, s, sl);
+  s.slice[0] = sl.lo; s.slice[1] = sl.hi; s.slice[2] = sl.N; s.slice[3] = sl.ulo; s.slice[4] = sl.uhi; s.slice[5] = sl.U;
+  s.slice[6] = sl.P; s.slice[7] = active ? 1 : 0;
+}
+__device__ inline bool plan_slice_fetch(const PlanSmem& s, PlanSlice& sl) {
+  sl.lo = s.slice[0]; sl.hi = s.slice[1]; sl.N = s.slice[2]; sl.ulo = s.slice[3]; sl.uhi = s.slice[4]; sl.U = s.slice[5];
+  sl.P = static_cast<int>(s.slice[6]);
+  return s.slice[7] != 0;
+}
 // CTA that owns flat block index x (decode mode).
 __device__ __forceinline__ int plan_cta_of(const PlanSlice& sl, long long x) {
   return static_cast<int>(plan_div((x + 1) * sl.P - 1, static_cast<int>(sl.N)));
 }
 
-// One thread plans the next round starting at flat index x: fills segs, misc[0] = number of
-// segments, misc[1..2] = where the following round starts.
+// One thread plans the next round starting at flat index x: fills the geometry of segs (plan_round_finish
+// adds the rest), misc[0] = number of segments, misc[1..2] = where the following round starts.
 __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, const PlanSlice& sl, long long x) {
   const int B = p.batch, Hkv = p.num_kv_heads;
   const bool chunk_mode = p.chunk_blocks > 0;
@@ -187,30 +214,8 @@ __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, cons
     sg.b = cb; sg.g = cg; sg.j0 = cj; sg.n = static_cast<int>(n); sg.list_off = used;
     sg.seq_blocks = nb;
     sg.ctx_len = 0;     // filled in by plan_stage_ids, off this thread's serial path
-    if (chunk_mode) {
-      const int nch = s.pre_unit[cb + 1] - s.pre_unit[cb], c = cj / p.chunk_blocks;
-      sg.partial = 1;
-      sg.slot = c;
-      sg.expected = nch;
-      // the CTA's run of this (sequence, kv head): units [max(fu, ulo), min(fu + nch, uhi))
-      const long long fu = static_cast<long long>(Hkv) * s.pre_unit[cb] + static_cast<long long>(cg) * nch, u = fu + c;
-      const int Un = static_cast<int>(sl.U);
-      const int cta_f = static_cast<int>(plan_div((fu + 1) * sl.P - 1, Un)), cta_l = static_cast<int>(plan_div((fu + nch) * sl.P - 1, Un));
-      sg.first_cta = cta_f;
-      sg.run_expected = cta_l - cta_f + 1;
-      sg.run_slot = 2 * blockIdx.x + (cta_f < static_cast<int>(blockIdx.x) ? 0 : 1);
-      sg.run_flags = ((c == 0 || u == sl.ulo) ? kRunFirst : 0) | ((c == nch - 1 || u == sl.uhi - 1) ? kRunLast : 0) |
-                     (cta_l == cta_f ? kRunWhole : 0);
-    } else {
-      sg.partial = !(cj == 0 && n == nb);
-      sg.slot = 2 * blockIdx.x + (cj > 0 ? 0 : 1);
-      const long long fs = static_cast<long long>(Hkv) * s.pre_blk[cb] + static_cast<long long>(cg) * nb;
-      sg.first_cta = plan_cta_of(sl, fs);
-      sg.expected = plan_cta_of(sl, fs + nb - 1) - sg.first_cta + 1;
-      sg.run_flags = kRunFirst | kRunLast | (sg.partial ? 0 : kRunWhole);
-      sg.run_slot = sg.slot;
-      sg.run_expected = sg.expected;
-    }
+    sg.partial = chunk_mode ? 1 : !(cj == 0 && n == nb);
+    sg.slot = sg.expected = sg.run_flags = sg.run_slot = sg.run_expected = sg.first_cta = 0;   // plan_round_finish
     s.segs[nseg++] = sg;
     used += static_cast<int>(n);
     xx += n;
@@ -227,6 +232,39 @@ __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, cons
   s.misc[0] = nseg;
   s.misc[1] = static_cast<int>(xx & 0xffffffffll);
   s.misc[2] = static_cast<int>(xx >> 32);
+}
+
+// What plan_round left out of segment k: the fields that cost divisions.  Thread k of the CTA calls this
+// for k < number of segments, so the segments' divisions run side by side.
+__device__ inline void plan_round_finish(const DecodeParams& p, const PlanSmem& s, const PlanSlice& sl, int k) {
+  const int Hkv = p.num_kv_heads;
+  const bool chunk_mode = p.chunk_blocks > 0;
+  Segment& sg = s.segs[k];
+  const int nb = sg.seq_blocks;
+  {
+    if (chunk_mode) {
+      const int nch = s.pre_unit[sg.b + 1] - s.pre_unit[sg.b], c = sg.j0 / p.chunk_blocks;
+      sg.slot = c;
+      sg.expected = nch;
+      // the CTA's run of this (sequence, kv head): units [max(fu, ulo), min(fu + nch, uhi))
+      const long long fu = static_cast<long long>(Hkv) * s.pre_unit[sg.b] + static_cast<long long>(sg.g) * nch, u = fu + c;
+      const int Un = static_cast<int>(sl.U);
+      const int cta_f = static_cast<int>(plan_div((fu + 1) * sl.P - 1, Un)), cta_l = static_cast<int>(plan_div((fu + nch) * sl.P - 1, Un));
+      sg.first_cta = cta_f;
+      sg.run_expected = cta_l - cta_f + 1;
+      sg.run_slot = 2 * blockIdx.x + (cta_f < static_cast<int>(blockIdx.x) ? 0 : 1);
+      sg.run_flags = ((c == 0 || u == sl.ulo) ? kRunFirst : 0) | ((c == nch - 1 || u == sl.uhi - 1) ? kRunLast : 0) |
+                     (cta_l == cta_f ? kRunWhole : 0);
+    } else {
+      sg.slot = 2 * blockIdx.x + (sg.j0 > 0 ? 0 : 1);
+      const long long fs = static_cast<long long>(Hkv) * s.pre_blk[sg.b] + static_cast<long long>(sg.g) * nb;
+      sg.first_cta = plan_cta_of(sl, fs);
+      sg.expected = plan_cta_of(sl, fs + nb - 1) - sg.first_cta + 1;
+      sg.run_flags = kRunFirst | kRunLast | (sg.partial ? 0 : kRunWhole);
+      sg.run_slot = sg.slot;
+      sg.run_expected = sg.expected;
+    }
+  }
 }
 
 // Physical block ids of every planned segment -> shared memory (range-checked: a bad id is
