@@ -12,8 +12,8 @@ import sys
 PKG_DIR = os.path.dirname(os.path.abspath(__file__))
 SRC_DIR = os.path.join(PKG_DIR, "csrc")
 LIB_PATH = os.path.join(PKG_DIR, "libcoopt.so")
-SOURCES = ["coopt_api.cu", "coopt_write.cu", "coopt_decode.cu", "coopt_decode_umma.cu", "coopt_prefill.cu", "coopt_static.cu"]
-HEADERS = ["coopt_common.cuh", "coopt_plan.cuh", os.path.join("..", "..", "include", "coopt.h")]
+SOURCES = ["coopt_api.cu", "coopt_write.cu", "coopt_decode.cu", "coopt_decode_umma.cu", "coopt_prefill.cu", "coopt_prefill_umma.cu", "coopt_static.cu"]
+HEADERS = ["coopt_common.cuh", "coopt_plan.cuh", "coopt_umma.cuh", os.path.join("..", "..", "include", "coopt.h")]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
     "--shared", "-Xcompiler", "-fPIC", "-cudart", "static", "--expt-relaxed-constexpr",

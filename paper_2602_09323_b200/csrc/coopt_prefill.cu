@@ -413,11 +413,19 @@ int launch_prefill_one(const PrefillParams& p, dim3 grid, cudaStream_t stream) {
 
 }  // namespace
 
+int launch_paged_prefill_umma(const coopt_cache* c, const void* q, void* out, const int32_t* cu_q_lens, const int32_t* block_table,
+                              int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                              int32_t total_q, int32_t causal, float sm_scale, void* workspace, cudaStream_t stream);
+
 int launch_paged_prefill(const coopt_cache* c, const void* q, void* out, const int32_t* cu_q_lens,
                          const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
                          int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t causal, float sm_scale,
                          void* workspace, cudaStream_t stream) {
   if (c->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;
+  // head_dim 128: the tcgen05 kernel; head_dim 64: the mma.sync kernel of this file
+  if (c->head_dim == 128)
+    return launch_paged_prefill_umma(c, q, out, cu_q_lens, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads,
+                                     total_q, causal, sm_scale, workspace, stream);
   PrefillParams p;
   p.cache = static_cast<const uint8_t*>(c->data);
   p.q = static_cast<const __nv_bfloat16*>(q);

@@ -1,0 +1,549 @@
+// Chunked prefill against the paged FP8 cache on the 5th-generation tensor cores (head_dim 128): Eq. 1
+// with the causal K_{<=t}, Eq. 6 dequantisation on load, Eq. 7-8 grouped-query sharing, Eq. 9 valid
+// blocks only, Eq. 10 max-subtracted softmax, for runs of several query tokens per sequence.
+//
+// A CTA owns one (sequence, kv head, tile of consecutive query tokens).  Its 128 rows are the (query
+// token, query head of the group) pairs of the tile, so the K/V stream of the kv head is fetched once
+// for all G heads (Algorithm 2).  The E4M3 codes of the cache feed tcgen05.mma kind::f8f6f4 as they are:
+//     S [128 rows x 128 keys] = Q  [128 x D] . Ktile^T      Q as two exact E4M3 terms of the bf16 query
+//     O [128 rows x D]       += P  [128 x 128 keys] . Vtile  P as three E4M3 terms of the probabilities
+// with fp32 accumulators in tensor memory.  The K scale of a block multiplies the logits of its 16 keys,
+// the V scale is folded into the probabilities.
+//
+// The context is walked twice, 128 keys (eight cache blocks) at a time.  The first walk fetches K only and
+// leaves every row's maximum logit (and the largest V scale); the second recomputes the logits, so every
+// probability is exp(s - final maximum) <= 1 and the output accumulator in tensor memory is never
+// rescaled.  The second product over K costs a third more tensor work and K traffic (out of L2), and
+// removes the read-modify-write of 128 x 128 accumulators whenever a maximum moves.
+//
+// Warp roles (352 threads):
+//   warps 0-3, 4-7   two softmax teams, even and odd tiles; thread r of a team owns row r: it reads the
+//               row's 128 logits from tensor memory 16 at a time (one cache block: one pair of scales),
+//               so maxima and sums need no exchange between threads;
+//   warp 8      copies: gather requests over the tensor map of the cache (K parts, V parts, headers of
+//               four granules each) into a ring of three stages;
+//   warp 9      one lane issues the S instructions; warp 10 one lane issues the P V instructions.
+// Every wait is bounded; a wait that runs out is reported in the status word and all roles leave through
+// the common exit, which frees the tensor memory.
+#include "coopt_umma.cuh"
+
+namespace coopt {
+
+namespace {
+
+constexpr int kPuTeam = 128;
+constexpr int kPuSm = 2 * kPuTeam;
+constexpr int kPuProducer = 8, kPuSWarp = 9, kPuPvWarp = 10;
+constexpr int kPuThreads = 352;
+constexpr int kPuTileBlocks = 8;
+constexpr int kPuTileKeys = kPuTileBlocks * kBlockSize;   // 128
+constexpr int kPuD = 128;
+constexpr int kPuStages = 3;
+constexpr float kPuLog2e = 1.4426950408889634f;
+constexpr float kPuGain = 256.0f;                          // probabilities are carried times 2^8 (at most 256 < 448)
+
+struct PrefillUmmaParams {
+  const __nv_bfloat16* q;
+  __nv_bfloat16* out;
+  const int* cu_q_lens;
+  const int* block_table;
+  const int* context_lens;
+  int max_blocks_per_seq;
+  int batch, num_q_heads, num_kv_heads, group;
+  int num_blocks;
+  int tile_queries;        // query tokens per CTA = 128 / group
+  int causal;
+  float sm_scale_log2;
+  int* status;
+};
+
+struct PuCfg {
+  static constexpr int kPart = kBlockSize * kPuD;                 // 2048: K (or V) codes of one granule
+  static constexpr int kGran = 2 * kPart + kFp8Header;
+  static constexpr int kKArea = kPuTileBlocks * kPart;            // 16 KB
+  static constexpr int kHdrOff = 2 * kKArea;
+  static constexpr int kStageBytes = kHdrOff + kPuTileBlocks * kFp8Header;   // 33,024
+  static constexpr int kOperand = 128 * 128;                      // one 128 x 128 operand of codes
+  static constexpr int kRingOff = 0;
+  static constexpr int kQOff = kRingOff + kPuStages * kStageBytes;   // Q: lead term, remainder term
+  static constexpr int kPOff = kQOff + 2 * kOperand;                 // P: [team][term], three terms (12 bits) per probability
+  static constexpr int kPTerms = 3;
+  static constexpr int kBarOff = kPOff + 2 * kPTerms * kOperand;
+  static constexpr int kNumBars = 3 * kPuStages + 2 + 2 + 2;         // full, empty, kfree, sfull, sfree, pfull
+  static constexpr int kMiscOff = kBarOff + kNumBars * 8;
+  static constexpr int kSmemBytes = kMiscOff + 64;
+  static_assert(kStageBytes % 128 == 0 && kSmemBytes <= 232448, "shared memory of one CTA");
+};
+
+__global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const PrefillUmmaParams p, const __grid_constant__ CUtensorMap map_part,
+                                                                          const __grid_constant__ CUtensorMap map_hdr) {
+  using C = PuCfg;
+  constexpr int D = kPuD;
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint8_t* ring = smem + C::kRingOff;
+  uint8_t* qbuf = smem + C::kQOff;
+  uint8_t* pbuf = smem + C::kPOff;
+  // float [2 teams][128] maxima and [2 teams][128] sums share the probability operands' memory: the maxima are
+  // exchanged before the first probability is written, the sums after the last P V instruction has finished
+  float* xch = reinterpret_cast<float*>(smem + C::kPOff);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
+  uint64_t* bar_full = bars;                         // [kPuStages] copies of a tile landed
+  uint64_t* bar_empty = bar_full + kPuStages;        // [kPuStages] second walk: the P V instructions of the tile are done
+  uint64_t* bar_kfree = bar_empty + kPuStages;       // [kPuStages] first walk: the tile's team has read its logits and scales
+  uint64_t* bar_sfull = bar_kfree + kPuStages;       // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
+  uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's four warps have read them (and the tile's scales)
+  uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's probabilities of a tile are in shared memory
+  int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory, [4..5] V scale maxima
+  volatile int* abort_flag = misc + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 3);
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int G = p.group, Hq = p.num_q_heads, Hkv = p.num_kv_heads;
+  const int g = blockIdx.y;
+  const int TQ = p.tile_queries;
+
+  // ---- which (sequence, query tile) is this CTA's ----------------------------------------------
+  if (tid == 0) {
+    int left = blockIdx.x, found = -1, q0 = 0;
+    for (int b = 0; b < p.batch; ++b) {
+      const int n = max(0, p.cu_q_lens[b + 1] - p.cu_q_lens[b]);
+      const int nt = (n + TQ - 1) / TQ;
+      if (left < nt) { found = b; q0 = (nt - 1 - left) * TQ; break; }   // late (long) tiles first
+      left -= nt;
+    }
+    misc[0] = found;
+    misc[1] = q0;
+    *abort_flag = 0;
+    for (int i = 0; i < kPuStages; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 1); mbar_init(&bar_kfree[i], 4); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 4); mbar_init(&bar_pfull[i], kPuTeam); }
+    mbar_fence_init();
+  }
+  if (tid == kPuProducer * 32) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_part) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hdr) : "memory");
+  }
+  __syncthreads();
+  const int b = misc[0];
+  if (b < 0) return;                                 // uniform over the CTA: nothing has been allocated yet
+  const int q0 = misc[1];
+  const int row_base = p.cu_q_lens[b];
+  const int n_new = p.cu_q_lens[b + 1] - row_base;
+  const int nq = min(TQ, n_new - q0);
+  const int L = max(0, min(p.context_lens[b], p.max_blocks_per_seq * kBlockSize));
+  // last position any row of the tile may see (Eq. 1: K_{<=t})
+  const int kv_end = p.causal ? max(0, min(L, L - n_new + q0 + nq)) : L;
+  const int n_tiles = (kv_end + kPuTileKeys - 1) / kPuTileKeys;
+  const int n_blocks = (kv_end + kBlockSize - 1) / kBlockSize;
+
+  // ---- this thread's row (softmax teams: thread r of either team owns row r) ---------------------
+  const int r = tid & (kPuTeam - 1);
+  const int qi = r / G;
+  const bool live = tid < kPuSm && qi < nq;
+  const size_t grow = static_cast<size_t>(row_base + q0 + (live ? qi : 0)) * Hq + g * G + (live ? r % G : 0);
+  // index of the last visible key of the row; -1 hides everything
+  const int lim = live ? (p.causal ? min(L - 1, L - n_new + q0 + qi) : L - 1) : -1;
+
+  if (n_tiles == 0) {
+    // nothing visible: all-zero rows
+    if (tid < kPuTeam && live)
+      for (int d = 0; d < D; d += 8) *reinterpret_cast<uint4*>(p.out + grow * D + d) = make_uint4(0u, 0u, 0u, 0u);
+    return;
+  }
+
+  // ---- set-up: tensor memory, the query operand ---------------------------------------
+  if (warp == kPuSWarp) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  // Row r of the query operand: the bf16 row scaled by a power of two into [128, 256) (undone on the
+  // logits) is the exact sum of its nearest E4M3 value and the E4M3 value of the remainder.  Element
+  // (row, byte k) of an operand sits at (row / 8) * 1024 + (k / 16) * 128 + (row % 8) * 16 + k % 16.
+  float qscale = 0.0f;       // logits of this row = tensor-memory value * qscale * K scale of the block
+  if (tid < kPuTeam) {
+    uint4 raw[D / 8];
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) raw[c] = live ? *reinterpret_cast<const uint4*>(p.q + grow * D + c * 8) : make_uint4(0u, 0u, 0u, 0u);
+    uint32_t amax = 0;
+#pragma unroll
+    for (int c = 0; c < D / 8; ++c) {
+      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) amax = max(amax, max((w[e] << 16) & 0x7FFFFFFFu, w[e] & 0x7FFF0000u));   // |bf16| as fp32 bits
+    }
+    int k2 = 0;
+    if (amax != 0u) k2 = max(-64, min(64, 134 - static_cast<int>((amax >> 23) & 0xFF)));
+    const float up = __uint_as_float(static_cast<uint32_t>(k2 + 127) << 23);
+    qscale = p.sm_scale_log2 * __uint_as_float(static_cast<uint32_t>(127 - k2) << 23);
+    uint8_t* qrow = qbuf + (r >> 3) * 1024 + (r & 7) * 16;
+#pragma unroll
+    for (int c = 0; c < D / 16; ++c) {            // 16 elements = one 16-byte chunk of each term
+      uint32_t lead[4], rest[4];
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {               // four elements = two packed pairs
+        const uint4 v = raw[2 * c + (e >> 1)];
+        const uint32_t w0 = (e & 1) ? v.z : v.x, w1 = (e & 1) ? v.w : v.y;
+        uint32_t h0 = pack_f16x2(__uint_as_float(w0 << 16) * up, __uint_as_float(w0 & 0xFFFF0000u) * up);
+        uint32_t h1 = pack_f16x2(__uint_as_float(w1 << 16) * up, __uint_as_float(w1 & 0xFFFF0000u) * up);
+        const uint32_t l0 = e4m3_term(h0, 1.0f), l1 = e4m3_term(h1, 1.0f);
+        lead[e] = l0 | (l1 << 16);
+        rest[e] = f16x2_to_e4m3x2(h0) | (f16x2_to_e4m3x2(h1) << 16);
+      }
+      *reinterpret_cast<uint4*>(qrow + c * 128) = make_uint4(lead[0], lead[1], lead[2], lead[3]);
+      *reinterpret_cast<uint4*>(qrow + C::kOperand + c * 128) = make_uint4(rest[0], rest[1], rest[2], rest[3]);
+    }
+  }
+  if (tid >= kPuTeam && tid < kPuSm) {
+    // team 1 shares team 0's operand; it only needs the row's scale
+    uint32_t amax = 0;
+    if (live) {
+#pragma unroll
+      for (int c = 0; c < D / 8; ++c) {
+        const uint4 v = *reinterpret_cast<const uint4*>(p.q + grow * D + c * 8);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) amax = max(amax, max((w[e] << 16) & 0x7FFFFFFFu, w[e] & 0x7FFF0000u));
+      }
+    }
+    int k2 = 0;
+    if (amax != 0u) k2 = max(-64, min(64, 134 - static_cast<int>((amax >> 23) & 0xFF)));
+    qscale = p.sm_scale_log2 * __uint_as_float(static_cast<uint32_t>(127 - k2) << 23);
+  }
+  fence_proxy_async();
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t tmem_o = tmem + 256;                 // logits buffer b at column 128 b, output at 256
+  const uint32_t lane_base = static_cast<uint32_t>(warp & 3) * 32u << 16;
+  const int total = 2 * n_tiles;                      // tiles of both walks, numbered in order of use
+
+  if (warp == kPuProducer) {
+    // ================= copies: first walk K parts and headers, second walk V parts as well ================
+    // Lane 3 q + w (q = 0, 1; w = 0, 1, 2) fetches the K parts (w = 0), the V parts (w = 1) or the headers
+    // (w = 2) of granules 4 q .. 4 q + 3 of the tile.  Rows past the last block repeat the tile's first one.
+    bool ok = true;
+    const int q4 = lane / 3, what = lane - 3 * q4;
+    const int x = what * (C::kPart / 8);
+    const uint32_t dst_off = what == 0 ? q4 * 4 * C::kPart : what == 1 ? C::kKArea + q4 * 4 * C::kPart : C::kHdrOff + q4 * 4 * kFp8Header;
+    const CUtensorMap* map = what == 2 ? &map_hdr : &map_part;
+    // the physical blocks of a tile are looked up one tile ahead of their use (range-checked: a bad id is
+    // reported in the status word and replaced by block 0, never dereferenced)
+    const int* trow = p.block_table + static_cast<size_t>(b) * p.max_blocks_per_seq;
+    auto lookup = [&](int T, int (&rows)[4]) {
+      const int t = T >= n_tiles ? T - n_tiles : T;
+      const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        rows[i] = 0;
+        if (lane < 6 && T < total) {
+          const int j = q4 * 4 + i;
+          int id = trow[t * kPuTileBlocks + (j < nb ? j : 0)];
+          if (id < 0 || id >= p.num_blocks) { atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG); id = 0; }
+          rows[i] = id * Hkv + g;
+        }
+      }
+    };
+    int rows[4], rows_next[4];
+    lookup(0, rows_next);
+    for (int T = 0; T < total; ++T) {
+      const bool second = T >= n_tiles;
+      const int t = second ? T - n_tiles : T;
+      const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
+      const int ngroups = (nb + 3) / 4;
+#pragma unroll
+      for (int i = 0; i < 4; ++i) rows[i] = rows_next[i];
+      lookup(T + 1, rows_next);
+      const uint32_t stage = T % kPuStages;
+      uint8_t* st = ring + stage * C::kStageBytes;
+      if (lane == 0) {
+        if (T >= kPuStages) {
+          // who used the stage before: a tile of the first walk frees it when its team has read the logits
+          // and the scales, a tile of the second walk when its P V instructions are done.  Both signals are
+          // per stage: their next phase cannot complete before this refill, so the parity waited for is never
+          // overtaken (a per-buffer signal can be, once the teams have drained the whole ring).
+          const int U = T - kPuStages;
+          if (U < n_tiles) ok = wait_bar(&bar_kfree[stage], (U / kPuStages) & 1u, abort_flag);
+          else {
+            // second-walk uses of this stage so far (tiles U' < T, U' >= n_tiles, U' % kPuStages == stage): U is the latest
+            const int first = n_tiles + ((static_cast<int>(stage) - n_tiles % kPuStages) + kPuStages) % kPuStages;
+            const int use = (U - first) / kPuStages;
+            ok = wait_bar(&bar_empty[stage], use & 1u, abort_flag);
+          }
+        }
+        if (ok) mbar_expect_tx(&bar_full[stage], ngroups * 4 * ((second ? 2 : 1) * C::kPart + kFp8Header));
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane < 3 * ngroups && (second || what != 1)) gather4_g2s(st + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[stage]);
+    }
+    if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+  } else if (warp == kPuSWarp) {
+    // ================= logits: S = Q . Ktile^T, both terms of Q (one lane) ====================================
+    if (lane == 0) {
+      bool ok = true;
+      const uint64_t desc_k = umma_desc(smem_u32(ring), 128, 8 * D), desc_q = umma_desc(smem_u32(qbuf), 128, 1024);
+      for (int T = 0; T < total && ok; ++T) {
+        const uint32_t stage = T % kPuStages, buf = T & 1u, use = T >> 1;
+        ok = wait_bar(&bar_full[stage], (T / kPuStages) & 1u, abort_flag);
+        if (ok && use > 0) ok = wait_bar(&bar_sfree[buf], (use - 1) & 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint64_t dk = desc_k + ((stage * C::kStageBytes) >> 4);
+#pragma unroll
+        for (int term = 0; term < 2; ++term)
+#pragma unroll
+          for (int ks = 0; ks < D / 32; ++ks)
+            umma_f8(tmem + 128 * buf, desc_q + ((term * C::kOperand) >> 4) + ks * 16, dk + ks * 16, umma_idesc(128), (term | ks) != 0);
+        umma_commit(&bar_sfull[buf]);
+      }
+      if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+    }
+  } else if (warp == kPuPvWarp) {
+    // ================= outputs: O += P . Vtile, both terms of P (one lane) ===================================
+    if (lane == 0) {
+      bool ok = true;
+      const uint64_t desc_v = umma_desc(smem_u32(ring + C::kKArea), C::kPart, 128), desc_p = umma_desc(smem_u32(pbuf), 128, 1024);
+      for (int T = n_tiles; T < total && ok; ++T) {
+        const int t = T - n_tiles;
+        const uint32_t stage = T % kPuStages, team = T & 1u;
+        // the team's tiles of the second walk so far
+        const int first = n_tiles + ((static_cast<int>(team) - n_tiles % 2) + 2) % 2;
+        const uint32_t use = (T - first) >> 1;
+        ok = wait_bar(&bar_pfull[team], use & 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
+        const int nks = (nb + 1) >> 1;                // 32 keys (two granules) per instruction
+        const uint64_t dv = desc_v + ((stage * C::kStageBytes) >> 4), dp = desc_p + ((team * C::kPTerms * C::kOperand) >> 4);
+#pragma unroll
+        for (int term = 0; term < C::kPTerms; ++term)
+          for (int ks = 0; ks < nks; ++ks)
+            umma_f8(tmem_o, dp + ((term * C::kOperand) >> 4) + ks * 16, dv + ks * ((2 * C::kPart) >> 4), umma_idesc(D), (t | term | ks) != 0);
+        umma_commit(&bar_empty[stage]);     // the stage and the team's probability operand are free again
+      }
+      if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+    }
+  } else {
+    // ================= softmax teams ================================================================================
+    const int team = warp >> 2;
+    bool bad = false;
+    float m_row = -INFINITY, l_row = 0.0f, v_max = 0.0f;
+    uint8_t* prow = pbuf + team * C::kPTerms * C::kOperand + (r >> 3) * 1024 + (r & 7) * 16;
+
+    // ---- first walk: the row's maximum logit, and the largest V scale ------------------------------------
+    for (int T = team; T < n_tiles; T += 2) {
+      const uint32_t stage = T % kPuStages, buf = T & 1u;
+      const uint8_t* st = ring + stage * C::kStageBytes;
+      bool ok = !bad && wait_bar(&bar_full[stage], (T / kPuStages) & 1u, abort_flag);
+      ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      bad = bad || !ok;
+      if (bad) break;
+      tc_fence_after();
+      const int key0 = T * kPuTileKeys;
+      const int nkeys = min(kPuTileKeys, kv_end - key0);
+#pragma unroll 2
+      for (int c = 0; c < kPuTileBlocks; ++c) {
+        if (c * kBlockSize >= nkeys) break;                       // uniform over the CTA
+        uint32_t s[16];
+        tmem_ld16_issue(tmem + 128 * buf + 16 * c + lane_base, s);
+        const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + c * kFp8Header);
+        const float sk = hdr[0] * qscale;
+        v_max = fmaxf(v_max, hdr[1]);
+        const int visible = lim - (key0 + c * kBlockSize);         // keys 0 .. visible of this block are seen by the row
+        tmem_ld_wait(s);
+#pragma unroll
+        for (int j = 0; j < 16; ++j)
+          if (j <= visible) m_row = fmaxf(m_row, __uint_as_float(s[j]) * sk);
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&bar_sfree[buf]); mbar_arrive(&bar_kfree[stage]); }
+    }
+    // both teams' maxima (row r of either team is the same row)
+    xch[team * 128 + r] = m_row;
+    if (r == 0) reinterpret_cast<float*>(misc + 4)[team] = v_max;
+    bad = barrier_or(1, kPuSm, bad);
+    if (!bad) {
+      m_row = fmaxf(xch[r], xch[128 + r]);
+      const float* vm = reinterpret_cast<const float*>(misc + 4);
+      v_max = fmaxf(vm[0], vm[1]);
+    }
+    bad = barrier_or(1, kPuSm, bad);          // everybody has read the maxima: their memory may take probabilities
+    const float m_use = m_row == -INFINITY ? 0.0f : m_row;
+    const float v_inv = v_max > 0.0f ? kPuGain / v_max : 0.0f;
+
+    // ---- second walk: probabilities against the final maximum, two E4M3 terms each -----------------------
+    int mine = 0;                                                  // this team's tiles of the second walk so far
+    for (int T = n_tiles + ((team - n_tiles % 2) + 2) % 2; T < total && !bad; T += 2, ++mine) {
+      const int t = T - n_tiles;
+      const uint32_t stage = T % kPuStages, buf = T & 1u;
+      uint8_t* st = ring + stage * C::kStageBytes;
+      bool ok = wait_bar(&bar_full[stage], (T / kPuStages) & 1u, abort_flag);
+      ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
+      // the team's previous tile must have left the probability operand
+      if (ok && mine > 0) {
+        const int Tp = T - 2;
+        const uint32_t sp = Tp % kPuStages;
+        const int first = n_tiles + ((static_cast<int>(sp) - n_tiles % kPuStages) + kPuStages) % kPuStages;
+        ok = wait_bar(&bar_empty[sp], ((Tp - first) / kPuStages) & 1u, abort_flag);
+      }
+      ok = __all_sync(0xffffffffu, ok);
+      bad = bad || !ok;
+      if (bad) break;
+      tc_fence_after();
+      const int key0 = t * kPuTileKeys;
+      const int nkeys = min(kPuTileKeys, kv_end - key0);
+      const int nb = (nkeys + kBlockSize - 1) / kBlockSize;
+#pragma unroll 2
+      for (int c = 0; c < kPuTileBlocks; ++c) {
+        uint4 lead4 = make_uint4(0u, 0u, 0u, 0u), rest4 = make_uint4(0u, 0u, 0u, 0u), last4 = make_uint4(0u, 0u, 0u, 0u);
+        if (c < nb) {
+          uint32_t s[16];
+          tmem_ld16_issue(tmem + 128 * buf + 16 * c + lane_base, s);
+          const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + c * kFp8Header);
+          const float sk = hdr[0] * qscale;
+          const float pv = hdr[1] * v_inv;
+          const int visible = lim - (key0 + c * kBlockSize);
+          tmem_ld_wait(s);
+          uint32_t lw[4], rw[4], tw[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            float pe[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const float x = ex2(__uint_as_float(s[4 * e + j]) * sk - m_use);
+              pe[j] = (4 * e + j <= visible) ? x : 0.0f;
+              l_row += pe[j];
+            }
+            uint32_t h0 = pack_f16x2(pe[0] * pv, pe[1] * pv), h1 = pack_f16x2(pe[2] * pv, pe[3] * pv);
+            // each term is the E4M3 value nearest to what the earlier ones left over (the differences are exact)
+            const uint32_t l0 = e4m3_term(h0, 1.0f), l1 = e4m3_term(h1, 1.0f);
+            const uint32_t r0 = e4m3_term(h0, 1.0f), r1 = e4m3_term(h1, 1.0f);
+            lw[e] = l0 | (l1 << 16);
+            rw[e] = r0 | (r1 << 16);
+            tw[e] = f16x2_to_e4m3x2(h0) | (f16x2_to_e4m3x2(h1) << 16);
+          }
+          lead4 = make_uint4(lw[0], lw[1], lw[2], lw[3]);
+          rest4 = make_uint4(rw[0], rw[1], rw[2], rw[3]);
+          last4 = make_uint4(tw[0], tw[1], tw[2], tw[3]);
+        }
+        if (c < 2 * ((nb + 1) >> 1)) {                 // what the P V instructions of this tile read
+          *reinterpret_cast<uint4*>(prow + c * 128) = lead4;
+          *reinterpret_cast<uint4*>(prow + C::kOperand + c * 128) = rest4;
+          *reinterpret_cast<uint4*>(prow + 2 * C::kOperand + c * 128) = last4;
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_sfree[buf]);
+      // V codes of slots past the context inside the last block are cleared (row r = dim r of V^T), and
+      // so is the slot behind an odd number of blocks, which the last instruction also reads
+      if ((nkeys & 15) != 0) {
+        uint4* row = reinterpret_cast<uint4*>(st + C::kKArea + (nkeys >> 4) * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
+        const int keep = nkeys & 15;
+        uint4 w = *row;
+        uint32_t* ww = reinterpret_cast<uint32_t*>(&w);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int left = keep - 4 * j;
+          ww[j] &= left >= 4 ? 0xFFFFFFFFu : (left <= 0 ? 0u : (1u << (8 * left)) - 1u);
+        }
+        *row = w;
+      }
+      if ((nb & 1) != 0)
+        *reinterpret_cast<uint4*>(st + C::kKArea + nb * C::kPart + (r >> 3) * 128 + (r & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+      fence_proxy_async();
+      mbar_arrive(&bar_pfull[team]);
+    }
+
+    // ---- the last P V instruction has finished: normalise and store ---------------------------------------
+    if (!bad) {
+      const int Tl = total - 1;
+      const uint32_t sl = Tl % kPuStages;
+      const int first = n_tiles + ((static_cast<int>(sl) - n_tiles % kPuStages) + kPuStages) % kPuStages;
+      bool ok = wait_bar(&bar_empty[sl], ((Tl - first) / kPuStages) & 1u, abort_flag);
+      ok = __all_sync(0xffffffffu, ok);
+      bad = !ok;
+    }
+    xch[256 + team * 128 + r] = l_row;
+    bad = barrier_or(1, kPuSm, bad);
+    if (!bad) {
+      tc_fence_after();
+      const float l_all = xch[256 + r] + xch[384 + r];
+      const float k = l_all > 0.0f ? v_max / (kPuGain * l_all) : 0.0f;
+      // team 0 stores dims 0..63 of the row, team 1 dims 64..127
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[16];
+        tmem_ld16_issue(tmem_o + team * 64 + 16 * c + lane_base, o);
+        tmem_ld_wait(o);
+        if (live) {
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) w[j] = pack_bf16x2(__uint_as_float(o[2 * j]) * k, __uint_as_float(o[2 * j + 1]) * k);
+          uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + team * 64 + 16 * c);
+          dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+      tc_fence_before();
+    }
+    if (bad && r == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+  }
+
+  // ---- exit: copies still in flight get a bounded time to land, tensor memory is returned -----------
+  __syncthreads();
+  if (*abort_flag != 0 && warp == kPuProducer && lane == 0) {
+    for (int s = 0; s < kPuStages && s < total; ++s) {
+      const int last = total - 1 - s;
+      mbar_wait_bounded(&bar_full[last % kPuStages], (last / kPuStages) & 1u);
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == kPuSWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512) : "memory");
+}
+
+}  // namespace
+
+int launch_paged_prefill_umma(const coopt_cache* c, const void* q, void* out, const int32_t* cu_q_lens, const int32_t* block_table,
+                              int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                              int32_t total_q, int32_t causal, float sm_scale, void* workspace, cudaStream_t stream) {
+  PrefillUmmaParams p;
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.cu_q_lens = cu_q_lens;
+  p.block_table = block_table;
+  p.context_lens = context_lens;
+  p.max_blocks_per_seq = max_blocks_per_seq;
+  p.batch = batch;
+  p.num_q_heads = num_q_heads;
+  p.num_kv_heads = c->num_kv_heads;
+  p.group = num_q_heads / c->num_kv_heads;
+  p.num_blocks = c->num_blocks;
+  p.tile_queries = 128 / p.group;
+  p.causal = causal;
+  p.sm_scale_log2 = sm_scale * kPuLog2e;
+  p.status = static_cast<int*>(workspace);
+  const long long tiles = static_cast<long long>(total_q) / p.tile_queries + batch;   // every sequence adds at most one partly filled tile
+  if (tiles > 0x7fffffffll) return COOPT_ERR_UNSUPPORTED;
+  CUtensorMap map_part, map_hdr;
+  const long long granules = static_cast<long long>(c->num_blocks) * c->num_kv_heads;
+  if (!encode_cache_map(&map_part, c->data, granules, PuCfg::kGran, PuCfg::kPart / 8) ||
+      !encode_cache_map(&map_hdr, c->data, granules, PuCfg::kGran, kFp8Header / 8))
+    return COOPT_ERR_CUDA;
+  static bool configured[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
+  if (dev < 64 && !configured[dev]) {
+    if (cudaFuncSetAttribute(paged_prefill_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PuCfg::kSmemBytes) != cudaSuccess)
+      return COOPT_ERR_CUDA;
+    configured[dev] = true;
+  }
+  const dim3 grid(static_cast<unsigned>(tiles), static_cast<unsigned>(c->num_kv_heads));
+  paged_prefill_umma_kernel<<<grid, kPuThreads, PuCfg::kSmemBytes, stream>>>(p, map_part, map_hdr);
+  return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
+}
+
+}  // namespace coopt

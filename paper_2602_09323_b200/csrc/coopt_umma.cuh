@@ -1,0 +1,135 @@
+// What the kernels built on the 5th-generation tensor cores share: descriptors and wrappers of the
+// tcgen05 instructions, the gather form of the tensor copy, bounded waits, the E4M3 term split, and
+// the host-side encoding of the cache as a tensor map.
+#pragma once
+
+#include <cuda.h>
+
+#include "coopt_common.cuh"
+
+namespace coopt {
+
+#ifdef __CUDACC__
+
+// ---- tcgen05 wrappers ----------------------------------------------------------------------------
+// Shared-memory operand descriptor, K-major, no swizzle: element (row r, byte k) of the operand sits
+// at (r / 8) * sbo + (k / 16) * lbo + (r % 8) * 16 + k % 16 from the start address.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint32_t sbo) {
+  return static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>(lbo >> 4) << 16) |
+         (static_cast<uint64_t>(sbo >> 4) << 32) | (1ull << 46);
+}
+// Instruction descriptor: E4M3 x E4M3 -> fp32, both operands K-major, M = 128, N = n.
+__device__ __forceinline__ constexpr uint32_t umma_idesc(int n) {
+  return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
+}
+__device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"
+               ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// One commit per group of instructions: a second commit with no instruction in between was seen to
+// arrive before the group had finished, so every consumer of a group waits on the same mbarrier.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// 16 consecutive fp32 columns of this thread's tensor-memory lane; tmem_ld_wait() before the values are used.
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+                 "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr));
+}
+// The registers are named as operands so that no use of them can be scheduled ahead of the wait.
+__device__ __forceinline__ void tmem_ld_wait(uint32_t (&r)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]), "+r"(r[8]),
+                 "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+               :: "memory");
+}
+
+// One request: columns [x, x + box width) (in 8-byte elements) of the four rows r0..r3 of the 2-D tensor,
+// landing as four consecutive box rows in shared memory; completes on the mbarrier with its byte count.
+__device__ __forceinline__ void gather4_g2s(void* dst, const CUtensorMap* map, int x, int r0, int r1, int r2, int r3, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cta.global.tile::gather4.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+               ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(r0), "r"(r1), "r"(r2), "r"(r3), "r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Named barrier `id` over `count` threads, carrying an OR reduction of a per-thread flag.
+__device__ __forceinline__ bool barrier_or(int id, int count, bool flag) {
+  uint32_t r;
+  asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %3, 0;\n barrier.cta.red.or.pred q, %1, %2, p;\n selp.u32 %0, 1, 0, q;\n}"
+               : "=r"(r) : "r"(id), "r"(count), "r"(static_cast<uint32_t>(flag)) : "memory");
+  return r != 0;
+}
+// Bounded wait that also gives up when another role has already given up.  try_wait lets the hardware
+// park the warp, so waiting warps do not take issue slots from the two single-lane roles that share
+// their schedulers.  The clock and the abort flag are looked at once in 256 unsuccessful tries.
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  uint64_t t0 = 0;
+#pragma unroll 1
+  for (uint32_t tries = 1;; ++tries) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((tries & 0xFFu) == 0) {
+      if (*abort_flag != 0) return false;
+      const uint64_t now = global_timer_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+    }
+  }
+}
+
+// Order-preserving map float <-> int, so that one redux.sync gives a warp-wide float maximum.
+__device__ __forceinline__ int f32_to_ordered(float x) {
+  const int i = __float_as_int(x);
+  return i ^ ((i >> 31) & 0x7FFFFFFF);
+}
+__device__ __forceinline__ float ordered_to_f32(int i) { return __int_as_float(i ^ ((i >> 31) & 0x7FFFFFFF)); }
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+  return x;
+}
+// Two f16 values -> two E4M3 codes (low half in bits 0..7), round to nearest even, saturating.
+__device__ __forceinline__ uint32_t f16x2_to_e4m3x2(uint32_t h2) {
+  uint16_t d;
+  asm("cvt.rn.satfinite.e4m3x2.f16x2 %0, %1;" : "=h"(d) : "r"(h2));
+  return d;
+}
+// codes = e4m3(h2); h2 is replaced by (h2 - value(codes)) * gain.  The difference is exact in f16.
+__device__ __forceinline__ uint32_t e4m3_term(uint32_t& h2, float gain) {
+  const uint32_t codes = f16x2_to_e4m3x2(h2);
+  const uint32_t back = e4m3x2_to_f16x2_lo(codes);
+  const __half2 rest = __hmul2(__hsub2(*reinterpret_cast<const __half2*>(&h2), *reinterpret_cast<const __half2*>(&back)),
+                               __float2half2_rn(gain));
+  h2 = *reinterpret_cast<const uint32_t*>(&rest);
+  return codes;
+}
+
+#endif  // __CUDACC__
+
+// The cache as the copy engine sees it: [granules][granule bytes / 8] 8-byte elements, one box row of
+// `box_elems` elements per gathered granule.
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                      const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                      CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+inline bool encode_cache_map(CUtensorMap* map, const void* cache, long long granules, int gran_bytes, int box_elems) {
+  static TensorMapEncodeFn encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult res;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess || !fn) return false;
+    encode = reinterpret_cast<TensorMapEncodeFn>(fn);
+  }
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(gran_bytes / 8), static_cast<cuuint64_t>(granules)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(gran_bytes)};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_elems), 1}, elem_strides[2] = {1, 1};
+  return encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT64, 2, const_cast<void*>(cache), dims, strides, box, elem_strides,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace coopt
