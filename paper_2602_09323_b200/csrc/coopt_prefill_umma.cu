@@ -21,7 +21,9 @@
 //               row's 128 logits from tensor memory 16 at a time (one cache block: one pair of scales),
 //               so maxima and sums need no exchange between threads;
 //   warp 8      copies: gather requests over the tensor map of the cache (K parts, V parts, headers of
-//               four granules each) into a ring of three stages;
+//               four granules each) into six slots of 16 KB + 256 B.  The first walk uses all six for K
+//               tiles (and their scales); in the second walk two take K tiles, freed as soon as the logits
+//               are computed, and four take V tiles and the scales, held until the P V instructions are done;
 //   warp 9      one lane issues the S instructions; warp 10 one lane issues the P V instructions.
 // Every wait is bounded; a wait that runs out is reported in the status word and all roles leave through
 // the common exit, which frees the tensor memory.
@@ -38,7 +40,8 @@ constexpr int kPuThreads = 352;
 constexpr int kPuTileBlocks = 8;
 constexpr int kPuTileKeys = kPuTileBlocks * kBlockSize;   // 128
 constexpr int kPuD = 128;
-constexpr int kPuStages = 3;
+constexpr int kPuSlots = 6;                                // of the copy ring
+constexpr int kPuKSlots = 2, kPuVSlots = 4;               // second walk: slots 0-1 take K tiles, slots 2-5 V tiles and scales
 constexpr float kPuLog2e = 1.4426950408889634f;
 constexpr float kPuGain = 256.0f;                          // probabilities are carried times 2^8 (at most 256 < 448)
 
@@ -60,19 +63,19 @@ struct PrefillUmmaParams {
 struct PuCfg {
   static constexpr int kPart = kBlockSize * kPuD;                 // 2048: K (or V) codes of one granule
   static constexpr int kGran = 2 * kPart + kFp8Header;
-  static constexpr int kKArea = kPuTileBlocks * kPart;            // 16 KB
-  static constexpr int kHdrOff = 2 * kKArea;
-  static constexpr int kStageBytes = kHdrOff + kPuTileBlocks * kFp8Header;   // 33,024
+  static constexpr int kKArea = kPuTileBlocks * kPart;            // 16 KB: the K parts, or the V parts, of a tile
+  static constexpr int kHdrOff = kKArea;                          // behind them the eight headers (scales) of the tile
+  static constexpr int kSlot = kHdrOff + kPuTileBlocks * kFp8Header;   // 16,640
   static constexpr int kOperand = 128 * 128;                      // one 128 x 128 operand of codes
   static constexpr int kRingOff = 0;
-  static constexpr int kQOff = kRingOff + kPuStages * kStageBytes;   // Q: lead term, remainder term
+  static constexpr int kQOff = kRingOff + kPuSlots * kSlot;          // Q: lead term, remainder term
   static constexpr int kPOff = kQOff + 2 * kOperand;                 // P: [team][term], three terms (12 bits) per probability
   static constexpr int kPTerms = 3;
   static constexpr int kBarOff = kPOff + 2 * kPTerms * kOperand;
-  static constexpr int kNumBars = 3 * kPuStages + 2 + 2 + 2;         // full, empty, kfree, sfull, sfree, pfull
+  static constexpr int kNumBars = 2 * kPuSlots + kPuKSlots + kPuVSlots + 2 + 2 + 2;   // full, free1, kdone, vdone, sfull, sfree, pfull
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kSmemBytes = kMiscOff + 64;
-  static_assert(kStageBytes % 128 == 0 && kSmemBytes <= 232448, "shared memory of one CTA");
+  static_assert(kSlot % 128 == 0 && kSmemBytes <= 232448, "shared memory of one CTA");
 };
 
 __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const PrefillUmmaParams p, const __grid_constant__ CUtensorMap map_part,
@@ -87,10 +90,13 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   // exchanged before the first probability is written, the sums after the last P V instruction has finished
   float* xch = reinterpret_cast<float*>(smem + C::kPOff);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
-  uint64_t* bar_full = bars;                         // [kPuStages] copies of a tile landed
-  uint64_t* bar_empty = bar_full + kPuStages;        // [kPuStages] second walk: the P V instructions of the tile are done
-  uint64_t* bar_kfree = bar_empty + kPuStages;       // [kPuStages] first walk: the tile's team has read its logits and scales
-  uint64_t* bar_sfull = bar_kfree + kPuStages;       // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
+  // Every signal that frees a slot is per slot: its next phase cannot complete before the slot has been
+  // refilled, so the parity a waiter looks for is never overtaken.
+  uint64_t* bar_full = bars;                         // [kPuSlots] the copies into the slot have landed
+  uint64_t* bar_free1 = bar_full + kPuSlots;         // [kPuSlots] first walk: the tile's team has read its logits and scales
+  uint64_t* bar_kdone = bar_free1 + kPuSlots;        // [kPuKSlots] second walk: the logits of the K tile in the slot are computed
+  uint64_t* bar_vdone = bar_kdone + kPuKSlots;       // [kPuVSlots] second walk: the P V instructions of the V tile in the slot are done
+  uint64_t* bar_sfull = bar_vdone + kPuVSlots;       // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
   uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's four warps have read them (and the tile's scales)
   uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's probabilities of a tile are in shared memory
   int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory, [4..5] V scale maxima
@@ -114,7 +120,9 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     misc[0] = found;
     misc[1] = q0;
     *abort_flag = 0;
-    for (int i = 0; i < kPuStages; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 1); mbar_init(&bar_kfree[i], 4); }
+    for (int i = 0; i < kPuSlots; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_free1[i], 4); }
+    for (int i = 0; i < kPuKSlots; ++i) mbar_init(&bar_kdone[i], 1);
+    for (int i = 0; i < kPuVSlots; ++i) mbar_init(&bar_vdone[i], 1);
     for (int i = 0; i < 2; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 4); mbar_init(&bar_pfull[i], kPuTeam); }
     mbar_fence_init();
   }
@@ -216,6 +224,13 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   const uint32_t tmem_o = tmem + 256;                 // logits buffer b at column 128 b, output at 256
   const uint32_t lane_base = static_cast<uint32_t>(warp & 3) * 32u << 16;
   const int total = 2 * n_tiles;                      // tiles of both walks, numbered in order of use
+  // Slots and the phase of a slot's "landed" barrier.  First walk: tile T lands in slot T % 6 (its use
+  // T / 6 of that slot).  Second walk: the K parts of tile t land in slot t % 2 (use t / 2 after the slot's
+  // first-walk uses), its V parts and scales in slot 2 + t % 4 (use t / 4 after the first-walk uses).
+  auto uses1 = [&](int slot) { return n_tiles > slot ? (n_tiles - slot + kPuSlots - 1) / kPuSlots : 0; };
+  auto kslot_par = [&](int t) { return static_cast<uint32_t>(uses1(t % kPuKSlots) + t / kPuKSlots) & 1u; };
+  auto vslot_par = [&](int t) { return static_cast<uint32_t>(uses1(kPuKSlots + t % kPuVSlots) + t / kPuVSlots) & 1u; };
+  uint32_t pend_mask = 0, pend_par = 0;               // copy lane: the latest phase expected of every slot it has filled
 
   if (warp == kPuProducer) {
     // ================= copies: first walk K parts and headers, second walk V parts as well ================
@@ -224,57 +239,73 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     bool ok = true;
     const int q4 = lane / 3, what = lane - 3 * q4;
     const int x = what * (C::kPart / 8);
-    const uint32_t dst_off = what == 0 ? q4 * 4 * C::kPart : what == 1 ? C::kKArea + q4 * 4 * C::kPart : C::kHdrOff + q4 * 4 * kFp8Header;
+    const uint32_t dst_off = what == 2 ? C::kHdrOff + q4 * 4 * kFp8Header : q4 * 4 * C::kPart;       // inside the slot
     const CUtensorMap* map = what == 2 ? &map_hdr : &map_part;
-    // the physical blocks of a tile are looked up one tile ahead of their use (range-checked: a bad id is
-    // reported in the status word and replaced by block 0, never dereferenced)
+    // The physical blocks are looked up 32 at a time (four tiles, one per lane), a batch ahead of their use, so
+    // that the copy lane never waits for the block table (range-checked: a bad id is reported in the status
+    // word and replaced by block 0, never dereferenced).  Batches are numbered through both walks.
     const int* trow = p.block_table + static_cast<size_t>(b) * p.max_blocks_per_seq;
-    auto lookup = [&](int T, int (&rows)[4]) {
-      const int t = T >= n_tiles ? T - n_tiles : T;
-      const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        rows[i] = 0;
-        if (lane < 6 && T < total) {
-          const int j = q4 * 4 + i;
-          int id = trow[t * kPuTileBlocks + (j < nb ? j : 0)];
-          if (id < 0 || id >= p.num_blocks) { atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG); id = 0; }
-          rows[i] = id * Hkv + g;
-        }
-      }
+    const int nbatch = (n_tiles + 3) / 4;
+    auto load_batch = [&](int lb) -> int {
+      if (lb >= 2 * nbatch) return 0;
+      const int j = (lb >= nbatch ? lb - nbatch : lb) * 32 + lane;
+      int id = j < n_blocks ? trow[j] : 0;
+      if (id < 0 || id >= p.num_blocks) { atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG); id = 0; }
+      return id;
     };
-    int rows[4], rows_next[4];
-    lookup(0, rows_next);
+    int cur_lb = 0;
+    int ids_cur = load_batch(0), ids_next = load_batch(1);
     for (int T = 0; T < total; ++T) {
       const bool second = T >= n_tiles;
       const int t = second ? T - n_tiles : T;
       const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
       const int ngroups = (nb + 3) / 4;
+      const int lb = (second ? nbatch : 0) + (t >> 2);
+      if (lb != cur_lb) { ids_cur = ids_next; cur_lb = lb; ids_next = load_batch(lb + 1); }
+      int rows[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) rows[i] = rows_next[i];
-      lookup(T + 1, rows_next);
-      const uint32_t stage = T % kPuStages;
-      uint8_t* st = ring + stage * C::kStageBytes;
-      if (lane == 0) {
-        if (T >= kPuStages) {
-          // who used the stage before: a tile of the first walk frees it when its team has read the logits
-          // and the scales, a tile of the second walk when its P V instructions are done.  Both signals are
-          // per stage: their next phase cannot complete before this refill, so the parity waited for is never
-          // overtaken (a per-buffer signal can be, once the teams have drained the whole ring).
-          const int U = T - kPuStages;
-          if (U < n_tiles) ok = wait_bar(&bar_kfree[stage], (U / kPuStages) & 1u, abort_flag);
-          else {
-            // second-walk uses of this stage so far (tiles U' < T, U' >= n_tiles, U' % kPuStages == stage): U is the latest
-            const int first = n_tiles + ((static_cast<int>(stage) - n_tiles % kPuStages) + kPuStages) % kPuStages;
-            const int use = (U - first) / kPuStages;
-            ok = wait_bar(&bar_empty[stage], use & 1u, abort_flag);
+      for (int i = 0; i < 4; ++i) {
+        const int j = (q4 & 1) * 4 + i;                             // block of the tile (lanes past the six copy lanes fetch along)
+        rows[i] = __shfl_sync(0xffffffffu, ids_cur, (t & 3) * 8 + (j < nb ? j : 0)) * Hkv + g;
+      }
+      if (!second) {
+        const int slot = T % kPuSlots;
+        if (lane == 0) {
+          if (T >= kPuSlots) ok = wait_bar(&bar_free1[slot], static_cast<uint32_t>(T / kPuSlots - 1) & 1u, abort_flag);
+          if (ok) {
+            mbar_expect_tx(&bar_full[slot], ngroups * 4 * (C::kPart + kFp8Header));
+            pend_mask |= 1u << slot;
+            pend_par = (pend_par & ~(1u << slot)) | ((static_cast<uint32_t>(T / kPuSlots) & 1u) << slot);
           }
         }
-        if (ok) mbar_expect_tx(&bar_full[stage], ngroups * 4 * ((second ? 2 : 1) * C::kPart + kFp8Header));
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane < 3 * ngroups && what != 1)
+          gather4_g2s(ring + slot * C::kSlot + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[slot]);
+      } else {
+        const int ks = t % kPuKSlots, vq = t % kPuVSlots, vs = kPuKSlots + vq;
+        if (lane == 0) {
+          // who used the slots before: the second walk's tile two (K) or four (V) back, else the slot's last tile of the first walk
+          if (t >= kPuKSlots) ok = wait_bar(&bar_kdone[ks], static_cast<uint32_t>(t / kPuKSlots - 1) & 1u, abort_flag);
+          else if (uses1(ks) > 0) ok = wait_bar(&bar_free1[ks], static_cast<uint32_t>(uses1(ks) - 1) & 1u, abort_flag);
+          if (ok) {
+            if (t >= kPuVSlots) ok = wait_bar(&bar_vdone[vq], static_cast<uint32_t>(t / kPuVSlots - 1) & 1u, abort_flag);
+            else if (uses1(vs) > 0) ok = wait_bar(&bar_free1[vs], static_cast<uint32_t>(uses1(vs) - 1) & 1u, abort_flag);
+          }
+          if (ok) {
+            mbar_expect_tx(&bar_full[ks], ngroups * 4 * C::kPart);
+            mbar_expect_tx(&bar_full[vs], ngroups * 4 * (C::kPart + kFp8Header));
+            pend_mask |= (1u << ks) | (1u << vs);
+            pend_par = (pend_par & ~((1u << ks) | (1u << vs))) | (kslot_par(t) << ks) | (vslot_par(t) << vs);
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (!ok) break;
+        if (lane < 3 * ngroups) {
+          const int slot = what == 0 ? ks : vs;
+          gather4_g2s(ring + slot * C::kSlot + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[slot]);
+        }
       }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane < 3 * ngroups && (second || what != 1)) gather4_g2s(st + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[stage]);
     }
     if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
   } else if (warp == kPuSWarp) {
@@ -283,12 +314,15 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       bool ok = true;
       const uint64_t desc_k = umma_desc(smem_u32(ring), 128, 8 * D), desc_q = umma_desc(smem_u32(qbuf), 128, 1024);
       for (int T = 0; T < total && ok; ++T) {
-        const uint32_t stage = T % kPuStages, buf = T & 1u, use = T >> 1;
-        ok = wait_bar(&bar_full[stage], (T / kPuStages) & 1u, abort_flag);
+        const uint32_t buf = T & 1u, use = T >> 1;
+        const bool second = T >= n_tiles;
+        const int t = second ? T - n_tiles : T;
+        const uint32_t slot = second ? t % kPuKSlots : T % kPuSlots;
+        ok = wait_bar(&bar_full[slot], second ? kslot_par(t) : static_cast<uint32_t>(T / kPuSlots) & 1u, abort_flag);
         if (ok && use > 0) ok = wait_bar(&bar_sfree[buf], (use - 1) & 1u, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const uint64_t dk = desc_k + ((stage * C::kStageBytes) >> 4);
+        const uint64_t dk = desc_k + ((slot * C::kSlot) >> 4);
 #pragma unroll
         for (int term = 0; term < 2; ++term)
 #pragma unroll
@@ -302,10 +336,10 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     // ================= outputs: O += P . Vtile, both terms of P (one lane) ===================================
     if (lane == 0) {
       bool ok = true;
-      const uint64_t desc_v = umma_desc(smem_u32(ring + C::kKArea), C::kPart, 128), desc_p = umma_desc(smem_u32(pbuf), 128, 1024);
+      const uint64_t desc_v = umma_desc(smem_u32(ring), C::kPart, 128), desc_p = umma_desc(smem_u32(pbuf), 128, 1024);
       for (int T = n_tiles; T < total && ok; ++T) {
         const int t = T - n_tiles;
-        const uint32_t stage = T % kPuStages, team = T & 1u;
+        const uint32_t vq = t % kPuVSlots, team = T & 1u;
         // the team's tiles of the second walk so far
         const int first = n_tiles + ((static_cast<int>(team) - n_tiles % 2) + 2) % 2;
         const uint32_t use = (T - first) >> 1;
@@ -314,12 +348,12 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         tc_fence_after();
         const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
         const int nks = (nb + 1) >> 1;                // 32 keys (two granules) per instruction
-        const uint64_t dv = desc_v + ((stage * C::kStageBytes) >> 4), dp = desc_p + ((team * C::kPTerms * C::kOperand) >> 4);
+        const uint64_t dv = desc_v + (((kPuKSlots + vq) * C::kSlot) >> 4), dp = desc_p + ((team * C::kPTerms * C::kOperand) >> 4);
 #pragma unroll
         for (int term = 0; term < C::kPTerms; ++term)
           for (int ks = 0; ks < nks; ++ks)
             umma_f8(tmem_o, dp + ((term * C::kOperand) >> 4) + ks * 16, dv + ks * ((2 * C::kPart) >> 4), umma_idesc(D), (t | term | ks) != 0);
-        umma_commit(&bar_empty[stage]);     // the stage and the team's probability operand are free again
+        umma_commit(&bar_vdone[vq]);        // the V slot and the team's probability operand are free again
       }
       if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     }
@@ -332,9 +366,9 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
 
     // ---- first walk: the row's maximum logit, and the largest V scale ------------------------------------
     for (int T = team; T < n_tiles; T += 2) {
-      const uint32_t stage = T % kPuStages, buf = T & 1u;
-      const uint8_t* st = ring + stage * C::kStageBytes;
-      bool ok = !bad && wait_bar(&bar_full[stage], (T / kPuStages) & 1u, abort_flag);
+      const uint32_t slot = T % kPuSlots, buf = T & 1u;
+      const uint8_t* st = ring + slot * C::kSlot;
+      bool ok = !bad && wait_bar(&bar_full[slot], static_cast<uint32_t>(T / kPuSlots) & 1u, abort_flag);
       ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       bad = bad || !ok;
@@ -358,7 +392,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&bar_sfree[buf]); mbar_arrive(&bar_kfree[stage]); }
+      if (lane == 0) { mbar_arrive(&bar_sfree[buf]); mbar_arrive(&bar_free1[slot]); }
     }
     // both teams' maxima (row r of either team is the same row)
     xch[team * 128 + r] = m_row;
@@ -377,17 +411,14 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     int mine = 0;                                                  // this team's tiles of the second walk so far
     for (int T = n_tiles + ((team - n_tiles % 2) + 2) % 2; T < total && !bad; T += 2, ++mine) {
       const int t = T - n_tiles;
-      const uint32_t stage = T % kPuStages, buf = T & 1u;
-      uint8_t* st = ring + stage * C::kStageBytes;
-      bool ok = wait_bar(&bar_full[stage], (T / kPuStages) & 1u, abort_flag);
+      const uint32_t vq = t % kPuVSlots, buf = T & 1u;
+      uint8_t* st = ring + (kPuKSlots + vq) * C::kSlot;            // the tile's V parts, and behind them its scales
+      bool ok = wait_bar(&bar_full[kPuKSlots + vq], vslot_par(t), abort_flag);
       ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
+      // the logits are computed: the tile's K slot can be refilled
+      if (ok && (warp & 3) == 0 && lane == 0) mbar_arrive(&bar_kdone[t % kPuKSlots]);
       // the team's previous tile must have left the probability operand
-      if (ok && mine > 0) {
-        const int Tp = T - 2;
-        const uint32_t sp = Tp % kPuStages;
-        const int first = n_tiles + ((static_cast<int>(sp) - n_tiles % kPuStages) + kPuStages) % kPuStages;
-        ok = wait_bar(&bar_empty[sp], ((Tp - first) / kPuStages) & 1u, abort_flag);
-      }
+      if (ok && mine > 0) ok = wait_bar(&bar_vdone[(t - 2) % kPuVSlots], static_cast<uint32_t>((t - 2) / kPuVSlots) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       bad = bad || !ok;
       if (bad) break;
@@ -440,7 +471,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       // V codes of slots past the context inside the last block are cleared (row r = dim r of V^T), and
       // so is the slot behind an odd number of blocks, which the last instruction also reads
       if ((nkeys & 15) != 0) {
-        uint4* row = reinterpret_cast<uint4*>(st + C::kKArea + (nkeys >> 4) * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
+        uint4* row = reinterpret_cast<uint4*>(st + (nkeys >> 4) * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
         const int keep = nkeys & 15;
         uint4 w = *row;
         uint32_t* ww = reinterpret_cast<uint32_t*>(&w);
@@ -452,17 +483,15 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         *row = w;
       }
       if ((nb & 1) != 0)
-        *reinterpret_cast<uint4*>(st + C::kKArea + nb * C::kPart + (r >> 3) * 128 + (r & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+        *reinterpret_cast<uint4*>(st + nb * C::kPart + (r >> 3) * 128 + (r & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
       fence_proxy_async();
       mbar_arrive(&bar_pfull[team]);
     }
 
     // ---- the last P V instruction has finished: normalise and store ---------------------------------------
     if (!bad) {
-      const int Tl = total - 1;
-      const uint32_t sl = Tl % kPuStages;
-      const int first = n_tiles + ((static_cast<int>(sl) - n_tiles % kPuStages) + kPuStages) % kPuStages;
-      bool ok = wait_bar(&bar_empty[sl], ((Tl - first) / kPuStages) & 1u, abort_flag);
+      const int tl = n_tiles - 1;
+      bool ok = wait_bar(&bar_vdone[tl % kPuVSlots], static_cast<uint32_t>(tl / kPuVSlots) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       bad = !ok;
     }
@@ -495,10 +524,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   // ---- exit: copies still in flight get a bounded time to land, tensor memory is returned -----------
   __syncthreads();
   if (*abort_flag != 0 && warp == kPuProducer && lane == 0) {
-    for (int s = 0; s < kPuStages && s < total; ++s) {
-      const int last = total - 1 - s;
-      mbar_wait_bounded(&bar_full[last % kPuStages], (last / kPuStages) & 1u);
-    }
+    for (int slot = 0; slot < kPuSlots; ++slot)
+      if ((pend_mask >> slot) & 1u) mbar_wait_bounded(&bar_full[slot], (pend_par >> slot) & 1u);
   }
   tc_fence_before();
   __syncthreads();
