@@ -85,3 +85,38 @@ def test_chunked_prefill_full_size_sampled():
         for r in rows:
             ref[r, h] = part[r, h]
     helpers.check_attention(out, ref, what="chunked prefill full size")
+
+
+@pytest.mark.parametrize("hq,hkv", [(16, 2), (12, 2), (4, 4)])
+def test_group_sizes_up_to_eight_on_the_tensor_memory_kernel(hq, hkv):
+    """head_dim 128 with G = 8, 6 and 1: 16, 21 and 128 query tokens per 128-row tile, tiles that end in the
+    middle of a cache block, a sequence that is all new tokens and one with a single new token."""
+    lens = [513, 300, 129, 47, 1024]
+    q_lens = [200, 300, 1, 20, 33]
+    w = workloads.make_workload("prefill_g", lens, hq, hkv, 128, seed=3 * hq + hkv, q_lens=q_lens)
+    out = _gpu_prefill(w, helpers.gpu_fill(w))
+    helpers.check_attention(out, _oracle(w), what=f"prefill hq{hq} hkv{hkv}")
+
+
+def test_long_context_prefill_many_tiles_and_block_batches():
+    """A 40,000-token context (2,500 blocks, 313 tiles of 128 keys, 79 batches of block ids) behind 96 new
+    tokens: the copy ring wraps many times in both walks; sampled rows against the oracle."""
+    L, n = 40000, 96
+    w = workloads.make_workload("prefill_long", [L, 700], 10, 2, 128, seed=29, q_lens=[n, 50])
+    out = _gpu_prefill(w, helpers.gpu_fill(w))
+    assert torch.isfinite(out.float()).all()
+    pairs = [(r, h) for r in (0, 1, 50, n - 1, n, n + 49) for h in (0, 4, 5, 9)]
+    ref = _oracle(w, pairs=pairs)
+    helpers.check_attention(out, ref, what="long prefill")
+
+
+def test_prefill_twice_is_bitwise_identical_and_all_zero_v_blocks_are_handled():
+    """Blocks whose V values are all zero (scale 0) still take part in the softmax; two runs give the same bits."""
+    w = workloads.make_workload("prefill_zero_v", [400, 90], 10, 2, 128, seed=31, q_lens=[60, 90])
+    w.v[16:48] = 0                      # two whole blocks of the first sequence
+    w.v[400 + 32:400 + 48] = 0          # one block of the second
+    cache = helpers.gpu_fill(w)
+    out1 = _gpu_prefill(w, cache)
+    out2 = _gpu_prefill(w, cache)
+    assert torch.equal(out1, out2)
+    helpers.check_attention(out1, _oracle(w), what="prefill zero v")
