@@ -422,6 +422,7 @@ int launch_paged_prefill(const coopt_cache* c, const void* q, void* out, const i
                          int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t causal, float sm_scale,
                          void* workspace, cudaStream_t stream) {
   if (c->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;
+  if (num_q_heads / c->num_kv_heads > kPfRows) return COOPT_ERR_UNSUPPORTED;   // a tile holds at least one query token of every head of the group
   // head_dim 128: the tcgen05 kernel; head_dim 64: the mma.sync kernel of this file
   if (c->head_dim == 128)
     return launch_paged_prefill_umma(c, q, out, cu_q_lens, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads,
