@@ -577,15 +577,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         if (team == 0 && more) load_q(plan.segs[si + 1]);
 
         // the team's running softmax over its tiles of this segment
-        float m_run[kGMax], l_run[kGMax], o_reg[kGMax], a_prev[kGMax];
+        float m_run[kGMax], l_run[kGMax], o_reg[kGMax];
 #pragma unroll
-        for (int h = 0; h < kGMax; ++h) { m_run[h] = -INFINITY; l_run[h] = 0.0f; o_reg[h] = 0.0f; a_prev[h] = 0.0f; }
+        for (int h = 0; h < kGMax; ++h) { m_run[h] = -INFINITY; l_run[h] = 0.0f; o_reg[h] = 0.0f; }
         float vref = 0.0f;
         bool pending = false;       // a tile of this team whose P V product is not folded in yet
         bool q_due = team == 0 && more;   // the next segment's query is published behind this team's first tile
         uint32_t pend_tile = 0;
 
-        // O_tile -> registers: o = o * a + (term0 + term1 / 16 + term2 / 256)
+        // O_tile -> registers: o += term0 + term1 / 16 + term2 / 256 (o is kept on the scale of the tile being folded in)
         auto fold_issue = [&](uint32_t (&r)[NP]) {
           bool ok = !bad && wait_bar(&bar_empty[pend_tile % C::kStages], (pend_tile / C::kStages) & 1u, abort_flag);
           ok = __all_sync(0xffffffffu, ok);
@@ -605,7 +605,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           if (lane == 0) mbar_arrive(&bar_ofree[pend_tile & 3u]);
 #pragma unroll
           for (int h = 0; h < kGMax; ++h)
-            o_reg[h] = o_reg[h] * a_prev[h] + (__uint_as_float(r[h]) + __uint_as_float(r[kGMax + h]) * 0.0625f +
+            o_reg[h] += (__uint_as_float(r[h]) + __uint_as_float(r[kGMax + h]) * 0.0625f +
                                                __uint_as_float(r[2 * kGMax + h]) * 0.00390625f);
           pending = false;
         };
@@ -712,7 +712,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             fold_finish(o_raw);
           }
 #pragma unroll
-          for (int h = 0; h < kGMax; ++h) a_prev[h] = a_o[h];
+          for (int h = 0; h < kGMax; ++h) o_reg[h] *= a_o[h];      // what is folded in so far, on the scale of this tile's product
           pending = true;
           pend_tile = tile_no;
           if (q_due) { publish_q(seg_no + 1); q_due = false; }
@@ -742,7 +742,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         old_seg = seg_no;
         vref_old = vref;
 #pragma unroll
-        for (int h = 0; h < kGMax; ++h) o_old[h] = pending ? o_reg[h] * a_prev[h] : 0.0f;
+        for (int h = 0; h < kGMax; ++h) o_old[h] = pending ? o_reg[h] : 0.0f;
         ++seg_no;
       }
       if (old_open) flush_old();              // the round's last segment
