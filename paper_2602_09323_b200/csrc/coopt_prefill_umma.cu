@@ -16,15 +16,16 @@
 // rescaled.  The second product over K costs a third more tensor work and K traffic (out of L2), and
 // removes the read-modify-write of 128 x 128 accumulators whenever a maximum moves.
 //
-// Warp roles (352 threads):
-//   warps 0-3, 4-7   two softmax teams, even and odd tiles; thread r of a team owns row r: it reads the
-//               row's 128 logits from tensor memory 16 at a time (one cache block: one pair of scales),
-//               so maxima and sums need no exchange between threads;
-//   warp 8      copies: gather requests over the tensor map of the cache (K parts, V parts, headers of
+// Warp roles (608 threads):
+//   warps 0-7, 8-15  two softmax teams, even and odd tiles.  Two threads of a team share row r: warps 0-3 of
+//               the team take the tile's first four cache blocks, warps 4-7 the last four; a thread reads its
+//               row's logits from tensor memory 16 at a time (one cache block: one pair of scales), and
+//               maxima and sums are exchanged only at the end of a walk;
+//   warp 16     copies: gather requests over the tensor map of the cache (K parts, V parts, headers of
 //               four granules each) into six slots of 16 KB + 256 B.  The first walk uses all six for K
 //               tiles (and their scales); in the second walk two take K tiles, freed as soon as the logits
 //               are computed, and four take V tiles and the scales, held until the P V instructions are done;
-//   warp 9      one lane issues the S instructions; warp 10 one lane issues the P V instructions.
+//   warp 17     one lane issues the S instructions; warp 18 one lane issues the P V instructions.
 // Every wait is bounded; a wait that runs out is reported in the status word and all roles leave through
 // the common exit, which frees the tensor memory.
 #include "coopt_umma.cuh"
@@ -33,10 +34,11 @@ namespace coopt {
 
 namespace {
 
-constexpr int kPuTeam = 128;
-constexpr int kPuSm = 2 * kPuTeam;
-constexpr int kPuProducer = 8, kPuSWarp = 9, kPuPvWarp = 10;
-constexpr int kPuThreads = 352;
+constexpr int kPuRows = 128;                               // rows of a tile = threads of half a team
+constexpr int kPuTeam = 2 * kPuRows;                       // eight warps: four tensor-memory lane quarters x two halves of the columns
+constexpr int kPuSm = 2 * kPuTeam;                         // warps 0-15
+constexpr int kPuProducer = 16, kPuSWarp = 17, kPuPvWarp = 18;
+constexpr int kPuThreads = 608;
 constexpr int kPuTileBlocks = 8;
 constexpr int kPuTileKeys = kPuTileBlocks * kBlockSize;   // 128
 constexpr int kPuD = 128;
@@ -86,7 +88,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   uint8_t* ring = smem + C::kRingOff;
   uint8_t* qbuf = smem + C::kQOff;
   uint8_t* pbuf = smem + C::kPOff;
-  // float [2 teams][128] maxima and [2 teams][128] sums share the probability operands' memory: the maxima are
+  // float [4 parts of a row][128] maxima and [4][128] sums share the probability operands' memory: the maxima are
   // exchanged before the first probability is written, the sums after the last P V instruction has finished
   float* xch = reinterpret_cast<float*>(smem + C::kPOff);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
@@ -97,9 +99,9 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   uint64_t* bar_kdone = bar_free1 + kPuSlots;        // [kPuKSlots] second walk: the logits of the K tile in the slot are computed
   uint64_t* bar_vdone = bar_kdone + kPuKSlots;       // [kPuVSlots] second walk: the P V instructions of the V tile in the slot are done
   uint64_t* bar_sfull = bar_vdone + kPuVSlots;       // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
-  uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's four warps have read them (and the tile's scales)
+  uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's eight warps have read them (and the tile's scales)
   uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's probabilities of a tile are in shared memory
-  int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory, [4..5] V scale maxima
+  int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory, [4..7] V scale maxima
   volatile int* abort_flag = misc + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 3);
 
@@ -120,10 +122,10 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     misc[0] = found;
     misc[1] = q0;
     *abort_flag = 0;
-    for (int i = 0; i < kPuSlots; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_free1[i], 4); }
+    for (int i = 0; i < kPuSlots; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_free1[i], 8); }
     for (int i = 0; i < kPuKSlots; ++i) mbar_init(&bar_kdone[i], 1);
     for (int i = 0; i < kPuVSlots; ++i) mbar_init(&bar_vdone[i], 1);
-    for (int i = 0; i < 2; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 4); mbar_init(&bar_pfull[i], kPuTeam); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 8); mbar_init(&bar_pfull[i], kPuTeam); }
     mbar_fence_init();
   }
   if (tid == kPuProducer * 32) {
@@ -143,8 +145,9 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   const int n_tiles = (kv_end + kPuTileKeys - 1) / kPuTileKeys;
   const int n_blocks = (kv_end + kBlockSize - 1) / kBlockSize;
 
-  // ---- this thread's row (softmax teams: thread r of either team owns row r) ---------------------
-  const int r = tid & (kPuTeam - 1);
+  // ---- this thread's row (softmax teams: row r belongs to the two threads r and r + 128 of either team) ---
+  const int r = tid & (kPuRows - 1);
+  const int half = (tid >> 7) & 1;                    // which four cache blocks of a tile
   const int qi = r / G;
   const bool live = tid < kPuSm && qi < nq;
   const size_t grow = static_cast<size_t>(row_base + q0 + (live ? qi : 0)) * Hq + g * G + (live ? r % G : 0);
@@ -153,7 +156,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
 
   if (n_tiles == 0) {
     // nothing visible: all-zero rows
-    if (tid < kPuTeam && live)
+    if (tid < kPuRows && live)
       for (int d = 0; d < D; d += 8) *reinterpret_cast<uint4*>(p.out + grow * D + d) = make_uint4(0u, 0u, 0u, 0u);
     return;
   }
@@ -167,54 +170,44 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   // logits) is the exact sum of its nearest E4M3 value and the E4M3 value of the remainder.  Element
   // (row, byte k) of an operand sits at (row / 8) * 1024 + (k / 16) * 128 + (row % 8) * 16 + k % 16.
   float qscale = 0.0f;       // logits of this row = tensor-memory value * qscale * K scale of the block
-  if (tid < kPuTeam) {
-    uint4 raw[D / 8];
-#pragma unroll
-    for (int c = 0; c < D / 8; ++c) raw[c] = live ? *reinterpret_cast<const uint4*>(p.q + grow * D + c * 8) : make_uint4(0u, 0u, 0u, 0u);
-    uint32_t amax = 0;
-#pragma unroll
-    for (int c = 0; c < D / 8; ++c) {
-      const uint32_t w[4] = {raw[c].x, raw[c].y, raw[c].z, raw[c].w};
-#pragma unroll
-      for (int e = 0; e < 4; ++e) amax = max(amax, max((w[e] << 16) & 0x7FFFFFFFu, w[e] & 0x7FFF0000u));   // |bf16| as fp32 bits
-    }
-    int k2 = 0;
-    if (amax != 0u) k2 = max(-64, min(64, 134 - static_cast<int>((amax >> 23) & 0xFF)));
-    const float up = __uint_as_float(static_cast<uint32_t>(k2 + 127) << 23);
-    qscale = p.sm_scale_log2 * __uint_as_float(static_cast<uint32_t>(127 - k2) << 23);
-    uint8_t* qrow = qbuf + (r >> 3) * 1024 + (r & 7) * 16;
-#pragma unroll
-    for (int c = 0; c < D / 16; ++c) {            // 16 elements = one 16-byte chunk of each term
-      uint32_t lead[4], rest[4];
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {               // four elements = two packed pairs
-        const uint4 v = raw[2 * c + (e >> 1)];
-        const uint32_t w0 = (e & 1) ? v.z : v.x, w1 = (e & 1) ? v.w : v.y;
-        uint32_t h0 = pack_f16x2(__uint_as_float(w0 << 16) * up, __uint_as_float(w0 & 0xFFFF0000u) * up);
-        uint32_t h1 = pack_f16x2(__uint_as_float(w1 << 16) * up, __uint_as_float(w1 & 0xFFFF0000u) * up);
-        const uint32_t l0 = e4m3_term(h0, 1.0f), l1 = e4m3_term(h1, 1.0f);
-        lead[e] = l0 | (l1 << 16);
-        rest[e] = f16x2_to_e4m3x2(h0) | (f16x2_to_e4m3x2(h1) << 16);
-      }
-      *reinterpret_cast<uint4*>(qrow + c * 128) = make_uint4(lead[0], lead[1], lead[2], lead[3]);
-      *reinterpret_cast<uint4*>(qrow + C::kOperand + c * 128) = make_uint4(rest[0], rest[1], rest[2], rest[3]);
-    }
-  }
-  if (tid >= kPuTeam && tid < kPuSm) {
-    // team 1 shares team 0's operand; it only needs the row's scale
+  if (tid < kPuSm) {
+    // every thread of the teams needs its row's scale; threads 0..127 also build the operand
     uint32_t amax = 0;
     if (live) {
-#pragma unroll
+#pragma unroll 4
       for (int c = 0; c < D / 8; ++c) {
         const uint4 v = *reinterpret_cast<const uint4*>(p.q + grow * D + c * 8);
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int e = 0; e < 4; ++e) amax = max(amax, max((w[e] << 16) & 0x7FFFFFFFu, w[e] & 0x7FFF0000u));
+        for (int e = 0; e < 4; ++e) amax = max(amax, max((w[e] << 16) & 0x7FFFFFFFu, w[e] & 0x7FFF0000u));   // |bf16| as fp32 bits
       }
     }
     int k2 = 0;
     if (amax != 0u) k2 = max(-64, min(64, 134 - static_cast<int>((amax >> 23) & 0xFF)));
     qscale = p.sm_scale_log2 * __uint_as_float(static_cast<uint32_t>(127 - k2) << 23);
+    if (tid < kPuRows) {
+      const float up = __uint_as_float(static_cast<uint32_t>(k2 + 127) << 23);
+      uint8_t* qrow = qbuf + (r >> 3) * 1024 + (r & 7) * 16;
+#pragma unroll 2
+      for (int c = 0; c < D / 16; ++c) {            // 16 elements = one 16-byte chunk of each term
+        uint4 raw[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) raw[k] = live ? *reinterpret_cast<const uint4*>(p.q + grow * D + c * 16 + k * 8) : make_uint4(0u, 0u, 0u, 0u);
+        uint32_t lead[4], rest[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {               // four elements = two packed pairs
+          const uint4 v = raw[e >> 1];
+          const uint32_t w0 = (e & 1) ? v.z : v.x, w1 = (e & 1) ? v.w : v.y;
+          uint32_t h0 = pack_f16x2(__uint_as_float(w0 << 16) * up, __uint_as_float(w0 & 0xFFFF0000u) * up);
+          uint32_t h1 = pack_f16x2(__uint_as_float(w1 << 16) * up, __uint_as_float(w1 & 0xFFFF0000u) * up);
+          const uint32_t l0 = e4m3_term(h0, 1.0f), l1 = e4m3_term(h1, 1.0f);
+          lead[e] = l0 | (l1 << 16);
+          rest[e] = f16x2_to_e4m3x2(h0) | (f16x2_to_e4m3x2(h1) << 16);
+        }
+        *reinterpret_cast<uint4*>(qrow + c * 128) = make_uint4(lead[0], lead[1], lead[2], lead[3]);
+        *reinterpret_cast<uint4*>(qrow + C::kOperand + c * 128) = make_uint4(rest[0], rest[1], rest[2], rest[3]);
+      }
+    }
   }
   fence_proxy_async();
   tc_fence_before();
@@ -359,7 +352,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     }
   } else {
     // ================= softmax teams ================================================================================
-    const int team = warp >> 2;
+    const int team = warp >> 3;
+    const int c_lo = half * (kPuTileBlocks / 2), c_hi = c_lo + kPuTileBlocks / 2;   // this thread's cache blocks of a tile
     bool bad = false;
     float m_row = -INFINITY, l_row = 0.0f, v_max = 0.0f;
     uint8_t* prow = pbuf + team * C::kPTerms * C::kOperand + (r >> 3) * 1024 + (r & 7) * 16;
@@ -377,8 +371,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       const int key0 = T * kPuTileKeys;
       const int nkeys = min(kPuTileKeys, kv_end - key0);
 #pragma unroll 2
-      for (int c = 0; c < kPuTileBlocks; ++c) {
-        if (c * kBlockSize >= nkeys) break;                       // uniform over the CTA
+      for (int c = c_lo; c < c_hi; ++c) {
+        if (c * kBlockSize >= nkeys) break;                       // uniform over the warp
         uint32_t s[16];
         tmem_ld16_issue(tmem + 128 * buf + 16 * c + lane_base, s);
         const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + c * kFp8Header);
@@ -394,14 +388,15 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       __syncwarp();
       if (lane == 0) { mbar_arrive(&bar_sfree[buf]); mbar_arrive(&bar_free1[slot]); }
     }
-    // both teams' maxima (row r of either team is the same row)
-    xch[team * 128 + r] = m_row;
-    if (r == 0) reinterpret_cast<float*>(misc + 4)[team] = v_max;
+    // the maxima of the four threads that saw part of row r (two teams x two halves of the columns)
+    const int part = team * 2 + half;
+    xch[part * kPuRows + r] = m_row;
+    if (r == 0) reinterpret_cast<float*>(misc + 4)[part] = v_max;
     bad = barrier_or(1, kPuSm, bad);
     if (!bad) {
-      m_row = fmaxf(xch[r], xch[128 + r]);
+      m_row = fmaxf(fmaxf(xch[r], xch[kPuRows + r]), fmaxf(xch[2 * kPuRows + r], xch[3 * kPuRows + r]));
       const float* vm = reinterpret_cast<const float*>(misc + 4);
-      v_max = fmaxf(vm[0], vm[1]);
+      v_max = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
     }
     bad = barrier_or(1, kPuSm, bad);          // everybody has read the maxima: their memory may take probabilities
     const float m_use = m_row == -INFINITY ? 0.0f : m_row;
@@ -416,7 +411,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       bool ok = wait_bar(&bar_full[kPuKSlots + vq], vslot_par(t), abort_flag);
       ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
       // the logits are computed: the tile's K slot can be refilled
-      if (ok && (warp & 3) == 0 && lane == 0) mbar_arrive(&bar_kdone[t % kPuKSlots]);
+      if (ok && (warp & 7) == 0 && lane == 0) mbar_arrive(&bar_kdone[t % kPuKSlots]);
       // the team's previous tile must have left the probability operand
       if (ok && mine > 0) ok = wait_bar(&bar_vdone[(t - 2) % kPuVSlots], static_cast<uint32_t>((t - 2) / kPuVSlots) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
@@ -427,7 +422,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       const int nkeys = min(kPuTileKeys, kv_end - key0);
       const int nb = (nkeys + kBlockSize - 1) / kBlockSize;
 #pragma unroll 2
-      for (int c = 0; c < kPuTileBlocks; ++c) {
+      for (int c = c_lo; c < c_hi; ++c) {
         uint4 lead4 = make_uint4(0u, 0u, 0u, 0u), rest4 = make_uint4(0u, 0u, 0u, 0u), last4 = make_uint4(0u, 0u, 0u, 0u);
         if (c < nb) {
           uint32_t s[16];
@@ -470,7 +465,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       if (lane == 0) mbar_arrive(&bar_sfree[buf]);
       // V codes of slots past the context inside the last block are cleared (row r = dim r of V^T), and
       // so is the slot behind an odd number of blocks, which the last instruction also reads
-      if ((nkeys & 15) != 0) {
+      if (half == 0 && (nkeys & 15) != 0) {
         uint4* row = reinterpret_cast<uint4*>(st + (nkeys >> 4) * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
         const int keep = nkeys & 15;
         uint4 w = *row;
@@ -482,7 +477,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         }
         *row = w;
       }
-      if ((nb & 1) != 0)
+      if (half == 0 && (nb & 1) != 0)
         *reinterpret_cast<uint4*>(st + nb * C::kPart + (r >> 3) * 128 + (r & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
       fence_proxy_async();
       mbar_arrive(&bar_pfull[team]);
@@ -495,23 +490,23 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       ok = __all_sync(0xffffffffu, ok);
       bad = !ok;
     }
-    xch[256 + team * 128 + r] = l_row;
+    xch[4 * kPuRows + part * kPuRows + r] = l_row;
     bad = barrier_or(1, kPuSm, bad);
     if (!bad) {
       tc_fence_after();
-      const float l_all = xch[256 + r] + xch[384 + r];
+      const float l_all = (xch[4 * kPuRows + r] + xch[5 * kPuRows + r]) + (xch[6 * kPuRows + r] + xch[7 * kPuRows + r]);
       const float k = l_all > 0.0f ? v_max / (kPuGain * l_all) : 0.0f;
-      // team 0 stores dims 0..63 of the row, team 1 dims 64..127
+      // the four threads of row r store 32 dims each
 #pragma unroll
-      for (int c = 0; c < 4; ++c) {
+      for (int c = 0; c < 2; ++c) {
         uint32_t o[16];
-        tmem_ld16_issue(tmem_o + team * 64 + 16 * c + lane_base, o);
+        tmem_ld16_issue(tmem_o + part * 32 + 16 * c + lane_base, o);
         tmem_ld_wait(o);
         if (live) {
           uint32_t w[8];
 #pragma unroll
           for (int j = 0; j < 8; ++j) w[j] = pack_bf16x2(__uint_as_float(o[2 * j]) * k, __uint_as_float(o[2 * j + 1]) * k);
-          uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + team * 64 + 16 * c);
+          uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + part * 32 + 16 * c);
           dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
           dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
         }
