@@ -229,6 +229,16 @@ __device__ inline void plan_round(const DecodeParams& p, const PlanSmem& s, cons
       }
     }
   }
+  // Decode mode: segments are independent, so the ones that cover their whole sequence go last.  A piece of
+  // a cut sequence then reaches the workspace early, its merge (by whichever CTA delivers last) happens while
+  // the stream still runs, and the CTA's own end is a plain store instead of a counter trip and a merge.
+  // (Only the first and the last segment of a slice can be pieces of a cut sequence.)
+  if (!chunk_mode && nseg > 1 && s.segs[nseg - 1].partial) {
+    const int to = s.segs[0].partial ? 1 : 0;
+    const Segment last = s.segs[nseg - 1];
+    for (int i = nseg - 1; i > to; --i) s.segs[i] = s.segs[i - 1];
+    s.segs[to] = last;
+  }
   s.misc[0] = nseg;
   s.misc[1] = static_cast<int>(xx & 0xffffffffll);
   s.misc[2] = static_cast<int>(xx >> 32);
