@@ -463,7 +463,7 @@ def main():
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch on this workload, from the
 # ncu capture summarised under profiles/ (None while the kernel is newer than the capture).
-DRAM_TRAFFIC_PER_LAUNCH = 136.16e6 + 4.29e6
+DRAM_TRAFFIC_PER_LAUNCH = 136.54e6 + 3.80e6
 
 if __name__ == "__main__":
     main()
