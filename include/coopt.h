@@ -158,6 +158,9 @@ int coopt_paged_decode_static(const coopt_cache* cache, const void* q, void* out
  *                 positions and, when causal != 0, query i sees positions 0..len-n+i
  *   chunk_size    tokens per chunk, a multiple of 16, at most 32768
  *   total_q       cu_q_lens[batch] as known by the host (sizes the launch)
+ * Precondition when total_q == batch: every sequence has exactly one query token, i.e. cu_q_lens is
+ * 0, 1, .., batch (any other split of the same total is reported as COOPT_ERR_INVALID_ARG in the
+ * workspace status word and the output is then meaningless).
  * When every sequence has exactly one query token (total_q == batch) each chunk c of
  * (sequence b, query head h) produces m_c (max logit, natural-log units after sm_scale),
  * l_c (sum of exp(logit - m_c)) and o_c (softmax-weighted V inside the chunk, fp32), stored
@@ -227,6 +230,16 @@ int coopt_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 int coopt_chunk_partials(int32_t batch, int32_t num_q_heads, int32_t head_dim, int32_t max_blocks_per_seq,
                          int32_t chunk_size, size_t* o_offset, size_t* m_offset, size_t* l_offset,
                          int32_t* max_chunks);
+
+/*
+ * coopt_selftest_bounded_wait -- diagnostic: one warp waits on a barrier that never completes, with the
+ * same bounded wait every role of the attention kernels uses (a 2 s limit there), and gives up after
+ * about limit_ns nanoseconds (1 .. 100,000,000).  The paper has no counterpart.  On return from the
+ * stream, *status (DEVICE int32, zero before the call) holds COOPT_ERR_TIMEOUT and *elapsed_us (DEVICE
+ * int32, may be NULL) the microseconds the warp waited; the context stays usable.
+ * Errors: INVALID_ARG (null status, limit out of range), CUDA.
+ */
+int coopt_selftest_bounded_wait(uint64_t limit_ns, int32_t* status, int32_t* elapsed_us, void* stream);
 
 const char* coopt_status_string(int status);
 int coopt_version(void);

@@ -64,6 +64,7 @@ _SIGNATURES = {
                                          ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_void_p,
                                          ctypes.c_size_t, ctypes.c_void_p]),
     "coopt_step_staging_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 5),
+    "coopt_selftest_bounded_wait": (ctypes.c_int, [ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "coopt_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "coopt_version": (ctypes.c_int, []),
 }
@@ -241,6 +242,16 @@ def chunk_partials(workspace: torch.Tensor, batch: int, num_q_heads: int, head_d
     f = lambda off, n: workspace[off:off + 4 * n].view(torch.float32)
     return (f(o.value, rows * head_dim).view(batch, num_q_heads, mc.value, head_dim),
             f(m.value, rows).view(batch, num_q_heads, mc.value), f(l.value, rows).view(batch, num_q_heads, mc.value))
+
+
+def selftest_bounded_wait(limit_ns: int):
+    """coopt_selftest_bounded_wait: returns (status word, microseconds waited) after synchronising."""
+    res = torch.zeros(2, dtype=torch.int32, device="cuda")
+    st = load_library().coopt_selftest_bounded_wait(int(limit_ns), ctypes.c_void_p(res.data_ptr()),
+                                                    ctypes.c_void_p(res.data_ptr() + 4), _stream())
+    _check(st, "coopt_selftest_bounded_wait")
+    torch.cuda.synchronize()
+    return int(res[0].item()), int(res[1].item())
 
 
 def step_staging_bytes(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, max_blocks_per_seq: int) -> int:

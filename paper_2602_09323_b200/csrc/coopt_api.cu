@@ -1,5 +1,7 @@
 // Host side of the C ABI: argument checks, workspace arithmetic, dispatch to the launchers.
 #include <mutex>
+#include <utility>
+#include <vector>
 
 #include "coopt_common.cuh"
 
@@ -9,7 +11,8 @@ int launch_kv_write(const coopt_cache* c, const void* k, const void* v, int64_t 
                     int num_tokens, cudaStream_t stream);
 int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
                         int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
-                        float sm_scale, int32_t chunk_size, void* workspace, int planned_ctas, cudaStream_t stream);
+                        float sm_scale, int32_t chunk_size, const int32_t* cu_q_lens, void* workspace, int planned_ctas,
+                        cudaStream_t stream);
 int launch_paged_prefill(const coopt_cache* c, const void* q, void* out, const int32_t* cu_q_lens,
                          const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
                          int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t causal, float sm_scale,
@@ -40,6 +43,19 @@ const DeviceInfo* device_info() {
   return &info[dev];
 }
 
+bool configure_kernel_smem(const void* kernel, int bytes) {
+  static std::mutex mu;
+  static std::vector<std::pair<const void*, int>> done;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  for (const auto& d : done)
+    if (d.first == kernel && d.second == dev) return true;
+  if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  done.emplace_back(kernel, dev);
+  return true;
+}
+
 namespace {
 
 bool cache_shape_ok(int head_dim, int block_size, int dtype) {
@@ -65,6 +81,9 @@ int planned_ctas(int batch, int num_kv_heads, int max_blocks_per_seq) {
   return decode_planned_ctas(sms, static_cast<long long>(batch) * num_kv_heads * max_blocks_per_seq);
 }
 
+}  // namespace
+
+// Every host-side check of a decode-style call (shared with the entry points of other files).
 int check_attention_args(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
                          int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads) {
   const int rc = check_cache(c);
@@ -81,7 +100,6 @@ int check_attention_args(const coopt_cache* c, const void* q, void* out, const i
   return COOPT_OK;
 }
 
-}  // namespace
 }  // namespace coopt
 
 using namespace coopt;
@@ -166,7 +184,7 @@ int coopt_paged_decode(const coopt_cache* cache, const void* q, void* out, const
     return COOPT_ERR_WORKSPACE;
   const int P = planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq);
   return launch_paged_decode(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads, sm_scale,
-                             0, workspace, P, static_cast<cudaStream_t>(stream));
+                             0, nullptr, workspace, P, static_cast<cudaStream_t>(stream));
 }
 
 int coopt_decode_step(const coopt_cache* cache, const void* k_new, const void* v_new, int64_t kv_token_stride,
@@ -186,7 +204,7 @@ int coopt_decode_step(const coopt_cache* cache, const void* k_new, const void* v
   if (rc != COOPT_OK) return rc;
   const int P = planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq);
   return launch_paged_decode(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads, sm_scale,
-                             0, workspace, P, static_cast<cudaStream_t>(stream));
+                             0, nullptr, workspace, P, static_cast<cudaStream_t>(stream));
 }
 
 int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, const int32_t* cu_q_lens,
@@ -206,7 +224,7 @@ int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, cons
     // one query token per sequence: the Opt-Pa chunk-and-merge decode
     const int P = planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq);
     return launch_paged_decode(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads,
-                               sm_scale, chunk_size, workspace, P, static_cast<cudaStream_t>(stream));
+                               sm_scale, chunk_size, cu_q_lens, workspace, P, static_cast<cudaStream_t>(stream));
   }
   return launch_paged_prefill(cache, q, out, cu_q_lens, block_table, max_blocks_per_seq, context_lens, batch,
                               num_q_heads, total_q, causal, sm_scale, workspace, static_cast<cudaStream_t>(stream));

@@ -180,5 +180,10 @@ struct DeviceInfo {
   int max_smem_optin;
 };
 const DeviceInfo* device_info();  // cached per device; nullptr if the CUDA runtime fails
+// Raises a kernel's dynamic shared-memory limit once per (kernel, device); safe from several host threads.
+bool configure_kernel_smem(const void* kernel, int bytes);
+// Host-side checks of a decode-style call: a coopt_status, nothing is enqueued.
+int check_attention_args(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
+                         int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads);
 
 }  // namespace coopt

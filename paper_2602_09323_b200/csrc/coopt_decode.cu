@@ -93,6 +93,7 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
   }
   plan_prefix(p, plan, tid, kThreads, ctx_early);
   if (tid == 0) plan_slice_publish(p, plan);
+  plan_check_single_query(p, tid, kThreads);
   __syncthreads();
 
   // sequences with an empty context: all-zero output rows
@@ -394,14 +395,7 @@ void chunk_partial_offsets(int batch, int num_q_heads, int head_dim, int max_chu
 template <int D>
 static int launch_one(const DecodeParams& p, int grid, cudaStream_t stream) {
   using C = Cfg<D>;
-  static bool configured[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
-  if (dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(paged_decode_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-      return COOPT_ERR_CUDA;
-    configured[dev] = true;
-  }
+  if (!configure_kernel_smem(reinterpret_cast<const void*>(&paged_decode_kernel<D>), C::kSmemBytes)) return COOPT_ERR_CUDA;
   paged_decode_kernel<D><<<grid, kThreads, C::kSmemBytes, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
@@ -410,13 +404,15 @@ int launch_paged_decode_umma(const DecodeParams& p, int head_dim, int grid, cuda
 
 int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
                         int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
-                        float sm_scale, int32_t chunk_size, void* workspace, int planned_ctas, cudaStream_t stream) {
+                        float sm_scale, int32_t chunk_size, const int32_t* cu_q_lens, void* workspace, int planned_ctas,
+                        cudaStream_t stream) {
   DecodeParams p;
   p.cache = static_cast<const uint8_t*>(c->data);
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.block_table = block_table;
   p.context_lens = context_lens;
+  p.cu_q_lens = cu_q_lens;
   p.max_blocks_per_seq = max_blocks_per_seq;
   p.batch = batch;
   p.num_q_heads = num_q_heads;

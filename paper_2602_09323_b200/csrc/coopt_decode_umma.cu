@@ -215,6 +215,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   }
   plan_prefix(p, plan, tid, kUmmaThreads, ctx_early);
   if (tid == 0) plan_slice_publish(p, plan);
+  plan_check_single_query(p, tid, kUmmaThreads);
   // sequences with an empty context: all-zero output rows
   for (int b = blockIdx.x; b < B; b += gridDim.x) {
     if (plan.pre_blk[b + 1] == plan.pre_blk[b])
@@ -776,14 +777,7 @@ int launch_umma_one(const DecodeParams& p, int grid, cudaStream_t stream) {
   if (!encode_cache_map(&map_part, p.cache, granules, C::kGran, C::kPart / 8) ||
       !encode_cache_map(&map_hdr, p.cache, granules, C::kGran, kFp8Header / 8))
     return COOPT_ERR_CUDA;
-  static bool configured[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
-  if (dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(paged_decode_umma_kernel<D, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-      return COOPT_ERR_CUDA;
-    configured[dev] = true;
-  }
+  if (!configure_kernel_smem(reinterpret_cast<const void*>(&paged_decode_umma_kernel<D, NP>), C::kSmemBytes)) return COOPT_ERR_CUDA;
   paged_decode_umma_kernel<D, NP><<<grid, kUmmaThreads, C::kSmemBytes, stream>>>(p, map_part, map_hdr);
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }

@@ -42,6 +42,7 @@ struct DecodeParams {
   __nv_bfloat16* out;
   const int* block_table;
   const int* context_lens;
+  const int* cu_q_lens;    // chunk mode: prefix sums of the query tokens per sequence (must be 0..batch); else null
   int max_blocks_per_seq;
   int batch, num_q_heads, num_kv_heads, group;
   int num_blocks;
@@ -98,6 +99,15 @@ __device__ __forceinline__ void plan_prefix_load(const DecodeParams& p, int tid,
     const int b = tid + k * nthreads;
     L[k] = b < p.batch ? p.context_lens[b] : 0;
   }
+}
+
+// The decode kernels serve coopt_paged_chunked only when every sequence has exactly one query token.  The
+// host sees no more than the total, so CTA 0 looks at the prefix sums themselves: any other split of the
+// same total is reported in the status word (the rows are then attributed to the wrong sequences).
+__device__ __forceinline__ void plan_check_single_query(const DecodeParams& p, int tid, int nthreads) {
+  if (p.cu_q_lens == nullptr || blockIdx.x != 0) return;
+  for (int b = tid; b <= p.batch; b += nthreads)
+    if (p.cu_q_lens[b] != b) atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG);
 }
 
 // Blocks (and chunks) per sequence and their prefix sums.  Every thread of the CTA calls this.

@@ -399,14 +399,7 @@ __global__ void __launch_bounds__(kPfThreads, 1) paged_prefill_kernel(const Pref
 template <int D>
 int launch_prefill_one(const PrefillParams& p, dim3 grid, cudaStream_t stream) {
   using C = PfCfg<D>;
-  static bool configured[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
-  if (dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(paged_prefill_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::kSmemBytes) != cudaSuccess)
-      return COOPT_ERR_CUDA;
-    configured[dev] = true;
-  }
+  if (!configure_kernel_smem(reinterpret_cast<const void*>(&paged_prefill_kernel<D>), C::kSmemBytes)) return COOPT_ERR_CUDA;
   paged_prefill_kernel<D><<<grid, kPfThreads, C::kSmemBytes, stream>>>(p);
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }

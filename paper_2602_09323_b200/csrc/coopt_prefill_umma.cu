@@ -555,14 +555,7 @@ int launch_paged_prefill_umma(const coopt_cache* c, const void* q, void* out, co
   if (!encode_cache_map(&map_part, c->data, granules, PuCfg::kGran, PuCfg::kPart / 8) ||
       !encode_cache_map(&map_hdr, c->data, granules, PuCfg::kGran, kFp8Header / 8))
     return COOPT_ERR_CUDA;
-  static bool configured[64] = {};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return COOPT_ERR_CUDA;
-  if (dev < 64 && !configured[dev]) {
-    if (cudaFuncSetAttribute(paged_prefill_umma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, PuCfg::kSmemBytes) != cudaSuccess)
-      return COOPT_ERR_CUDA;
-    configured[dev] = true;
-  }
+  if (!configure_kernel_smem(reinterpret_cast<const void*>(&paged_prefill_umma_kernel), PuCfg::kSmemBytes)) return COOPT_ERR_CUDA;
   const dim3 grid(static_cast<unsigned>(tiles), static_cast<unsigned>(c->num_kv_heads));
   paged_prefill_umma_kernel<<<grid, kPuThreads, PuCfg::kSmemBytes, stream>>>(p, map_part, map_hdr);
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;

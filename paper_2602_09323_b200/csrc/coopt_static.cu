@@ -41,13 +41,16 @@ extern "C" int coopt_paged_decode_static(const coopt_cache* cache, const void* q
                                          const int32_t* block_table, int32_t max_blocks_per_seq,
                                          const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
                                          float sm_scale, void* stream) {
-  if (cache == nullptr || cache->num_kv_heads <= 0) return COOPT_ERR_INVALID_ARG;
+  // every refusal comes before the first byte of the shared array is touched
+  int rc = coopt::check_attention_args(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads);
+  if (rc != COOPT_OK) return rc;
+  if (batch == 0) return COOPT_OK;
   const size_t need = coopt_workspace_bytes(batch, num_q_heads, cache->num_kv_heads, cache->head_dim,
                                             max_blocks_per_seq, 0, batch);
   if (need == 0) return COOPT_ERR_INVALID_ARG;
   if (need > static_cast<size_t>(COOPT_STATIC_SCRATCH_BYTES)) return COOPT_ERR_WORKSPACE;   // beyond the built-in maximum
   void* scratch = nullptr;
-  int rc = static_scratch_address(&scratch);
+  rc = static_scratch_address(&scratch);
   if (rc != COOPT_OK) return rc;
   // The array still holds whatever the previous call left: the control words must start at zero.
   rc = coopt_workspace_init(scratch, COOPT_STATIC_SCRATCH_BYTES, stream);

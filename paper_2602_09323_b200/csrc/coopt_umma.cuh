@@ -68,7 +68,8 @@ __device__ __forceinline__ bool barrier_or(int id, int count, bool flag) {
 // Bounded wait that also gives up when another role has already given up.  try_wait lets the hardware
 // park the warp, so waiting warps do not take issue slots from the two single-lane roles that share
 // their schedulers.  The clock and the abort flag are looked at once in 256 unsuccessful tries.
-__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
+                                         uint64_t limit_ns = kWaitLimitNs) {
   uint64_t t0 = 0;
 #pragma unroll 1
   for (uint32_t tries = 1;; ++tries) {
@@ -77,7 +78,7 @@ __device__ __forceinline__ bool wait_bar(uint64_t* bar, uint32_t parity, volatil
       if (*abort_flag != 0) return false;
       const uint64_t now = global_timer_ns();
       if (t0 == 0) t0 = now;
-      else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+      else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
   }
 }
@@ -117,13 +118,14 @@ typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint3
                                       const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                       CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 inline bool encode_cache_map(CUtensorMap* map, const void* cache, long long granules, int gran_bytes, int box_elems) {
-  static TensorMapEncodeFn encode = nullptr;
-  if (!encode) {
+  // looked up once; the initialisation of a function-local static is safe from several host threads
+  static const TensorMapEncodeFn encode = [] {
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult res;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess || !fn) return false;
-    encode = reinterpret_cast<TensorMapEncodeFn>(fn);
-  }
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &res) != cudaSuccess) fn = nullptr;
+    return reinterpret_cast<TensorMapEncodeFn>(fn);
+  }();
+  if (!encode) return false;
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(gran_bytes / 8), static_cast<cuuint64_t>(granules)};
   const cuuint64_t strides[1] = {static_cast<cuuint64_t>(gran_bytes)};
   const cuuint32_t box[2] = {static_cast<cuuint32_t>(box_elems), 1}, elem_strides[2] = {1, 1};

@@ -18,16 +18,34 @@ BF16_HALF_ULP = 2.0 ** -8
 
 
 def check_attention(got: torch.Tensor, ref: np.ndarray, plain: bool = False, what: str = ""):
+    """Elementwise and mean bounds against the float64 reference (NaN entries of ``ref`` are not
+    compared).  Besides the bound on |got - ref|, the kernel's own error is bounded apart from the
+    rounding of the output format: |got - bf16(ref)| <= 2e-2 + one bf16 ulp of ref."""
     got = got.detach().double().cpu().numpy()
     mask = ~np.isnan(ref)
     assert mask.any()
     assert np.isfinite(got[mask]).all(), f"{what}: non-finite output"
-    err = np.abs(got - ref)[mask]
-    bound = MAX_ABS + (0.0 if plain else BF16_HALF_ULP) * np.abs(ref[mask])
+    r = ref[mask]
+    err = np.abs(got[mask] - r)
+    bound = MAX_ABS + (0.0 if plain else BF16_HALF_ULP) * np.abs(r)
     worst = int(np.argmax(err - bound))
     assert np.all(err <= bound), f"{what}: max-abs {err.max():.4g} (excess at {worst}: {err[worst]:.4g} > {bound[worst]:.4g})"
     assert err.mean() <= MEAN_ABS, f"{what}: mean-abs {err.mean():.4g}"
+    r_bf16 = torch.from_numpy(r).to(torch.bfloat16).double().numpy()
+    ulp = np.where(r != 0, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(r), 1e-300))) - 7), 0.0)
+    own = np.abs(got[mask] - r_bf16)
+    assert np.all(own <= MAX_ABS + ulp), f"{what}: kernel error apart from output rounding {np.max(own - ulp):.4g}"
     return float(err.max()), float(err.mean())
+
+
+def check_cache_bit_exact(cache: binding.Cache, codes: np.ndarray, scales: np.ndarray, heads=None, what: str = ""):
+    """Every code, every scale (as bit patterns) and the rest of every header of the device cache against
+    the oracle's cache, for all blocks (unused blocks must still be all zero) and the given kv heads."""
+    g_codes, g_scales, g_rest = cache_to_logical(cache)
+    hs = slice(None) if heads is None else list(heads)
+    assert np.array_equal(g_codes[:, hs], codes[:, hs]), f"{what}: cache codes differ"
+    assert np.array_equal(g_scales[:, hs].view(np.uint32), scales[:, hs].view(np.uint32)), f"{what}: scales differ"
+    assert not g_rest[:, hs].any(), f"{what}: header padding is not zero"
 
 
 _PERM_CACHE = {}
@@ -48,13 +66,15 @@ def granule_index_map(cache: binding.Cache):
     return _PERM_CACHE[key]
 
 
-def cache_to_logical(cache: binding.Cache):
-    """Device cache -> the oracle's logical arrays.
+def cache_to_logical(cache: binding.Cache, heads=None):
+    """Device cache -> the oracle's logical arrays (``heads``: a slice of kv heads, default all).
 
     FP8: (codes uint8 [NB, H, 2, 16, D], scales float32 [NB, H, 2], header_rest uint8 [NB, H, 24]);
     bf16: values float32 [NB, H, 2, 16, D].
     """
     raw = cache.data.cpu().numpy().reshape(cache.num_blocks, cache.num_kv_heads, cache.granule_bytes)
+    if heads is not None:
+        raw = raw[:, heads]
     idx = granule_index_map(cache)
     if cache.dtype == binding.KV_FP8_E4M3:
         codes = raw[:, :, idx]                                   # [NB, H, 2, 16, D]
@@ -69,12 +89,13 @@ def cache_to_logical(cache: binding.Cache):
 
 
 def oracle_fp8_cache(w, calls=None, heads=None):
-    """Oracle cache for workload ``w`` filled by the given list of (row_start, row_stop) calls
-    (default: one call with every token)."""
+    """Oracle cache for workload ``w`` filled by the given list of calls, each a (row_start, row_stop)
+    pair or an array of row indices (default: one call with every token)."""
     codes, scales = kv_cache.new_cache(w.num_blocks, w.num_kv_heads, w.head_dim)
     k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
-    for a, b in (calls or [(0, k.shape[0])]):
-        kv_cache.kv_write(codes, scales, k[a:b], v[a:b], slots[a:b], heads=heads)
+    for call in (calls or [(0, k.shape[0])]):
+        rows = slice(*call) if isinstance(call, tuple) else np.asarray(call, dtype=np.int64)
+        kv_cache.kv_write(codes, scales, k[rows], v[rows], slots[rows], heads=heads)
     return codes, scales
 
 
@@ -82,8 +103,12 @@ def gpu_fill(w, dtype=binding.KV_FP8_E4M3, calls=None):
     """Device cache for workload ``w`` filled through coopt_kv_write with the same calls."""
     cache = binding.Cache(w.num_blocks, w.num_kv_heads, w.head_dim, dtype)
     k, v, slots = w.k.cuda(), w.v.cuda(), w.slot_mapping.cuda()
-    for a, b in (calls or [(0, k.shape[0])]):
-        binding.kv_write(cache, k[a:b], v[a:b], slots[a:b])
+    for call in (calls or [(0, k.shape[0])]):
+        if isinstance(call, tuple):
+            binding.kv_write(cache, k[call[0]:call[1]], v[call[0]:call[1]], slots[call[0]:call[1]])
+        else:
+            rows = torch.as_tensor(np.asarray(call, dtype=np.int64)).cuda()
+            binding.kv_write(cache, k[rows].contiguous(), v[rows].contiguous(), slots[rows].contiguous())
     return cache
 
 

@@ -116,23 +116,53 @@ def test_cold_l2_and_poisoned_workspace_do_not_change_the_result():
     assert torch.equal(outs[0], outs[1]) and torch.equal(outs[0], outs[2])
 
 
-def test_llama13b_decode_full_size_sampled():
-    """BASELINE configuration 2 at full size, in the launch configuration the benchmark times;
-    the oracle recomputes a sample of (sequence, query head) outputs from its own cache."""
+PLAIN_HEADS = [0, 5]      # kv heads of the outlier-free runs (all sequences, all query heads of these groups)
+
+
+def _pairs_of_heads(batch, group, kv_heads):
+    return [(b, h) for b in range(batch) for g in kv_heads for h in range(g * group, (g + 1) * group)]
+
+
+def test_llama13b_decode_full_size_every_output():
+    """BASELINE configuration 2 at full size, in the launch configuration the benchmark times: the whole
+    device cache against the oracle's bit for bit, and every (sequence, query head) output."""
     w = workloads.config_llama13b_decode()
-    out, _ = helpers.gpu_decode(w, helpers.gpu_fill(w))
-    rng = np.random.default_rng(1)
-    pairs = sorted({(int(b), int(h)) for b, h in zip(rng.integers(0, 32, 10), rng.integers(0, 40, 10))})
-    ref = np.full((32, 40, 128), np.nan)
-    k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
-    for b, h in pairs:
-        rows = slice(w.kv_offsets[b], w.kv_offsets[b] + 2048)
-        codes, scales = kv_cache.new_cache(w.num_blocks, 8, 128)
-        kv_cache.kv_write(codes, scales, k[rows], v[rows], slots[rows], heads=[h // 5])
-        ref[b, h] = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(),
-                                              w.context_lens, pairs=[(b, h)])[b, h]
+    cache = helpers.gpu_fill(w)
+    out, _ = helpers.gpu_decode(w, cache)
+    codes, scales = helpers.oracle_fp8_cache(w)
+    helpers.check_cache_bit_exact(cache, codes, scales, what="llama13b decode")
+    ref = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), w.context_lens)
     helpers.check_attention(out, ref, what="llama13b decode")
+
+
+def test_llama13b_decode_full_size_without_v_outliers_meets_the_plain_bound():
+    w = workloads.config_llama13b_decode(v_outliers=False)
+    cache = helpers.gpu_fill(w)
+    out, _ = helpers.gpu_decode(w, cache)
+    codes, scales = helpers.oracle_fp8_cache(w, heads=PLAIN_HEADS)
+    helpers.check_cache_bit_exact(cache, codes, scales, heads=PLAIN_HEADS, what="llama13b decode / plain")
+    ref = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), w.context_lens,
+                                    pairs=_pairs_of_heads(w.batch, 5, PLAIN_HEADS))
+    helpers.check_attention(out, ref, plain=True, what="llama13b decode / plain")
     assert torch.isfinite(out.float()).all()
+
+
+def test_llama13b_mha_ablation_full_size_every_output():
+    """BASELINE configuration 2's ablation at full size: 40 KV heads (one per query head) and a bf16 cache.
+    The oracle's un-quantised write and float64 attention, eight heads at a time to bound host memory."""
+    w = workloads.config_llama13b_mha_ablation()
+    cache = helpers.gpu_fill(w, dtype=binding.KV_BF16)
+    out, _ = helpers.gpu_decode(w, cache)
+    k, v, q = w.k.float().numpy(), w.v.float().numpy(), w.q.float().numpy()
+    slots, table = w.slot_mapping.numpy(), w.block_table.numpy()
+    ref = np.empty((w.batch, 40, 128))
+    for h0 in range(0, 40, 8):
+        vals = kv_cache.new_cache_bf16(w.num_blocks, 8, 128)
+        kv_cache.kv_write_bf16(vals, k[:, h0:h0 + 8], v[:, h0:h0 + 8], slots)
+        g_vals = helpers.cache_to_logical(cache, heads=slice(h0, h0 + 8))
+        assert np.array_equal(g_vals.view(np.uint32), vals.view(np.uint32)), "bf16 cache differs"
+        ref[:, h0:h0 + 8] = attention.paged_attention(q[:, h0:h0 + 8], vals, table, w.context_lens)
+    helpers.check_attention(out, ref, what="llama13b mha ablation")
 
 
 @pytest.mark.parametrize("chunk", [16, 64, 2048])
@@ -208,69 +238,53 @@ def test_decode_step_equals_write_then_decode_bit_for_bit():
     helpers.check_attention(outs[0], ref, what="decode step")
 
 
-def _oracle_sequence_cache(w, b, g, calls):
-    """Oracle cache of one sequence and kv head, written by the given (start, stop) row ranges."""
-    k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
-    codes, scales = kv_cache.new_cache(w.num_blocks, w.num_kv_heads, w.head_dim)
-    off = w.kv_offsets[b]
-    for a, z in calls:
-        kv_cache.kv_write(codes, scales, k[off + a:off + z], v[off + a:off + z], slots[off + a:off + z], heads=[g])
-    return codes, scales
-
-
-def test_mixed_length_serving_step_full_size_sampled():
-    """BASELINE configuration 3 at full size: 64 sequences with contexts uniform in [128, 8192]; the
-    history is filled in bulk, then one token per sequence is appended with coopt_kv_write (which may
-    grow a block's scale and re-express its resident codes) and the decode runs over the updated cache.
-    The oracle replays the same two writes for a sample of (sequence, query head) pairs."""
-    w = workloads.config_mixed_serving()
-    B, L = w.batch, w.context_lens
-    k, v, slots = w.k.cuda(), w.v.cuda(), w.slot_mapping.cuda()
-    last = torch.tensor([w.kv_offsets[b] + L[b] - 1 for b in range(B)])
-    hist = torch.ones(k.shape[0], dtype=torch.bool)
+def _serving_step_calls(w):
+    """Row indices of the two writes of a serving step: the history of every sequence, then its last token."""
+    last = np.array([w.kv_offsets[b] + L - 1 for b, L in enumerate(w.context_lens)])
+    hist = np.ones(w.k.shape[0], dtype=bool)
     hist[last] = False
-    hist_idx, new_idx = hist.nonzero().squeeze(1).cuda(), last.cuda()
-    cache = binding.Cache(w.num_blocks, 8, 128)
-    binding.kv_write(cache, k[hist_idx], v[hist_idx], slots[hist_idx])
-    binding.kv_write(cache, k[new_idx].contiguous(), v[new_idx].contiguous(), slots[new_idx].contiguous())
+    return [np.nonzero(hist)[0], last]
+
+
+@pytest.mark.parametrize("plain", [False, True])
+def test_mixed_length_serving_step_full_size_every_output(plain):
+    """BASELINE configuration 3 at full size: 64 sequences with contexts uniform in [128, 8192]; the history is
+    filled in bulk, then one token per sequence is appended with coopt_kv_write (which may grow a block's
+    scale and re-express its resident codes) and the decode runs over the updated cache.  The oracle replays
+    the same two writes; the whole cache is compared bit for bit and every output within the tolerance
+    (the outlier-free variant, on two kv heads, against the plain bound)."""
+    w = workloads.config_mixed_serving(v_outliers=not plain)
+    calls = _serving_step_calls(w)
+    heads = PLAIN_HEADS if plain else None
+    cache = helpers.gpu_fill(w, calls=calls)
     out, _ = helpers.gpu_decode(w, cache)
     assert torch.isfinite(out.float()).all()
-    rng = np.random.default_rng(3)
-    order = np.argsort(L)
-    picks = [(int(order[0]), 3), (int(order[-1]), 38), (int(rng.integers(0, B)), int(rng.integers(0, 40))),
-             (int(rng.integers(0, B)), int(rng.integers(0, 40)))]
-    ref = np.full((B, 40, 128), np.nan)
-    g_codes, g_scales, _ = helpers.cache_to_logical(cache)
-    for b, h in picks:
-        g = h // 5
-        codes, scales = _oracle_sequence_cache(w, b, g, [(0, L[b] - 1), (L[b] - 1, L[b])])
-        blks = w.block_table[b, :(L[b] + 15) // 16].numpy()
-        assert np.array_equal(g_codes[blks, g], codes[blks, g]) and np.array_equal(g_scales[blks, g], scales[blks, g])
-        ref[b, h] = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), L,
-                                              pairs=[(b, h)])[b, h]
-    helpers.check_attention(out, ref, what="mixed serving step")
+    codes, scales = helpers.oracle_fp8_cache(w, calls=calls, heads=heads)
+    helpers.check_cache_bit_exact(cache, codes, scales, heads=heads, what="mixed serving step")
+    pairs = _pairs_of_heads(w.batch, 5, PLAIN_HEADS) if plain else None
+    ref = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), w.context_lens, pairs=pairs)
+    helpers.check_attention(out, ref, plain=plain, what="mixed serving step")
 
 
-def test_long_context_chunked_full_size_sampled():
-    """BASELINE configuration 4 at full size: contexts of 32768 .. 131072 tokens, chunk size 2048, per-chunk
-    (m, l, o) exported and merged by log-sum-exp; the oracle recomputes two (sequence, query head) pairs."""
-    w = workloads.config_long_context()
+@pytest.mark.parametrize("plain", [False, True])
+def test_long_context_chunked_full_size_every_output(plain):
+    """BASELINE configuration 4 at full size: contexts of 32768 .. 131072 tokens, chunk size 2048; every
+    per-chunk (m, l, o) and every merged output against the oracle's chunk-and-merge path."""
+    w = workloads.config_long_context(v_outliers=not plain)
+    heads = PLAIN_HEADS if plain else None
     cache = helpers.gpu_fill(w)
     out, ws = helpers.gpu_decode(w, cache, chunk_size=2048)
     assert torch.isfinite(out.float()).all()
-    o_c, m_c, l_c = binding.chunk_partials(ws, w.batch, 40, 128, w.block_table.shape[1], 2048)
-    q = w.q.float().numpy()
-    ref = np.full((4, 40, 128), np.nan)
-    for b, h in [(0, 7), (3, 21)]:
-        L = w.context_lens[b]
-        codes, scales = _oracle_sequence_cache(w, b, h // 5, [(0, L)])
-        res, partials = attention.paged_attention_chunked(q, (codes, scales), w.block_table.numpy(), w.context_lens, 2048,
-                                                          pairs=[(b, h)])
-        ref[b, h] = res[b, h]
-        m, l, o = partials[(b, h)]
+    codes, scales = helpers.oracle_fp8_cache(w, heads=heads)
+    helpers.check_cache_bit_exact(cache, codes, scales, heads=heads, what="long context")
+    pairs = _pairs_of_heads(w.batch, 5, PLAIN_HEADS) if plain else None
+    ref, partials = attention.paged_attention_chunked(w.q.float().numpy(), (codes, scales), w.block_table.numpy(),
+                                                      w.context_lens, 2048, pairs=pairs)
+    o_c, m_c, l_c = (t.cpu().numpy() for t in binding.chunk_partials(ws, w.batch, 40, 128, w.block_table.shape[1], 2048))
+    for (b, h), (m, l, o) in partials.items():
         n = len(m)
-        assert n == L // 2048
-        assert np.allclose(m_c[b, h, :n].cpu().numpy(), m, rtol=1e-4, atol=1e-3)
-        assert np.allclose(l_c[b, h, :n].cpu().numpy(), l, rtol=5e-3, atol=1e-4)
-        assert np.allclose(o_c[b, h, :n].cpu().numpy(), o, rtol=5e-3, atol=2e-2)
-    helpers.check_attention(out, ref, what="long context chunked")
+        assert n == w.context_lens[b] // 2048
+        assert np.allclose(m_c[b, h, :n], m, rtol=1e-4, atol=1e-3)
+        assert np.allclose(l_c[b, h, :n], l, rtol=5e-3, atol=1e-4)
+        assert np.allclose(o_c[b, h, :n], o, rtol=5e-3, atol=2e-2)
+    helpers.check_attention(out, ref, plain=plain, what="long context chunked")

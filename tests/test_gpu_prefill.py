@@ -65,26 +65,29 @@ def test_causal_row_equals_decode_over_the_truncated_context():
         assert float((diff - 2.0 ** -7 * out[i].float().abs()).max()) <= 5e-3
 
 
-def test_chunked_prefill_full_size_sampled():
-    """BASELINE configuration 5 at full size: 8 sequences, 4096 cached + 512 new tokens, causal; the
-    oracle recomputes a sample of (query row, query head) outputs from its own cache."""
-    w = workloads.config_chunked_prefill()
-    out = _gpu_prefill(w, helpers.gpu_fill(w))
+@pytest.mark.parametrize("plain", [False, True])
+def test_chunked_prefill_full_size(plain):
+    """BASELINE configuration 5 at full size: 8 sequences, 4096 cached + 512 new tokens, causal.  The whole
+    device cache against the oracle's bit for bit; every query row and head of one (sequence, kv head) group,
+    and for every sequence and kv head the rows on both sides of every boundary between the kernel's tiles of
+    25 query tokens (plus the first and the last row), for one query head of the group."""
+    w = workloads.config_chunked_prefill(v_outliers=not plain)
+    cache = helpers.gpu_fill(w)
+    out = _gpu_prefill(w, cache)
     assert torch.isfinite(out.float()).all()
-    rng = np.random.default_rng(2)
-    k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
-    ref = np.full((8 * 512, 40, 128), np.nan)
-    q = w.q.float().numpy()
-    for b, h in zip(rng.integers(0, 8, 4), rng.integers(0, 40, 4)):
-        rows_kv = slice(w.kv_offsets[b], w.kv_offsets[b] + 4608)
-        codes, scales = kv_cache.new_cache(w.num_blocks, 8, 128)
-        kv_cache.kv_write(codes, scales, k[rows_kv], v[rows_kv], slots[rows_kv], heads=[h // 5])
-        rows = [int(b) * 512 + int(i) for i in (0, 1, 24, 25, 255, 511, int(rng.integers(0, 512)))]
-        part = attention.paged_attention(q, (codes, scales), w.block_table.numpy(), w.context_lens,
-                                         cu_q_lens=w.cu_q_lens.numpy(), causal=True, pairs=[(r, int(h)) for r in rows])
-        for r in rows:
-            ref[r, h] = part[r, h]
-    helpers.check_attention(out, ref, what="chunked prefill full size")
+    heads = [0, 5] if plain else None
+    codes, scales = helpers.oracle_fp8_cache(w, heads=heads)
+    helpers.check_cache_bit_exact(cache, codes, scales, heads=heads, what="chunked prefill")
+    kv_heads = heads or range(8)
+    full_b, full_g = 3, 5
+    pairs = {(full_b * 512 + i, h) for i in range(512) for h in range(full_g * 5, full_g * 5 + 5)}
+    edge_rows = sorted({0, 511} | {i for i in range(512) if i % 25 in (0, 24)})
+    for b in range(8):
+        for g in kv_heads:
+            pairs |= {(b * 512 + i, g * 5 + (b + g) % 5) for i in edge_rows}
+    ref = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), w.context_lens,
+                                    cu_q_lens=w.cu_q_lens.numpy(), causal=True, pairs=sorted(pairs))
+    helpers.check_attention(out, ref, plain=plain, what="chunked prefill full size")
 
 
 @pytest.mark.parametrize("hq,hkv", [(16, 2), (12, 2), (4, 4)])
