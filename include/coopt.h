@@ -113,7 +113,9 @@ int coopt_kv_write(const coopt_cache* cache, const void* k, const void* v, int64
  *   workspace     DEVICE, >= coopt_workspace_bytes(...) with chunk_size = 0, prepared once by
  *                 coopt_workspace_init(); reusable by later calls on the same stream
  * The context of every (sequence, kv head) is cut into byte-balanced pieces across the SMs;
- * pieces are merged by a log-sum-exp reduction inside the same launch.
+ * pieces are merged by a log-sum-exp reduction inside the same launch.  The cut is planned by a
+ * small launch of its own in front of the attention kernel (into the workspace); callers that run
+ * many layers per step plan once with coopt_decode_plan instead.
  * Errors: INVALID_ARG, UNSUPPORTED (group size num_q_heads/num_kv_heads not in 1..8 or not
  * integral, batch > 512, head_dim/block_size/dtype as above), WORKSPACE, CUDA.
  */
@@ -189,6 +191,81 @@ int coopt_decode_step(const coopt_cache* cache, const void* k_new, const void* v
                       const int64_t* slot_mapping, const void* q, void* out, const int32_t* block_table,
                       int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
                       float sm_scale, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Planned decode: the work decomposition of a decode step depends only on the context lengths and the
+ * block table, which every layer of a model shares within one step (the decode loop of Section 2 visits
+ * the same sequences once per layer; Eq. 9's valid blocks are the same in each).  coopt_decode_plan
+ * computes it once -- every CTA's share of the (sequence, kv head, block) list with the physical block
+ * ids looked up and range-checked -- and coopt_decode_step_planned / coopt_decode_layers read it in
+ * every launch instead of working it out again.
+ *
+ * coopt_plan_bytes      bytes of a plan buffer for these shapes (host arithmetic; 0 for bad arguments).
+ * coopt_decode_plan     fills `plan` (DEVICE, 16-byte aligned, >= coopt_plan_bytes) on `stream`.
+ *   block_table, context_lens   DEVICE, as for coopt_paged_decode; context_lens count the token a following
+ *                               step appends
+ *   num_blocks                  of the caches the plan will be used with (block ids are checked against it;
+ *                               a bad id is replaced by 0 and reported by the launches that use the plan)
+ *   chunk_size                  0 for decode; the chunk size of an Opt-Pa chunked call otherwise
+ * Errors: INVALID_ARG, UNSUPPORTED (batch > 512 and the other limits of coopt_paged_decode), WORKSPACE
+ * (plan buffer too small), CUDA.
+ */
+size_t coopt_plan_bytes(int32_t batch, int32_t num_kv_heads, int32_t max_blocks_per_seq, int32_t chunk_size);
+int coopt_decode_plan(const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch,
+                      int32_t num_kv_heads, int32_t num_blocks, int32_t chunk_size, void* plan, size_t plan_bytes,
+                      void* stream);
+
+/*
+ * coopt_decode_step_planned -- Algorithm 1 in ONE launch: phase 1 (the new token of every sequence is
+ * compressed to FP8 and stored, Eq. 5 skip rule, dynamic per-block scales exactly as coopt_kv_write) and
+ * phase 2 with Algorithms 2-3 (attention over the updated cache, exactly as coopt_paged_decode).  The CTA
+ * whose share of the plan holds the last block of a (sequence, kv head) writes that sequence's new token
+ * into it before its copy engine requests the block; no other CTA reads that block.
+ *   plan                       DEVICE, made by coopt_decode_plan for the same batch, num_kv_heads,
+ *                              max_blocks_per_seq, chunk_size and num_blocks (a mismatch is reported as
+ *                              COOPT_ERR_INVALID_ARG in the workspace status word and the launch does nothing)
+ *   k_new, v_new, slot_mapping DEVICE, as for coopt_decode_step; all three NULL = nothing is appended.
+ *                              Precondition: the new token of sequence b is its last position, i.e.
+ *                              slot_mapping[b] / 16 is the block-table entry of position context_lens[b] - 1
+ *                              and slot_mapping[b] % 16 == (context_lens[b] - 1) % 16 (else INVALID_ARG in the
+ *                              status word); sequences with slot_mapping[b] < 0 are not written (Eq. 5)
+ *   chunk_size                 0, or the plan's chunk size: per-chunk partials as coopt_paged_chunked
+ *   flags                      COOPT_FLAG_OVERLAP_PREVIOUS: the launch may start while the kernel before it
+ *                              in the stream still runs.  The caller guarantees that this kernel writes neither
+ *                              the plan nor this cache; everything else the step reads or writes (q, k_new,
+ *                              v_new, slot_mapping, out, workspace) is touched only after that kernel has
+ *                              finished.
+ * Results: cache bytes and output identical to coopt_kv_write followed by coopt_paged_decode.
+ * Errors: as coopt_paged_decode, plus UNSUPPORTED for a bf16 cache.
+ */
+#define COOPT_FLAG_OVERLAP_PREVIOUS 1u
+int coopt_decode_step_planned(const coopt_cache* cache, const void* plan, size_t plan_bytes, const void* k_new,
+                              const void* v_new, int64_t kv_token_stride, const int64_t* slot_mapping, const void* q, void* out,
+                              int32_t max_blocks_per_seq, int32_t batch, int32_t num_q_heads, int32_t chunk_size, float sm_scale,
+                              void* workspace, size_t workspace_bytes, uint32_t flags, void* stream);
+
+/*
+ * coopt_decode_layers -- the decode loop of Section 2 over the layers of a model for one step: one plan,
+ * then one coopt_decode_step_planned launch per layer, enqueued back to back on `stream`.
+ *   layers        HOST array of num_layers entries; every pointer inside is DEVICE memory: the layer's cache
+ *                 (all of one shape), its new token's k/v and slots (all NULL = no append), its q and out
+ *   block_table, context_lens, plan, workspace   shared by all layers
+ *   flags         COOPT_FLAG_OVERLAP_PREVIOUS lets layer l + 1 start while layer l drains (its copy engine
+ *                 reads only the plan and its own cache until layer l has finished)
+ * Errors: as the calls it makes; every argument of every layer is checked before anything is launched.
+ */
+typedef struct coopt_layer_io {
+  const coopt_cache* cache;
+  const void* k_new;            /* DEVICE bf16 [batch][num_kv_heads][head_dim] or NULL */
+  const void* v_new;
+  const int64_t* slot_mapping;  /* DEVICE int64 [batch] or NULL */
+  const void* q;                /* DEVICE bf16 [batch][num_q_heads][head_dim] */
+  void* out;
+} coopt_layer_io;
+int coopt_decode_layers(const coopt_layer_io* layers, int32_t num_layers, int64_t kv_token_stride, const int32_t* block_table,
+                        int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                        float sm_scale, void* plan, size_t plan_bytes, void* workspace, size_t workspace_bytes,
+                        uint32_t flags, void* stream);
 
 /*
  * coopt_decode_step_host — one serving step for callers whose step inputs live in HOST memory

@@ -32,6 +32,13 @@ class coopt_cache(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("block_size", ctypes.c_int32), ("dtype", ctypes.c_int32)]
 
 
+class coopt_layer_io(ctypes.Structure):
+    _fields_ = [("cache", ctypes.POINTER(coopt_cache)), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
+                ("slot_mapping", ctypes.c_void_p), ("q", ctypes.c_void_p), ("out", ctypes.c_void_p)]
+
+
+FLAG_OVERLAP_PREVIOUS = 1
+
 _SIGNATURES = {
     "coopt_granule_bytes": (ctypes.c_size_t, [ctypes.c_int32, ctypes.c_int32]),
     "coopt_cache_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 4),
@@ -64,6 +71,17 @@ _SIGNATURES = {
                                          ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_void_p,
                                          ctypes.c_size_t, ctypes.c_void_p]),
     "coopt_step_staging_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 5),
+    "coopt_plan_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 4),
+    "coopt_decode_plan": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
+                                         ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "coopt_decode_step_planned": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
+                                                 ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                                 ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
+                                                 ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32, ctypes.c_void_p]),
+    "coopt_decode_layers": (ctypes.c_int, [ctypes.POINTER(coopt_layer_io), ctypes.c_int32, ctypes.c_int64, ctypes.c_void_p,
+                                           ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
+                                           ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_uint32,
+                                           ctypes.c_void_p]),
     "coopt_selftest_bounded_wait": (ctypes.c_int, [ctypes.c_uint64, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]),
     "coopt_status_string": (ctypes.c_char_p, [ctypes.c_int]),
     "coopt_version": (ctypes.c_int, []),
@@ -72,6 +90,12 @@ _SIGNATURES = {
 
 def library_path() -> str:
     return _LIB_PATH
+
+
+def use_library(path: str) -> None:
+    """Bind to another build of the library (the trace build) instead of ``libcoopt.so``; call before any other use."""
+    global _lib, _LIB_PATH
+    _lib, _LIB_PATH = None, path
 
 
 def load_library() -> ctypes.CDLL:
@@ -194,6 +218,75 @@ def decode_step(cache: Cache, k_new: torch.Tensor, v_new: torch.Tensor, slot_map
                                           q.shape[0], q.shape[1], float(sm_scale), _ptr(workspace), workspace.numel(), _stream())
     _check(st, "coopt_decode_step")
     return out
+
+
+def plan_bytes(batch: int, num_kv_heads: int, max_blocks_per_seq: int, chunk_size: int = 0) -> int:
+    return load_library().coopt_plan_bytes(batch, num_kv_heads, max_blocks_per_seq, chunk_size)
+
+
+def decode_plan(block_table: torch.Tensor, context_lens: torch.Tensor, num_kv_heads: int, num_blocks: int,
+                chunk_size: int = 0, plan: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """coopt_decode_plan: the step's work decomposition, into ``plan`` (allocated here if not given)."""
+    assert block_table.dtype == torch.int32 and block_table.is_contiguous() and block_table.is_cuda
+    assert context_lens.dtype == torch.int32 and context_lens.is_cuda
+    batch, width = block_table.shape
+    if plan is None:
+        plan = torch.empty(plan_bytes(batch, num_kv_heads, width, chunk_size), dtype=torch.uint8, device=block_table.device)
+    st = load_library().coopt_decode_plan(_ptr(block_table), width, _ptr(context_lens), batch, num_kv_heads, num_blocks,
+                                          int(chunk_size), _ptr(plan), plan.numel(), _stream())
+    _check(st, "coopt_decode_plan")
+    return plan
+
+
+def decode_step_planned(cache: Cache, plan: torch.Tensor, q: torch.Tensor, max_blocks_per_seq: int, sm_scale: float,
+                        workspace: torch.Tensor, k_new: Optional[torch.Tensor] = None, v_new: Optional[torch.Tensor] = None,
+                        slot_mapping: Optional[torch.Tensor] = None, chunk_size: int = 0, flags: int = 0,
+                        out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """coopt_decode_step_planned: append (if k_new, v_new, slot_mapping are given) and attend in one launch."""
+    assert q.dtype == torch.bfloat16 and q.is_contiguous() and q.is_cuda
+    stride = 0
+    if k_new is not None:
+        assert k_new.dtype == torch.bfloat16 and v_new.dtype == torch.bfloat16 and k_new.is_contiguous() and v_new.is_contiguous()
+        assert slot_mapping.dtype == torch.int64 and slot_mapping.is_contiguous()
+        stride = k_new.shape[1] * k_new.shape[2]
+    if out is None:
+        out = torch.empty_like(q)
+    null = ctypes.c_void_p(None)
+    st = load_library().coopt_decode_step_planned(
+        cache.ref(), _ptr(plan), plan.numel(), _ptr(k_new) if k_new is not None else null,
+        _ptr(v_new) if v_new is not None else null, stride, _ptr(slot_mapping) if slot_mapping is not None else null,
+        _ptr(q), _ptr(out), max_blocks_per_seq, q.shape[0], q.shape[1], int(chunk_size), float(sm_scale), _ptr(workspace),
+        workspace.numel(), int(flags), _stream())
+    _check(st, "coopt_decode_step_planned")
+    return out
+
+
+class LayerSet:
+    """The host array of coopt_layer_io entries of a model's layers, built once (it only holds pointers)."""
+
+    def __init__(self, layers):
+        """``layers``: list of dicts with cache, q, out and optionally k_new, v_new, slot_mapping (CUDA tensors)."""
+        self.keep = layers
+        self.array = (coopt_layer_io * len(layers))()
+        for i, L in enumerate(layers):
+            io = self.array[i]
+            io.cache = ctypes.pointer(L["cache"].desc)
+            for name in ("k_new", "v_new", "slot_mapping"):
+                t = L.get(name)
+                setattr(io, name, t.data_ptr() if t is not None else None)
+            io.q, io.out = L["q"].data_ptr(), L["out"].data_ptr()
+        k = layers[0].get("k_new")
+        self.kv_stride = k.shape[1] * k.shape[2] if k is not None else 0
+
+
+def decode_layers(layer_set: LayerSet, block_table: torch.Tensor, context_lens: torch.Tensor, num_q_heads: int,
+                  sm_scale: float, plan: torch.Tensor, workspace: torch.Tensor, flags: int = 0) -> None:
+    """coopt_decode_layers: one plan, then one fused step per layer, enqueued back to back."""
+    st = load_library().coopt_decode_layers(layer_set.array, len(layer_set.array), layer_set.kv_stride, _ptr(block_table),
+                                            block_table.shape[1], _ptr(context_lens), block_table.shape[0], num_q_heads,
+                                            float(sm_scale), _ptr(plan), plan.numel(), _ptr(workspace), workspace.numel(),
+                                            int(flags), _stream())
+    _check(st, "coopt_decode_layers")
 
 
 def paged_decode_static(cache: Cache, q: torch.Tensor, block_table: torch.Tensor, context_lens: torch.Tensor,

@@ -17,7 +17,16 @@ int launch_paged_prefill(const coopt_cache* c, const void* q, void* out, const i
                          const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
                          int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t causal, float sm_scale,
                          void* workspace, cudaStream_t stream);
-size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int batch, int num_q_heads, int max_chunks);
+size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int batch, int num_q_heads, int num_kv_heads,
+                              int max_blocks_per_seq, int chunk_blocks, int max_chunks);
+size_t plan_bytes(int planned_ctas, int batch, int num_kv_heads, int max_blocks_per_seq, int chunk_blocks);
+int launch_decode_plan(const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch,
+                       int32_t num_kv_heads, int32_t num_blocks, int32_t chunk_size, int planned_ctas, void* plan,
+                       cudaStream_t stream);
+int launch_decode_planned(const coopt_cache* c, const void* plan, const void* k_new, const void* v_new, int64_t kv_token_stride,
+                          const int64_t* slot_mapping, const void* q, void* out, int32_t max_blocks_per_seq, int32_t batch,
+                          int32_t num_q_heads, float sm_scale, int32_t chunk_size, const int32_t* cu_q_lens, void* workspace,
+                          int planned_ctas, bool overlap_previous, cudaStream_t stream);
 size_t workspace_control_bytes();
 int decode_planned_ctas(int num_sms, long long upper_blocks);
 int decode_max_batch();
@@ -83,13 +92,22 @@ int planned_ctas(int batch, int num_kv_heads, int max_blocks_per_seq) {
 
 }  // namespace
 
+int check_attention_shapes(const coopt_cache* c, const void* q, void* out, int32_t max_blocks_per_seq, int32_t batch,
+                           int32_t num_q_heads);
+
 // Every host-side check of a decode-style call (shared with the entry points of other files).
 int check_attention_args(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
                          int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads) {
+  const int rc = check_attention_shapes(c, q, out, max_blocks_per_seq, batch, num_q_heads);
+  if (rc != COOPT_OK) return rc;
+  return block_table && context_lens ? COOPT_OK : COOPT_ERR_INVALID_ARG;
+}
+
+int check_attention_shapes(const coopt_cache* c, const void* q, void* out, int32_t max_blocks_per_seq, int32_t batch,
+                           int32_t num_q_heads) {
   const int rc = check_cache(c);
   if (rc != COOPT_OK) return rc;
-  if (!q || !out || !block_table || !context_lens || batch < 0 || max_blocks_per_seq <= 0 || num_q_heads <= 0)
-    return COOPT_ERR_INVALID_ARG;
+  if (!q || !out || batch < 0 || max_blocks_per_seq <= 0 || num_q_heads <= 0) return COOPT_ERR_INVALID_ARG;
   if (num_q_heads % c->num_kv_heads != 0) return COOPT_ERR_UNSUPPORTED;
   const int group = num_q_heads / c->num_kv_heads;
   if (group < 1 || group > 8) return COOPT_ERR_UNSUPPORTED;
@@ -152,7 +170,7 @@ size_t coopt_workspace_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_
   const int group = (num_q_heads + num_kv_heads - 1) / num_kv_heads;
   const int P = planned_ctas(batch, num_kv_heads, max_blocks_per_seq);
   const int mc = chunk_size > 0 ? max_chunks_of(max_blocks_per_seq, chunk_size) : 0;
-  return decode_workspace_bytes(P, group, head_dim, batch, num_q_heads, mc);
+  return decode_workspace_bytes(P, group, head_dim, batch, num_q_heads, num_kv_heads, max_blocks_per_seq, chunk_size / kBlockSize, mc);
 }
 
 int coopt_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -205,6 +223,95 @@ int coopt_decode_step(const coopt_cache* cache, const void* k_new, const void* v
   const int P = planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq);
   return launch_paged_decode(cache, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads, sm_scale,
                              0, nullptr, workspace, P, static_cast<cudaStream_t>(stream));
+}
+
+size_t coopt_plan_bytes(int32_t batch, int32_t num_kv_heads, int32_t max_blocks_per_seq, int32_t chunk_size) {
+  if (batch <= 0 || num_kv_heads <= 0 || max_blocks_per_seq <= 0 || chunk_size < 0 || chunk_size % kBlockSize != 0) return 0;
+  return plan_bytes(planned_ctas(batch, num_kv_heads, max_blocks_per_seq), batch, num_kv_heads, max_blocks_per_seq, chunk_size / kBlockSize);
+}
+
+static int check_plan_args(int32_t batch, int32_t num_kv_heads, int32_t max_blocks_per_seq, int32_t chunk_size, const void* plan,
+                           size_t plan_bytes_given) {
+  if (batch < 0 || num_kv_heads <= 0 || max_blocks_per_seq <= 0) return COOPT_ERR_INVALID_ARG;
+  if (chunk_size < 0 || chunk_size % kBlockSize != 0 || chunk_size / kBlockSize > decode_max_chunk_blocks()) return COOPT_ERR_INVALID_ARG;
+  if (batch > decode_max_batch() || static_cast<long long>(batch) * num_kv_heads > decode_counter_slots()) return COOPT_ERR_UNSUPPORTED;
+  if (static_cast<long long>(batch) * num_kv_heads * max_blocks_per_seq >= (1ll << 31)) return COOPT_ERR_UNSUPPORTED;
+  if (batch == 0) return COOPT_OK;
+  if (!plan || reinterpret_cast<uintptr_t>(plan) % 16 != 0) return COOPT_ERR_INVALID_ARG;
+  if (plan_bytes_given < coopt_plan_bytes(batch, num_kv_heads, max_blocks_per_seq, chunk_size)) return COOPT_ERR_WORKSPACE;
+  return COOPT_OK;
+}
+
+int coopt_decode_plan(const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch,
+                      int32_t num_kv_heads, int32_t num_blocks, int32_t chunk_size, void* plan, size_t plan_bytes_given,
+                      void* stream) {
+  const int rc = check_plan_args(batch, num_kv_heads, max_blocks_per_seq, chunk_size, plan, plan_bytes_given);
+  if (rc != COOPT_OK) return rc;
+  if (!block_table || !context_lens || num_blocks <= 0) return COOPT_ERR_INVALID_ARG;
+  if (batch == 0) return COOPT_OK;
+  return launch_decode_plan(block_table, max_blocks_per_seq, context_lens, batch, num_kv_heads, num_blocks, chunk_size,
+                            planned_ctas(batch, num_kv_heads, max_blocks_per_seq), plan, static_cast<cudaStream_t>(stream));
+}
+
+int coopt_decode_step_planned(const coopt_cache* cache, const void* plan, size_t plan_bytes_given, const void* k_new,
+                              const void* v_new, int64_t kv_token_stride, const int64_t* slot_mapping, const void* q, void* out,
+                              int32_t max_blocks_per_seq, int32_t batch, int32_t num_q_heads, int32_t chunk_size, float sm_scale,
+                              void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
+  int rc = check_attention_shapes(cache, q, out, max_blocks_per_seq, batch, num_q_heads);
+  if (rc != COOPT_OK) return rc;
+  if (cache->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;         // the bf16 ablation kernel plans for itself
+  rc = check_plan_args(batch, cache->num_kv_heads, max_blocks_per_seq, chunk_size, plan, plan_bytes_given);
+  if (rc != COOPT_OK) return rc;
+  const bool append = k_new || v_new || slot_mapping;
+  if (append && (!k_new || !v_new || !slot_mapping || kv_token_stride < static_cast<int64_t>(cache->num_kv_heads) * cache->head_dim))
+    return COOPT_ERR_INVALID_ARG;
+  if ((flags & ~static_cast<uint32_t>(COOPT_FLAG_OVERLAP_PREVIOUS)) != 0) return COOPT_ERR_INVALID_ARG;
+  if (batch == 0) return COOPT_OK;
+  if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, cache->num_kv_heads, cache->head_dim,
+                                                            max_blocks_per_seq, chunk_size, batch))
+    return COOPT_ERR_WORKSPACE;
+  return launch_decode_planned(cache, plan, k_new, v_new, kv_token_stride, slot_mapping, q, out, max_blocks_per_seq, batch,
+                               num_q_heads, sm_scale, chunk_size, nullptr, workspace,
+                               planned_ctas(batch, cache->num_kv_heads, max_blocks_per_seq),
+                               (flags & COOPT_FLAG_OVERLAP_PREVIOUS) != 0, static_cast<cudaStream_t>(stream));
+}
+
+int coopt_decode_layers(const coopt_layer_io* layers, int32_t num_layers, int64_t kv_token_stride, const int32_t* block_table,
+                        int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                        float sm_scale, void* plan, size_t plan_bytes_given, void* workspace, size_t workspace_bytes,
+                        uint32_t flags, void* stream) {
+  if (!layers || num_layers <= 0) return COOPT_ERR_INVALID_ARG;
+  // every check of every layer before anything is launched
+  const coopt_cache* c0 = layers[0].cache;
+  for (int32_t l = 0; l < num_layers; ++l) {
+    const coopt_layer_io& io = layers[l];
+    const int rc = check_attention_shapes(io.cache, io.q, io.out, max_blocks_per_seq, batch, num_q_heads);
+    if (rc != COOPT_OK) return rc;
+    if (io.cache->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;
+    if (io.cache->num_kv_heads != c0->num_kv_heads || io.cache->head_dim != c0->head_dim || io.cache->num_blocks != c0->num_blocks)
+      return COOPT_ERR_INVALID_ARG;                                             // one plan serves every layer
+    const bool append = io.k_new || io.v_new || io.slot_mapping;
+    if (append && (!io.k_new || !io.v_new || !io.slot_mapping || kv_token_stride < static_cast<int64_t>(c0->num_kv_heads) * c0->head_dim))
+      return COOPT_ERR_INVALID_ARG;
+  }
+  int rc = check_plan_args(batch, c0->num_kv_heads, max_blocks_per_seq, 0, plan, plan_bytes_given);
+  if (rc != COOPT_OK) return rc;
+  if (!block_table || !context_lens) return COOPT_ERR_INVALID_ARG;
+  if ((flags & ~static_cast<uint32_t>(COOPT_FLAG_OVERLAP_PREVIOUS)) != 0) return COOPT_ERR_INVALID_ARG;
+  if (batch == 0) return COOPT_OK;
+  if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, c0->num_kv_heads, c0->head_dim, max_blocks_per_seq, 0, batch))
+    return COOPT_ERR_WORKSPACE;
+  const int P = planned_ctas(batch, c0->num_kv_heads, max_blocks_per_seq);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = launch_decode_plan(block_table, max_blocks_per_seq, context_lens, batch, c0->num_kv_heads, c0->num_blocks, 0, P, plan, st);
+  for (int32_t l = 0; l < num_layers && rc == COOPT_OK; ++l) {
+    const coopt_layer_io& io = layers[l];
+    // layer l > 0 may start while layer l - 1 drains: its copy warp reads only the plan and its own cache
+    rc = launch_decode_planned(io.cache, plan, io.k_new, io.v_new, kv_token_stride, io.slot_mapping, io.q, io.out, max_blocks_per_seq,
+                               batch, num_q_heads, sm_scale, 0, nullptr, workspace, P,
+                               l > 0 && (flags & COOPT_FLAG_OVERLAP_PREVIOUS) != 0, st);
+  }
+  return rc;
 }
 
 int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, const int32_t* cu_q_lens,
@@ -302,6 +409,6 @@ const char* coopt_status_string(int status) {
   }
 }
 
-int coopt_version(void) { return 100; }
+int coopt_version(void) { return 200; }
 
 }  // extern "C"

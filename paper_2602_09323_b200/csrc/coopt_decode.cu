@@ -365,13 +365,25 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
 
 }  // namespace
 
-// Workspace layout: [header 256 B: word 0 = status][counters int32 x 16384][partials].
-size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int batch, int num_q_heads, int max_chunks) {
+// Workspace layout: [header 256 B: word 0 = status][counters int32 x 16384][partials][plan of a one-off call].
+size_t plan_bytes(int planned_ctas, int batch, int num_kv_heads, int max_blocks_per_seq, int chunk_blocks);
+int plan_cta_stride(int planned_ctas, int batch, int num_kv_heads, int max_blocks_per_seq, int chunk_blocks);
+int launch_decode_plan(const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch,
+                       int32_t num_kv_heads, int32_t num_blocks, int32_t chunk_size, int planned_ctas, void* plan,
+                       cudaStream_t stream);
+
+static size_t partials_bytes(int planned_ctas, int group, int head_dim, int batch, int num_q_heads, int max_chunks) {
   size_t bytes = kWsHeaderBytes + static_cast<size_t>(kCounterSlots) * 4;
   const size_t dec = static_cast<size_t>(2) * planned_ctas * group * (head_dim + 2) * 4;
   const size_t chk = static_cast<size_t>(batch) * num_q_heads * max_chunks * (head_dim + 2) * 4;
   // chunk mode holds both: the per-chunk partials it exports and the merged pieces of the CTAs' runs
-  return bytes + (max_chunks > 0 ? chk + dec + 256 : dec) + 256;
+  return (bytes + (max_chunks > 0 ? chk + dec + 256 : dec) + 256 + 255) / 256 * 256;
+}
+size_t decode_workspace_bytes(int planned_ctas, int group, int head_dim, int batch, int num_q_heads, int num_kv_heads,
+                              int max_blocks_per_seq, int chunk_blocks, int max_chunks) {
+  // calls that bring no plan of their own (coopt_paged_decode, coopt_paged_chunked) plan into the workspace
+  return partials_bytes(planned_ctas, group, head_dim, batch, num_q_heads, max_chunks) +
+         plan_bytes(planned_ctas, batch, num_kv_heads, max_blocks_per_seq, chunk_blocks);
 }
 size_t workspace_control_bytes() { return kWsHeaderBytes + static_cast<size_t>(kCounterSlots) * 4; }
 
@@ -400,13 +412,13 @@ static int launch_one(const DecodeParams& p, int grid, cudaStream_t stream) {
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
 
-int launch_paged_decode_umma(const DecodeParams& p, int head_dim, int grid, cudaStream_t stream);
+int launch_paged_decode_umma(const DecodeParams& p, int head_dim, int grid, bool overlap_previous, cudaStream_t stream);
 
-int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
-                        int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
-                        float sm_scale, int32_t chunk_size, const int32_t* cu_q_lens, void* workspace, int planned_ctas,
-                        cudaStream_t stream) {
-  DecodeParams p;
+// Everything of DecodeParams that does not depend on where the plan comes from.
+static void fill_decode_params(DecodeParams& p, const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
+                               int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                               float sm_scale, int32_t chunk_size, const int32_t* cu_q_lens, void* workspace, int planned_ctas) {
+  p = DecodeParams{};
   p.cache = static_cast<const uint8_t*>(c->data);
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.out = static_cast<__nv_bfloat16*>(out);
@@ -448,9 +460,48 @@ int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const in
     p.run_m = p.part_m;
     p.run_l = p.part_l;
   }
-  // FP8 cache: the tcgen05 kernel; bf16 ablation cache: the mma.sync kernel of this file
-  if (c->dtype == COOPT_KV_FP8_E4M3) return launch_paged_decode_umma(p, c->head_dim, planned_ctas, stream);
-  return c->head_dim == 128 ? launch_one<128>(p, planned_ctas, stream) : launch_one<64>(p, planned_ctas, stream);
+}
+
+static void attach_plan(DecodeParams& p, const void* plan) {
+  p.plan_header = static_cast<const PlanHeader*>(plan);
+  p.plan = static_cast<const uint8_t*>(plan) + kPlanHeaderBytes;
+  p.plan_cta_stride = plan_cta_stride(p.planned_ctas, p.batch, p.num_kv_heads, p.max_blocks_per_seq, p.chunk_blocks);
+  p.plan_key = plan_key(p.planned_ctas, p.batch, p.num_kv_heads, p.chunk_blocks, p.max_blocks_per_seq, p.num_blocks);
+}
+
+// A call that brings no plan: the FP8 kernel's plan is made in the workspace first (one more small launch);
+// the bf16 ablation kernel plans inside its own CTAs.
+int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const int32_t* block_table,
+                        int32_t max_blocks_per_seq, const int32_t* context_lens, int32_t batch, int32_t num_q_heads,
+                        float sm_scale, int32_t chunk_size, const int32_t* cu_q_lens, void* workspace, int planned_ctas,
+                        cudaStream_t stream) {
+  DecodeParams p;
+  fill_decode_params(p, c, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads, sm_scale, chunk_size,
+                     cu_q_lens, workspace, planned_ctas);
+  if (c->dtype != COOPT_KV_FP8_E4M3)
+    return c->head_dim == 128 ? launch_one<128>(p, planned_ctas, stream) : launch_one<64>(p, planned_ctas, stream);
+  void* plan = static_cast<uint8_t*>(workspace) + partials_bytes(planned_ctas, p.group, c->head_dim, batch, num_q_heads, p.max_chunks);
+  const int rc = launch_decode_plan(block_table, max_blocks_per_seq, context_lens, batch, c->num_kv_heads, c->num_blocks, chunk_size,
+                                    planned_ctas, plan, stream);
+  if (rc != COOPT_OK) return rc;
+  attach_plan(p, plan);
+  return launch_paged_decode_umma(p, c->head_dim, planned_ctas, false, stream);
+}
+
+// A call that brings its plan (coopt_decode_plan) and may append one token per sequence in the same launch.
+int launch_decode_planned(const coopt_cache* c, const void* plan, const void* k_new, const void* v_new, int64_t kv_token_stride,
+                          const int64_t* slot_mapping, const void* q, void* out, int32_t max_blocks_per_seq, int32_t batch,
+                          int32_t num_q_heads, float sm_scale, int32_t chunk_size, const int32_t* cu_q_lens, void* workspace,
+                          int planned_ctas, bool overlap_previous, cudaStream_t stream) {
+  DecodeParams p;
+  fill_decode_params(p, c, q, out, nullptr, max_blocks_per_seq, nullptr, batch, num_q_heads, sm_scale, chunk_size, cu_q_lens,
+                     workspace, planned_ctas);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.slot_mapping = reinterpret_cast<const long long*>(slot_mapping);
+  p.kv_token_stride = kv_token_stride;
+  attach_plan(p, plan);
+  return launch_paged_decode_umma(p, c->head_dim, planned_ctas, overlap_previous, stream);
 }
 
 }  // namespace coopt

@@ -36,10 +36,20 @@
 //               exported as its own (m, l, o)), and writes a run that covers its sequence straight to the output.
 // A run that does not cover its whole sequence leaves (m, l, o) in the workspace; the CTA that
 // delivers the last piece merges all pieces by log-sum-exp and writes the bf16 output.
+// What the CTA has to do comes from a plan (coopt_plan.cu) that one bulk copy brings into shared memory:
+// its rounds of segments with the physical block ids already looked up.  A step that appends a token per
+// sequence (Algorithm 1 phase 1 followed by phase 2 in one launch) lets team 1 write the new token's
+// granule of every (sequence, kv head) whose last block lies in this CTA's slice -- no other CTA reads that
+// block -- before the copy warp requests the tile that holds it.
 // Every wait is bounded; a wait that runs out is reported in the workspace status word and all roles
 // leave through the common exit, which frees the tensor memory.
+#include <mutex>
+#include <vector>
+
 #include "coopt_plan.cuh"
+#include "coopt_trace.cuh"
 #include "coopt_umma.cuh"
+#include "coopt_write.cuh"
 
 namespace coopt {
 
@@ -74,23 +84,22 @@ struct UCfg {
   static constexpr int kRingOff = 0;
   static constexpr int kQOff = kRingOff + kStages * kStageBytes;
   static constexpr int kPOff = kQOff + 2 * kQBytes;
-  static constexpr int kIdsOff = kPOff + 4 * kPBytes;
-  static constexpr int kPreBlkOff = kIdsOff + kCap * 4;
-  static constexpr int kPreUnitOff = kPreBlkOff + (kMaxBatch + 4) * 4;
-  static constexpr int kSegOff = kPreUnitOff + (kMaxBatch + 4) * 4;
-  static constexpr int kXchOff = kSegOff + kMaxSeg * static_cast<int>(sizeof(Segment));
+  static constexpr int kPlanOff = kPOff + 4 * kPBytes;             // one round of the plan: header, segments, block ids
+  static constexpr int kXchOff = kPlanOff + (kPlanRoundMax + 127) / 128 * 128;
   static constexpr int kMlOff = kXchOff + 2 * kXchFloats * 4;       // [2 segment parities][2 teams][kMlFloats]
   static constexpr int kRedOff = kMlOff + 2 * 2 * kMlFloats * 4;
   // int red_max [2 teams][4 warps][12], uint red_q [4][8], float qscale [2][8]
   static constexpr int kRedBytes = (2 * 4 * 12 + 4 * 8 + 2 * 8) * 4;
   static constexpr int kBarOff = kRedOff + kRedBytes;
-  static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2;
+  static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2 + 2;
+  static constexpr int kWriteStage = 4 * kBlockSize * D;       // staging of team 1's four warps for the fused append
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kSmemBytes = kMiscOff + 128;            // 64 bytes of planner words and flags, 64 of the published slice
   static_assert(kStageBytes % 128 == 0 && kKArea % 128 == 0 && kHdrOff % 128 == 0 && (kGatherRows * kPart) % 128 == 0 &&
                     (kGatherRows * kFp8Header) % 128 == 0, "tensor copies land on 128-byte boundaries");
   static_assert(kPart / 8 <= 256 && kGran % 16 == 0, "one box row is at most 256 eight-byte elements");
   static_assert(kSmemBytes <= 232448, "shared memory of one CTA");
+  static_assert(kWriteStage <= kStageBytes && kPlanFirstChunk <= kPlanRoundMax && kPlanOff % 128 == 0, "staging areas");
 };
 
 // The CTA that delivered the last piece of a (sequence, kv head) merges all pieces by log-sum-exp (the
@@ -156,13 +165,14 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   uint8_t* ring = smem + C::kRingOff;
   uint8_t* qbuf = smem + C::kQOff;
   uint8_t* pbuf = smem + C::kPOff;
+  uint8_t* plan_smem = smem + C::kPlanOff;
+  const PlanRound* round_hdr = reinterpret_cast<const PlanRound*>(plan_smem);
   PlanSmem plan;
-  plan.ids = reinterpret_cast<int*>(smem + C::kIdsOff);
-  plan.pre_blk = reinterpret_cast<int*>(smem + C::kPreBlkOff);
-  plan.pre_unit = reinterpret_cast<int*>(smem + C::kPreUnitOff);
-  plan.segs = reinterpret_cast<Segment*>(smem + C::kSegOff);
-  plan.misc = reinterpret_cast<int*>(smem + C::kMiscOff);          // [0..2] planner
-  plan.slice = reinterpret_cast<long long*>(smem + C::kMiscOff + 64);
+  plan.segs = reinterpret_cast<Segment*>(plan_smem + 64);
+  plan.ids = nullptr;                                               // behind the round's segments
+  plan.pre_blk = plan.pre_unit = nullptr;
+  plan.misc = reinterpret_cast<int*>(smem + C::kMiscOff);          // flags and the tensor-memory address
+  plan.slice = nullptr;
   float* xch = reinterpret_cast<float*>(smem + C::kXchOff);         // [2 teams][kXchFloats]
   float* mlbuf = reinterpret_cast<float*>(smem + C::kMlOff);        // [2 segment parities][2 teams][kMlFloats]
   int* red_max = reinterpret_cast<int*>(smem + C::kRedOff);         // [2][4][12] per-warp maxima of a tile (ordered ints)
@@ -178,6 +188,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   uint64_t* bar_qfull = bar_ofree + 4;              // [2] query operand of a segment is in shared memory
   uint64_t* bar_efull = bar_qfull + 2;              // [2] both teams' pieces of a segment are in the exchange area
   uint64_t* bar_efree = bar_efull + 2;              // [2] the epilogue warp has read them
+  uint64_t* bar_plan = bar_efree + 2;               // a piece of the plan has landed in shared memory
+  uint64_t* bar_wdone = bar_plan + 1;               // team 1 has written the round's new tokens to the cache
   volatile int* abort_flag = plan.misc + 4;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(plan.misc + 5);
 
@@ -188,14 +200,15 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   // ---- set-up ---------------------------------------------------------------------------------------
   // two trips to memory start before anything else: the context lengths for the planner, and the copy
   // engine's view of the cache (fetched on first use otherwise, in front of the first tile)
-  int ctx_early[2];
-  plan_prefix_load(p, tid, kUmmaThreads, ctx_early);
+  COOPT_TRACE_CYCLES(p.trace, kTrEntry, tid == 0);
+  COOPT_TRACE_NS(p.trace, kTrEntryNs, tid == 0);
+  const uint8_t* plan_region = p.plan + static_cast<size_t>(blockIdx.x) * p.plan_cta_stride;
   if (tid == kProducerWarp * 32) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_part) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hdr) : "memory");
   }
   // rows of Qg / Pg that no head uses must hold zero codes
-  for (int i = tid; i < (C::kIdsOff - C::kQOff) / 16; i += kUmmaThreads)
+  for (int i = tid; i < (C::kPlanOff - C::kQOff) / 16; i += kUmmaThreads)
     reinterpret_cast<uint4*>(smem + C::kQOff)[i] = make_uint4(0u, 0u, 0u, 0u);
   if (tid == 0) {
     for (int i = 0; i < C::kStages; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_empty[i], 1); }
@@ -206,46 +219,81 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       mbar_init(&bar_ofree[i], 4);
     }
     for (int i = 0; i < 2; ++i) { mbar_init(&bar_qfull[i], kTeamThreads); mbar_init(&bar_efull[i], kSmThreads); mbar_init(&bar_efree[i], 1); }
+    mbar_init(bar_plan, 1);
+    mbar_init(bar_wdone, 4);
     mbar_fence_init();
     *abort_flag = 0;
+    // the first round of this CTA's plan: its size is not known yet, so a fixed first piece is fetched
+    mbar_expect_tx(bar_plan, kPlanFirstChunk);
+    bulk_copy_g2s(plan_smem, plan_region, kPlanFirstChunk, bar_plan);
   }
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmemCols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  }
-  plan_prefix(p, plan, tid, kUmmaThreads, ctx_early);
-  if (tid == 0) plan_slice_publish(p, plan);
-  plan_check_single_query(p, tid, kUmmaThreads);
-  // sequences with an empty context: all-zero output rows
-  for (int b = blockIdx.x; b < B; b += gridDim.x) {
-    if (plan.pre_blk[b + 1] == plan.pre_blk[b])
-      for (int i = tid; i < Hq * D; i += kUmmaThreads) p.out[static_cast<size_t>(b) * Hq * D + i] = __float2bfloat16(0.0f);
   }
   fence_proxy_async();
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  // Launched as a programmatic dependent of the kernel before it, this CTA may have started while that kernel
+  // still runs.  Only the copy warp goes ahead (the plan and the cache blocks it requests were complete before
+  // that kernel began); every other role waits here for it to finish, because the queries, the new tokens, the
+  // output and the workspace may all be its results.  Without such a launch the wait returns at once.
+  if (warp != kProducerWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  plan_check_single_query(p, tid, kUmmaThreads);
+  // sequences with an empty context: all-zero output rows (the epilogue warp has nothing else to do yet)
+  if (warp == kEpilogueWarp) {
+    for (int b = blockIdx.x; b < B; b += gridDim.x) {
+      if ((p.plan_header->empty_bits[b >> 5] >> (b & 31)) & 1u) {
+        uint4* row = reinterpret_cast<uint4*>(p.out + static_cast<size_t>(b) * Hq * D);
+        for (int i = lane; i < Hq * D / 8; i += 32) row[i] = make_uint4(0u, 0u, 0u, 0u);
+      }
+    }
+  }
+  COOPT_TRACE_CYCLES(p.trace, kTrSetupDone, tid == 0);
   const uint32_t tmem_o = tmem + 64;                           // logits buffer b at column 16 b, output buffer b at 64 + NP b
   const uint32_t lane_base = static_cast<uint32_t>(warp & 3) * 32u << 16;
 
-  PlanSlice sl;
-  const bool active = plan_slice_fetch(plan, sl);
-
+  const bool has_new = p.k_new != nullptr;      // this launch also appends one token per sequence
   // counters that persist across rounds (every role advances its own copy identically)
   uint32_t tile_no = 0;     // tiles so far: ring stage, and team / buffer = tile_no & 1
   uint32_t seg_no = 0;      // segments so far: parity of the Q buffer and of the exchange area
 
-  long long x = active ? sl.lo : 0;
-  const long long x_end = active ? sl.hi : 0;
-  while (x < x_end) {
-    if (tid == 0) plan_round(p, plan, sl, x);
-    __syncthreads();
-    const int nseg = plan.misc[0];
-    const long long x_next = (static_cast<long long>(plan.misc[2]) << 32) | static_cast<unsigned int>(plan.misc[1]);
-    if (tid < nseg) plan_round_finish(p, plan, sl, tid);
-    plan_stage_ids(p, plan, nseg, tid, kUmmaThreads);
-    __syncthreads();
+  uint32_t round_no = 0, plan_phase = 0;
+  size_t plan_at = 0;                            // where the current round starts in the CTA's plan region
+  for (;;) {
+    // ---- this round of the plan: what the first fetch did not bring is fetched now ---------------------
+    bool plan_ok = wait_bar(bar_plan, plan_phase & 1u, abort_flag);
+    ++plan_phase;
+    const int round_bytes = plan_ok ? round_hdr->bytes : 0;
+    if (plan_ok && round_bytes > kPlanFirstChunk) {
+      if (tid == 0) {
+        mbar_expect_tx(bar_plan, round_bytes - kPlanFirstChunk);
+        bulk_copy_g2s(plan_smem + kPlanFirstChunk, plan_region + plan_at + kPlanFirstChunk, round_bytes - kPlanFirstChunk, bar_plan);
+      }
+      plan_ok = wait_bar(bar_plan, plan_phase & 1u, abort_flag);
+      ++plan_phase;
+    }
+    plan_ok = __syncthreads_and(plan_ok);       // one verdict for the whole CTA
+    if (!plan_ok) {
+      if (tid == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+      break;
+    }
+    const int nseg = round_hdr->nseg;
+    if (round_hdr->key != p.plan_key || nseg > kMaxSeg || round_bytes > kPlanRoundMax || round_hdr->n_ids > kCap) {
+      if (tid == 0) atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG);              // not a plan of this problem
+      break;
+    }
+    if (tid == 0 && round_hdr->status != 0) atomicCAS(p.status, 0, round_hdr->status);   // what the planner found
+    if (nseg <= 0) break;                                                        // nothing (left) to do
+    const bool last_round = round_hdr->last != 0;
+    plan.ids = reinterpret_cast<int*>(plan_smem + 64 + nseg * 64);
+    const uint32_t round_tile0 = tile_no;             // every role's tile counter agrees at the start of a round
+    uint8_t* write_stage = ring + ((round_tile0 + C::kStages - 1) % C::kStages) * C::kStageBytes;   // the stage the ring fills last
+    COOPT_TRACE_CYCLES(p.trace, kTrIdsStaged, tid == 0 && round_no == 0);
+    COOPT_TRACE_VALUE(p.trace, kTrNumSeg, tid == 0 && round_no == 0, nseg);
 
     if (warp == kProducerWarp) {
       // ================= copies: six gather requests per tile ==================================================
@@ -261,10 +309,20 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
                              : what == 1 ? C::kKArea + q4 * C::kGatherRows * C::kPart
                                          : C::kHdrOff + q4 * C::kGatherRows * kFp8Header;
       const CUtensorMap* map = what == 2 ? &map_hdr : &map_part;
+      // A step that appends tokens: the tile that holds a sequence's last block, and the ring stage that
+      // team 1 borrows as staging, are not requested before team 1 has written the round's new tokens.
+      bool writes_pending = has_new && round_hdr->n_tail > 0;
       for (int si = 0; si < nseg && ok; ++si) {
         const int n = plan.segs[si].n, g = plan.segs[si].g;
+        const bool seg_tail = (plan.segs[si].run_flags & kSegTail) != 0;
         const int* seg_ids = plan.ids + plan.segs[si].list_off;
         for (int k0 = 0; k0 < n; k0 += kTileBlocks) {
+          if (writes_pending && ((seg_tail && k0 + kTileBlocks >= n) || tile_no - round_tile0 == C::kStages - 1)) {
+            if (lane == 0) ok = wait_bar(bar_wdone, round_no & 1u, abort_flag);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            writes_pending = false;
+          }
           const int nb = min(kTileBlocks, n - k0);
           const int ngroups = (nb + C::kGatherRows - 1) / C::kGatherRows;
           int rows[C::kGatherRows] = {0, 0, 0, 0};
@@ -284,9 +342,12 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) break;
           if (lane < 3 * ngroups) gather4_g2s(st + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[stage]);
+          COOPT_TRACE_CYCLES(p.trace, kTrFirstCopy, lane == 0 && tile_no == 0);
+          COOPT_TRACE_CYCLES(p.trace, kTrLastCopy, lane == 0);
           ++tile_no;
         }
       }
+      COOPT_TRACE_VALUE(p.trace, kTrNumTiles, lane == 0, tile_no);
       if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     } else if (warp == kMmaWarp) {
       // ================= logits: S^T = Ktile . Qg^T (one lane) ================================================
@@ -305,6 +366,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             ok = wait_bar(&bar_full[stage], (tile_no / C::kStages) & 1u, abort_flag);
             if (ok && use > 0) ok = wait_bar(&bar_sfree[buf], (use - 1) & 1u, abort_flag);
             if (!ok) break;
+            COOPT_TRACE_CYCLES(p.trace, kTrFirstLanded, tile_no == 0);
+            COOPT_TRACE_CYCLES(p.trace, kTrLastLanded, true);
             tc_fence_after();
             const uint64_t dk = desc_k + ((stage * C::kStageBytes) >> 4);
 #pragma unroll
@@ -332,6 +395,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             for (int ks = 0; ks < nks; ++ks)
               umma_f8(tmem_o + NP * buf, dv + ks * ((2 * C::kPart) >> 4), dp + ks * 16, umma_idesc(NP), ks > 0 ? 1u : 0u);
             umma_commit(&bar_empty[stage]);     // the stage is free again and the tile's product is in its output buffer
+            COOPT_TRACE_CYCLES(p.trace, kTrLastPv, true);
           }
         }
         if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
@@ -353,6 +417,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         ok = wait_bar(&bar_efull[par], (seg_no >> 1) & 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
+        COOPT_TRACE_CYCLES(p.trace, kTrLastHandOff, lane == 0);
+        COOPT_TRACE_CYCLES(p.trace, kTrSegBase + static_cast<int>(seg_no), lane == 0 && seg_no < 20);
         const int h0 = sg.g * G;
         const size_t run_base = static_cast<size_t>(sg.run_slot) * G;
         // a run that an earlier round of this CTA began: its state was parked in the run's workspace slot
@@ -459,6 +525,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
 #pragma unroll
         for (int h = 0; h < kGMax; ++h) { acc[h] = make_float4(0.0f, 0.0f, 0.0f, 0.0f); acc_m[h] = -INFINITY; acc_l[h] = 0.0f; }
         __syncwarp();                         // every store of the piece has been issued
+        COOPT_TRACE_CYCLES(p.trace, kTrPieceStored, lane == 0);
         int last = 0;
         if (lane == 0) {
           // release (this CTA's piece is visible before the count moves) and acquire (the other pieces
@@ -470,9 +537,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           if (last) *counter = 0;             // ready for the next call
         }
         last = __shfl_sync(0xffffffffu, last, 0);
+        COOPT_TRACE_CYCLES(p.trace, kTrCounted, lane == 0);
         if (last && d0 < D)
           merge_run_pieces<D, kGMax>(p.run_o, p.run_m, p.run_l, p.out + (static_cast<size_t>(sg.b) * Hq + h0) * D, sg.first_cta, sg.run_expected, G, d0);
       }
+      COOPT_TRACE_CYCLES(p.trace, kTrEpilogueDone, lane == 0);
       if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     } else {
       // ================= softmax teams: thread t owns token t of its tiles and dim t of its output =====
@@ -572,9 +641,45 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       };
 
       if (team == 0 && nseg > 0) { load_q(plan.segs[0]); publish_q(seg_no); }
+      if (team == 1 && has_new) {
+        // ---- Algorithm 1 phase 1 inside the step: the new token of every (sequence, kv head) whose last block
+        // lies in this round.  Warp wq takes (tail segment, K | V) pairs wq, wq + 4, ..; the scale rule is the
+        // write kernels' own (write_part), staged in a ring stage the copy warp has not reached yet.
+        WriteParams wp;
+        wp.cache = const_cast<uint8_t*>(p.cache);
+        wp.k = p.k_new; wp.v = p.v_new;
+        wp.slot_mapping = reinterpret_cast<const int64_t*>(p.slot_mapping);
+        wp.token_stride = p.kv_token_stride;
+        wp.num_tokens = B; wp.num_kv_heads = Hkv; wp.num_blocks = p.num_blocks;
+        int task = 0;
+        for (int si = 0; si < nseg; ++si) {
+          const Segment& sg = plan.segs[si];
+          if (!(sg.run_flags & kSegTail)) continue;
+          for (int which = 0; which < 2; ++which, ++task) {
+            if ((task & 3) != wq) continue;
+            const long long slot = p.slot_mapping[sg.b];
+            if (slot < 0) continue;                                          // Eq. 5: the token is skipped
+            const long long blk = slot / kBlockSize;
+            // the new token is the sequence's last position: its slot must name the last block of the table
+            if (blk != plan.ids[sg.list_off + sg.n - 1] || static_cast<int>(slot % kBlockSize) != (sg.ctx_len - 1) % kBlockSize) {
+              if (lane == 0) atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG);
+            }
+            if (blk >= p.num_blocks) continue;
+            Group gr;
+            gr.n = 1; gr.blk = static_cast<int>(blk); gr.tok[0] = sg.b; gr.off[0] = static_cast<int>(slot % kBlockSize);
+            write_part<D, 1>(wp, gr, sg.g, which, write_stage + wq * (kBlockSize * D), lane);
+          }
+        }
+        // the granules are read next by the copy engine: order this warp's global (and staging) writes before it
+        asm volatile("fence.proxy.async;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_wdone);
+        COOPT_TRACE_CYCLES(p.trace, kTrWriteDone, t == 0);
+      }
       for (int si = 0; si < nseg; ++si) {
         const Segment sg = plan.segs[si];
         const bool more = si + 1 < nseg;
+        COOPT_TRACE_CYCLES(p.trace, kTrTeamSegBase + static_cast<int>(seg_no), tid == 0 && seg_no < 20);
         if (team == 0 && more) load_q(plan.segs[si + 1]);
 
         // the team's running softmax over its tiles of this segment
@@ -705,6 +810,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
               *reinterpret_cast<uint4*>(st + C::kKArea + nb * C::kPart + (t >> 3) * 128 + (t & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
             fence_proxy_async();
             mbar_arrive(&bar_pfull[buf]);
+            COOPT_TRACE_CYCLES(p.trace, kTrFirstProbs, tid == 0 && tile_no == 0);
           }
           // the product of the team's previous tile (its own buffers, so nothing above had to wait for it)
           if (pending) {
@@ -747,15 +853,23 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         ++seg_no;
       }
       if (old_open) flush_old();              // the round's last segment
+      COOPT_TRACE_CYCLES(p.trace, kTrTeamsDone, tid == 0);
       if (bad && t == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     }
 
     __syncthreads();
-    if (*abort_flag != 0) break;
+    if (*abort_flag != 0 || last_round) break;
     // roles that skipped their counters (idle lanes) are not using them; the others agree by construction
-    x = x_next;
-    __syncthreads();
+    plan_at += round_bytes;
+    ++round_no;
+    if (tid == 0) {
+      fence_proxy_async();                      // the round just read gives way to the next one
+      mbar_expect_tx(bar_plan, kPlanFirstChunk);
+      bulk_copy_g2s(plan_smem, plan_region + plan_at, kPlanFirstChunk, bar_plan);
+    }
   }
+  COOPT_TRACE_CYCLES(p.trace, kTrExit, tid == 0);
+  COOPT_TRACE_NS(p.trace, kTrExitNs, tid == 0);
 
   // ---- exit: copies still in flight get a bounded time to land, tensor memory is returned -----------
   if (*abort_flag != 0 && warp == kProducerWarp && lane == 0) {
@@ -769,26 +883,66 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   if (warp == kMmaWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(C::kTmemCols) : "memory");
 }
 
+// The copy engine's two views of a cache (parts, headers), encoded once per (cache, shape, device) and kept:
+// a serving loop launches on the same few caches over and over.
+struct CacheMaps {
+  const void* data;
+  long long granules;
+  int gran, part, dev;
+  CUtensorMap map_part, map_hdr;
+};
+bool cache_maps(const void* data, long long granules, int gran, int part, CUtensorMap* map_part, CUtensorMap* map_hdr) {
+  static std::mutex mu;
+  static std::vector<CacheMaps> known;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  for (const CacheMaps& m : known) {
+    if (m.data == data && m.granules == granules && m.gran == gran && m.part == part && m.dev == dev) {
+      *map_part = m.map_part; *map_hdr = m.map_hdr;
+      return true;
+    }
+  }
+  CacheMaps m;
+  m.data = data; m.granules = granules; m.gran = gran; m.part = part; m.dev = dev;
+  if (!encode_cache_map(&m.map_part, data, granules, gran, part / 8) || !encode_cache_map(&m.map_hdr, data, granules, gran, kFp8Header / 8))
+    return false;
+  if (known.size() >= 256) known.erase(known.begin());
+  known.push_back(m);
+  *map_part = m.map_part; *map_hdr = m.map_hdr;
+  return true;
+}
+
 template <int D, int NP>
-int launch_umma_one(const DecodeParams& p, int grid, cudaStream_t stream) {
+int launch_umma_one(DecodeParams p, int grid, bool overlap_previous, cudaStream_t stream) {
   using C = UCfg<D, NP>;
   CUtensorMap map_part, map_hdr;
   const long long granules = static_cast<long long>(p.num_blocks) * p.num_kv_heads;
-  if (!encode_cache_map(&map_part, p.cache, granules, C::kGran, C::kPart / 8) ||
-      !encode_cache_map(&map_hdr, p.cache, granules, C::kGran, kFp8Header / 8))
-    return COOPT_ERR_CUDA;
+  if (!cache_maps(p.cache, granules, C::kGran, C::kPart, &map_part, &map_hdr)) return COOPT_ERR_CUDA;
   if (!configure_kernel_smem(reinterpret_cast<const void*>(&paged_decode_umma_kernel<D, NP>), C::kSmemBytes)) return COOPT_ERR_CUDA;
-  paged_decode_umma_kernel<D, NP><<<grid, kUmmaThreads, C::kSmemBytes, stream>>>(p, map_part, map_hdr);
-  return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
+#ifdef COOPT_TRACE
+  p.trace = trace_buffer();
+#endif
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(grid));
+  cfg.blockDim = dim3(kUmmaThreads);
+  cfg.dynamicSmemBytes = C::kSmemBytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = overlap_previous ? 1 : 0;     // the kernel may then start while the one before it still runs
+  return cudaLaunchKernelEx(&cfg, paged_decode_umma_kernel<D, NP>, p, map_part, map_hdr) == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
 
 }  // namespace
 
 // FP8 cache: group sizes 1..5 use 16 probability rows, 6..8 use 32.
-int launch_paged_decode_umma(const DecodeParams& p, int head_dim, int grid, cudaStream_t stream) {
+int launch_paged_decode_umma(const DecodeParams& p, int head_dim, int grid, bool overlap_previous, cudaStream_t stream) {
   if (p.group <= 5)
-    return head_dim == 128 ? launch_umma_one<128, 16>(p, grid, stream) : launch_umma_one<64, 16>(p, grid, stream);
-  return head_dim == 128 ? launch_umma_one<128, 32>(p, grid, stream) : launch_umma_one<64, 32>(p, grid, stream);
+    return head_dim == 128 ? launch_umma_one<128, 16>(p, grid, overlap_previous, stream) : launch_umma_one<64, 16>(p, grid, overlap_previous, stream);
+  return head_dim == 128 ? launch_umma_one<128, 32>(p, grid, overlap_previous, stream) : launch_umma_one<64, 32>(p, grid, overlap_previous, stream);
 }
 
 }  // namespace coopt

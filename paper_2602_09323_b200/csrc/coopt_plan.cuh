@@ -33,8 +33,43 @@ struct Segment {
   int run_slot;      // workspace slot of the run's merged piece (two per CTA)
   int run_expected;  // number of CTAs that hold a run of this (sequence, kv head)
   int first_cta;     // the first of them
+  int pad[2];        // 64 bytes: segments are copied in 16-byte pieces
 };
 constexpr int kRunFirst = 1, kRunLast = 2, kRunWhole = 4;
+constexpr int kSegTail = 8;    // the segment ends with the last block of its sequence (where a new token lands)
+
+// A plan computed once (coopt_decode_plan) and read by every launch that shares its context lengths and
+// block table: per planned CTA a region of `cta_stride` bytes holding its rounds back to back, each round a
+// header, its segments and the staged physical block ids of those segments.
+struct PlanHeader {          // first 256 bytes of a plan
+  int magic, planned_ctas, batch, num_kv_heads;
+  int chunk_blocks, max_blocks_per_seq, cta_stride, status;
+  int num_blocks, max_chunks;
+  unsigned int empty_bits[kMaxBatch / 32];   // bit b: sequence b has no context (its output rows are zeros)
+  int pad[54 - kMaxBatch / 32];
+};
+struct PlanRound {           // 64 bytes in front of a round's segments
+  int nseg;                  // 0: the CTA has nothing (left) to do
+  int n_ids;
+  int bytes;                 // of the whole round record (header, segments, ids), a multiple of 16
+  int last;                  // 1: no round follows
+  int n_tail;                // segments that carry kSegTail
+  int key;                   // plan_key() of the problem the plan was made for
+  int status;                // a coopt_status the planner wants reported (a block id out of range, a plan that did not fit)
+  int pad[9];
+};
+// What a launch and the plan it is handed must agree on.
+__host__ __device__ inline int plan_key(int planned_ctas, int batch, int num_kv_heads, int chunk_blocks, int max_blocks_per_seq, int num_blocks) {
+  unsigned int h = 0x9e3779b9u;
+  const int v[6] = {planned_ctas, batch, num_kv_heads, chunk_blocks, max_blocks_per_seq, num_blocks};
+  for (int i = 0; i < 6; ++i) h = (h ^ static_cast<unsigned int>(v[i])) * 0x01000193u + 0x7f4a7c15u;
+  return static_cast<int>(h | 1u);
+}
+constexpr int kPlanMagic = 0x434f5031;
+constexpr int kPlanHeaderBytes = 256;
+constexpr int kPlanFirstChunk = 4096;   // what a CTA fetches of a round before it knows the round's size
+constexpr int kPlanRoundMax = 64 + kMaxSeg * 64 + kCap * 4;   // largest round record
+static_assert(sizeof(PlanHeader) == kPlanHeaderBytes && sizeof(PlanRound) == 64 && sizeof(Segment) == 64, "plan layout");
 
 struct DecodeParams {
   const uint8_t* cache;
@@ -43,6 +78,16 @@ struct DecodeParams {
   const int* block_table;
   const int* context_lens;
   const int* cu_q_lens;    // chunk mode: prefix sums of the query tokens per sequence (must be 0..batch); else null
+  const uint8_t* plan;     // FP8 kernel: the plan's CTA regions (behind the PlanHeader); cta_stride bytes each
+  int plan_cta_stride;
+  const PlanHeader* plan_header;
+  int plan_key;            // what every round header of the plan must carry
+  // fused append (all null / 0 when the call has no new tokens): Algorithm 1 phase 1 for one token per sequence
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  const long long* slot_mapping;
+  long long kv_token_stride;
+  unsigned long long* trace;   // time stamps (trace build only; null otherwise)
   int max_blocks_per_seq;
   int batch, num_q_heads, num_kv_heads, group;
   int num_blocks;
@@ -274,13 +319,13 @@ __device__ inline void plan_round_finish(const DecodeParams& p, const PlanSmem& 
       sg.run_expected = cta_l - cta_f + 1;
       sg.run_slot = 2 * blockIdx.x + (cta_f < static_cast<int>(blockIdx.x) ? 0 : 1);
       sg.run_flags = ((c == 0 || u == sl.ulo) ? kRunFirst : 0) | ((c == nch - 1 || u == sl.uhi - 1) ? kRunLast : 0) |
-                     (cta_l == cta_f ? kRunWhole : 0);
+                     (cta_l == cta_f ? kRunWhole : 0) | (sg.j0 + sg.n == nb ? kSegTail : 0);
     } else {
       sg.slot = 2 * blockIdx.x + (sg.j0 > 0 ? 0 : 1);
       const long long fs = static_cast<long long>(Hkv) * s.pre_blk[sg.b] + static_cast<long long>(sg.g) * nb;
       sg.first_cta = plan_cta_of(sl, fs);
       sg.expected = plan_cta_of(sl, fs + nb - 1) - sg.first_cta + 1;
-      sg.run_flags = kRunFirst | kRunLast | (sg.partial ? 0 : kRunWhole);
+      sg.run_flags = kRunFirst | kRunLast | (sg.partial ? 0 : kRunWhole) | (sg.j0 + sg.n == nb ? kSegTail : 0);
       sg.run_slot = sg.slot;
       sg.run_expected = sg.expected;
     }

@@ -1,0 +1,102 @@
+"""Where the time of one decode launch goes: ``python -m paper_2602_09323_b200.trace [--workload ...]``.
+
+Builds ``libcoopt_trace.so`` (the library's sources with ``-DCOOPT_TRACE``), runs the fused decode step of a
+workload a few times and prints, for the last launch, when each role of the tcgen05 kernel reached its
+milestones: per milestone the median, the earliest and the latest CTA, in microseconds from that CTA's own
+first instruction, and the span of the whole launch on the global timer.  The stamps cost a few stores per
+tile; the launch is a few per cent slower than in the ordinary library, so this is a breakdown, not a
+benchmark.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+
+import numpy as np
+import torch
+
+from . import binding, build, workloads
+
+SLOTS = 64
+MAX_CTAS = 1024
+NAMES = ["entry", "entry_ns", "setup_done", "plan_in_smem", "first_copy", "first_landed", "first_probs", "last_copy",
+         "last_landed", "last_pv", "teams_done", "last_hand_off", "piece_stored", "counted", "epilogue_done", "exit",
+         "exit_ns", "write_done", "num_seg", "num_tiles"]
+SEG_BASE, TEAM_SEG_BASE = 24, 44
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--workload", default="llama13b_decode", choices=["llama13b_decode", "mixed_serving", "long_context"])
+    ap.add_argument("--no-append", action="store_true", help="attention only (no new token written in the launch)")
+    ap.add_argument("--launches", type=int, default=12)
+    ap.add_argument("--sm-mhz", type=float, default=1965.0, help="SM clock used to turn cycles into microseconds")
+    args = ap.parse_args()
+    binding.use_library(build.build(trace=True))
+    lib = binding.load_library()
+    lib.coopt_trace_set_buffer.restype, lib.coopt_trace_set_buffer.argtypes = ctypes.c_int, [ctypes.c_void_p, ctypes.c_size_t]
+    torch.cuda.set_device(0)
+    chunk = 0
+    if args.workload == "llama13b_decode":
+        w = workloads.config_llama13b_decode()
+    elif args.workload == "mixed_serving":
+        w = workloads.config_mixed_serving()
+    else:
+        w, chunk = workloads.config_long_context(), 2048
+    B, Hq, Hkv, D = w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim
+    k, v, slots = w.k.cuda(), w.v.cuda(), w.slot_mapping.cuda()
+    last = torch.tensor([w.kv_offsets[b] + L - 1 for b, L in enumerate(w.context_lens)])
+    hist = torch.ones(k.shape[0], dtype=torch.bool)
+    hist[last] = False
+    hist_idx, new_idx = hist.nonzero().squeeze(1).cuda(), last.cuda()
+    k_new, v_new, s_new = k[new_idx].contiguous(), v[new_idx].contiguous(), slots[new_idx].contiguous()
+    caches = []
+    for _ in range(2):                      # two caches visited in turn: more than L2 between two visits of one
+        c = binding.Cache(w.num_blocks, Hkv, D)
+        binding.kv_write(c, k[hist_idx], v[hist_idx], slots[hist_idx])
+        caches.append(c)
+    table, lens, q = w.block_table.clamp(min=0).cuda(), w.context_lens_tensor.cuda(), w.q.cuda()
+    plan = binding.decode_plan(table, lens, Hkv, w.num_blocks, chunk)
+    ws = binding.new_workspace(B, Hq, Hkv, D, table.shape[1], chunk, B)
+    buf = torch.zeros(MAX_CTAS * SLOTS, dtype=torch.int64, device="cuda")
+    assert lib.coopt_trace_set_buffer(ctypes.c_void_p(buf.data_ptr()), buf.numel() * 8) == 0
+    out = torch.empty_like(q)
+    for i in range(args.launches):
+        buf.zero_()
+        if args.no_append:
+            binding.decode_step_planned(caches[i % 2], plan, q, table.shape[1], w.sm_scale, ws, chunk_size=chunk, out=out)
+        else:
+            binding.decode_step_planned(caches[i % 2], plan, q, table.shape[1], w.sm_scale, ws, k_new, v_new, s_new,
+                                        chunk_size=chunk, out=out)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    t = buf.cpu().numpy().reshape(MAX_CTAS, SLOTS)
+    t = t[t[:, 0] != 0]
+    us = 1.0 / args.sm_mhz
+    print(f"workload {args.workload}{' (no append)' if args.no_append else ''}: {t.shape[0]} CTAs, "
+          f"segments per CTA median {np.median(t[:, 18]):.0f} max {t[:, 18].max()}, tiles per CTA median {np.median(t[:, 19]):.0f} "
+          f"max {t[:, 19].max()}")
+    span = (t[:, 16].max() - t[:, 1].min()) / 1e3
+    print(f"launch span on the global timer: {span:.1f} us (first entry to last exit); entries spread over "
+          f"{(t[:, 1].max() - t[:, 1].min()) / 1e3:.1f} us, exits over {(t[:, 16].max() - t[:, 16].min()) / 1e3:.1f} us")
+    print(f"{'milestone':<16}{'median':>9}{'earliest':>10}{'latest':>9}   (us after the CTA's first instruction, {args.sm_mhz:.0f} MHz)")
+    for i, name in enumerate(NAMES):
+        if name in ("entry", "entry_ns", "exit_ns", "num_seg", "num_tiles"):
+            continue
+        col = t[:, i]
+        ok = col != 0
+        if not ok.any():
+            continue
+        rel = (col[ok] - t[ok, 0]) * us
+        print(f"{name:<16}{np.median(rel):9.2f}{rel.min():10.2f}{rel.max():9.2f}   ({int(ok.sum())} CTAs)")
+    for base, label in ((TEAM_SEG_BASE, "team 0 begins segment"), (SEG_BASE, "epilogue gets segment")):
+        for i in range(6):
+            col = t[:, base + i]
+            ok = col != 0
+            if ok.any():
+                rel = (col[ok] - t[ok, 0]) * us
+                print(f"{label + ' ' + str(i):<26}{np.median(rel):9.2f}{rel.min():10.2f}{rel.max():9.2f}   ({int(ok.sum())} CTAs)")
+
+
+if __name__ == "__main__":
+    main()
