@@ -104,7 +104,7 @@ int coopt_kv_write(const coopt_cache* cache, const void* k, const void* v, int64
  * (Eq. 1; Eq. 6 dequantisation on load; Eq. 7-8 grouped-query sharing: query head i reads
  * kv head floor(i / (num_q_heads / num_kv_heads)); Eq. 9: only blocks 0..ceil(len/16)-1 of a
  * sequence are read and the last one is masked past len; Eq. 10 max-subtracted softmax).
- *   q, out        DEVICE bf16 [batch][num_q_heads][head_dim], contiguous
+ *   q, out        DEVICE bf16 [batch][num_q_heads][head_dim], contiguous, 16-byte aligned
  *   block_table   DEVICE int32 [batch][max_blocks_per_seq]; entry j of row b is the physical
  *                 block of tokens 16j..16j+15 of sequence b; entries past the context are
  *                 never read
@@ -268,27 +268,33 @@ int coopt_decode_layers(const coopt_layer_io* layers, int32_t num_layers, int64_
                         uint32_t flags, void* stream);
 
 /*
- * coopt_decode_step_host — one serving step for callers whose step inputs live in HOST memory
- * (Section 2's token-insertion phase followed by the attention phase): copies the step's
- * inputs to the device, runs coopt_kv_write for the one new token of every sequence and
- * coopt_paged_decode over the updated cache, and copies the bf16 result back.  Everything is
- * enqueued on `stream`; the host buffers must stay valid (and should be pinned) until the
- * stream has been synchronised.  The cache and both scratch areas are DEVICE memory.
- *   q_host, out_host      HOST bf16 [batch][num_q_heads][head_dim]
- *   k_host, v_host        HOST bf16 [batch][num_kv_heads][head_dim] (the new token of each sequence)
- *   slot_mapping_host     HOST int64 [batch]
- *   block_table_host      HOST int32 [batch][max_blocks_per_seq]
- *   context_lens_host     HOST int32 [batch], counting the new token
- *   staging               DEVICE, >= coopt_step_staging_bytes(...) bytes, 256-byte aligned
- * Errors: as coopt_kv_write and coopt_paged_decode, WORKSPACE if staging is too small.
+ * coopt_decode_step_host -- one serving step for callers whose step inputs live in HOST memory (Section 2's
+ * token-insertion phase followed by the attention phase): ONE copy brings the step's inputs to the device,
+ * coopt_decode_plan and coopt_decode_step_planned run on them, ONE copy takes the bf16 result back.
+ * Everything is enqueued on `stream`; the host buffers must stay valid (and should be pinned) until the
+ * stream has been synchronised.
+ *   step_inputs_host   HOST, coopt_step_layout.in_bytes bytes: the step's inputs packed at the offsets that
+ *                      coopt_step_staging_layout() gives -- q bf16 [batch][num_q_heads][head_dim]; k_new,
+ *                      v_new bf16 [batch][num_kv_heads][head_dim]; slot_mapping int64 [batch]; block_table
+ *                      int32 [batch][max_blocks_per_seq]; context_lens int32 [batch], counting the new token
+ *   out_host           HOST bf16 [batch][num_q_heads][head_dim]
+ *   staging            DEVICE, >= coopt_step_layout.total_bytes, 256-byte aligned
+ *   plan, workspace    DEVICE, sized by coopt_plan_bytes / coopt_workspace_bytes (chunk_size 0)
+ * The new token of every sequence must be its last position (see coopt_decode_step_planned).
+ * Errors: as coopt_decode_plan and coopt_decode_step_planned; WORKSPACE if staging is too small.
  */
-int coopt_decode_step_host(const coopt_cache* cache, const void* q_host, const void* k_host, const void* v_host,
-                           const int64_t* slot_mapping_host, const int32_t* block_table_host,
-                           int32_t max_blocks_per_seq, const int32_t* context_lens_host, void* out_host,
-                           int32_t batch, int32_t num_q_heads, float sm_scale, void* staging, size_t staging_bytes,
-                           void* workspace, size_t workspace_bytes, void* stream);
-size_t coopt_step_staging_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
-                                int32_t max_blocks_per_seq);
+typedef struct coopt_step_layout {
+  size_t q, k_new, v_new, slot_mapping, block_table, context_lens;   /* byte offsets of the inputs */
+  size_t in_bytes;       /* bytes of the packed inputs = what is copied to the device */
+  size_t out;            /* byte offset of the result inside the device staging area */
+  size_t out_bytes;      /* bytes copied back */
+  size_t total_bytes;    /* bytes of the device staging area */
+} coopt_step_layout;
+int coopt_step_staging_layout(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                              int32_t max_blocks_per_seq, coopt_step_layout* layout);
+int coopt_decode_step_host(const coopt_cache* cache, const void* step_inputs_host, void* out_host, int32_t max_blocks_per_seq,
+                           int32_t batch, int32_t num_q_heads, float sm_scale, void* staging, size_t staging_bytes, void* plan,
+                           size_t plan_bytes, void* workspace, size_t workspace_bytes, void* stream);
 
 /* Workspace size for a call with these arguments (chunk_size = 0 for coopt_paged_decode).
  * Host arithmetic only (it asks the current device for its SM count once). */

@@ -32,6 +32,11 @@ class coopt_cache(ctypes.Structure):
                 ("head_dim", ctypes.c_int32), ("block_size", ctypes.c_int32), ("dtype", ctypes.c_int32)]
 
 
+class coopt_step_layout(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_size_t) for n in ("q", "k_new", "v_new", "slot_mapping", "block_table", "context_lens",
+                                               "in_bytes", "out", "out_bytes", "total_bytes")]
+
+
 class coopt_layer_io(ctypes.Structure):
     _fields_ = [("cache", ctypes.POINTER(coopt_cache)), ("k_new", ctypes.c_void_p), ("v_new", ctypes.c_void_p),
                 ("slot_mapping", ctypes.c_void_p), ("q", ctypes.c_void_p), ("out", ctypes.c_void_p)]
@@ -62,15 +67,14 @@ _SIGNATURES = {
     "coopt_workspace_init": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
     "coopt_chunk_partials": (ctypes.c_int, [ctypes.c_int32] * 5 + [ctypes.POINTER(ctypes.c_size_t)] * 3
                              + [ctypes.POINTER(ctypes.c_int32)]),
-    "coopt_decode_step_host": (ctypes.c_int, [ctypes.POINTER(coopt_cache)] + [ctypes.c_void_p] * 5 + [ctypes.c_int32]
-                               + [ctypes.c_void_p] * 2 + [ctypes.c_int32, ctypes.c_int32, ctypes.c_float,
-                                                          ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p,
-                                                          ctypes.c_size_t, ctypes.c_void_p]),
+    "coopt_decode_step_host": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
+                                              ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_void_p, ctypes.c_size_t,
+                                              ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
+    "coopt_step_staging_layout": (ctypes.c_int, [ctypes.c_int32] * 5 + [ctypes.c_void_p]),
     "coopt_decode_step": (ctypes.c_int, [ctypes.POINTER(coopt_cache), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64,
                                          ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int32,
                                          ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_float, ctypes.c_void_p,
                                          ctypes.c_size_t, ctypes.c_void_p]),
-    "coopt_step_staging_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 5),
     "coopt_plan_bytes": (ctypes.c_size_t, [ctypes.c_int32] * 4),
     "coopt_decode_plan": (ctypes.c_int, [ctypes.c_void_p, ctypes.c_int32, ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32,
                                          ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]),
@@ -347,18 +351,19 @@ def selftest_bounded_wait(limit_ns: int):
     return int(res[0].item()), int(res[1].item())
 
 
-def step_staging_bytes(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, max_blocks_per_seq: int) -> int:
-    return load_library().coopt_step_staging_bytes(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq)
+def step_staging_layout(batch: int, num_q_heads: int, num_kv_heads: int, head_dim: int, max_blocks_per_seq: int) -> coopt_step_layout:
+    lay = coopt_step_layout()
+    _check(load_library().coopt_step_staging_layout(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq,
+                                                    ctypes.byref(lay)), "coopt_step_staging_layout")
+    return lay
 
 
-def decode_step_host(cache: Cache, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, slot_mapping: torch.Tensor,
-                     block_table: torch.Tensor, context_lens: torch.Tensor, out: torch.Tensor, sm_scale: float,
-                     staging: torch.Tensor, workspace: torch.Tensor) -> None:
-    """coopt_decode_step_host: all step inputs and ``out`` are HOST (pinned) tensors; asynchronous."""
-    for t in (q, k, v, slot_mapping, block_table, context_lens, out):
-        assert not t.is_cuda and t.is_contiguous()
-    st = load_library().coopt_decode_step_host(cache.ref(), _ptr(q), _ptr(k), _ptr(v), _ptr(slot_mapping),
-                                               _ptr(block_table), block_table.shape[1], _ptr(context_lens), _ptr(out),
-                                               q.shape[0], q.shape[1], float(sm_scale), _ptr(staging), staging.numel(),
-                                               _ptr(workspace), workspace.numel(), _stream())
+def decode_step_host(cache: Cache, step_inputs: torch.Tensor, out: torch.Tensor, max_blocks_per_seq: int, num_q_heads: int,
+                     sm_scale: float, staging: torch.Tensor, plan: torch.Tensor, workspace: torch.Tensor) -> None:
+    """coopt_decode_step_host: ``step_inputs`` (uint8, packed per step_staging_layout) and ``out`` are HOST (pinned)
+    tensors; asynchronous."""
+    assert not step_inputs.is_cuda and step_inputs.is_contiguous() and not out.is_cuda and out.is_contiguous()
+    st = load_library().coopt_decode_step_host(cache.ref(), _ptr(step_inputs), _ptr(out), max_blocks_per_seq, out.shape[0],
+                                               num_q_heads, float(sm_scale), _ptr(staging), staging.numel(), _ptr(plan),
+                                               plan.numel(), _ptr(workspace), workspace.numel(), _stream())
     _check(st, "coopt_decode_step_host")

@@ -108,6 +108,7 @@ int check_attention_shapes(const coopt_cache* c, const void* q, void* out, int32
   const int rc = check_cache(c);
   if (rc != COOPT_OK) return rc;
   if (!q || !out || batch < 0 || max_blocks_per_seq <= 0 || num_q_heads <= 0) return COOPT_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(q) | reinterpret_cast<uintptr_t>(out)) % 16 != 0) return COOPT_ERR_INVALID_ARG;   // rows move in 16-byte pieces
   if (num_q_heads % c->num_kv_heads != 0) return COOPT_ERR_UNSUPPORTED;
   const int group = num_q_heads / c->num_kv_heads;
   if (group < 1 || group > 8) return COOPT_ERR_UNSUPPORTED;
@@ -338,63 +339,63 @@ int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, cons
 }
 
 namespace {
-struct StepStaging {
-  size_t q, out, k, v, slots, table, lens, total;
-};
-StepStaging step_staging(int batch, int hq, int hkv, int d, int max_blocks) {
+coopt_step_layout step_layout(int batch, int hq, int hkv, int d, int max_blocks) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-  StepStaging s;
+  coopt_step_layout s;
   size_t at = 0;
-  s.q = at;     at += up(static_cast<size_t>(batch) * hq * d * 2);
-  s.out = at;   at += up(static_cast<size_t>(batch) * hq * d * 2);
-  s.k = at;     at += up(static_cast<size_t>(batch) * hkv * d * 2);
-  s.v = at;     at += up(static_cast<size_t>(batch) * hkv * d * 2);
-  s.slots = at; at += up(static_cast<size_t>(batch) * 8);
-  s.table = at; at += up(static_cast<size_t>(batch) * max_blocks * 4);
-  s.lens = at;  at += up(static_cast<size_t>(batch) * 4);
-  s.total = at;
+  s.q = at;            at += up(static_cast<size_t>(batch) * hq * d * 2);
+  s.k_new = at;        at += up(static_cast<size_t>(batch) * hkv * d * 2);
+  s.v_new = at;        at += up(static_cast<size_t>(batch) * hkv * d * 2);
+  s.slot_mapping = at; at += up(static_cast<size_t>(batch) * 8);
+  s.block_table = at;  at += up(static_cast<size_t>(batch) * max_blocks * 4);
+  s.context_lens = at; at += up(static_cast<size_t>(batch) * 4);
+  s.in_bytes = at;
+  s.out = at;          at += up(static_cast<size_t>(batch) * hq * d * 2);
+  s.out_bytes = static_cast<size_t>(batch) * hq * d * 2;
+  s.total_bytes = at;
   return s;
 }
 }  // namespace
 
-size_t coopt_step_staging_bytes(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
-                                int32_t max_blocks_per_seq) {
-  if (batch < 0 || num_q_heads <= 0 || num_kv_heads <= 0 || head_dim <= 0 || max_blocks_per_seq <= 0) return 0;
-  return step_staging(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq).total;
+int coopt_step_staging_layout(int32_t batch, int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                              int32_t max_blocks_per_seq, coopt_step_layout* layout) {
+  if (batch < 0 || num_q_heads <= 0 || num_kv_heads <= 0 || head_dim <= 0 || max_blocks_per_seq <= 0 || !layout) return COOPT_ERR_INVALID_ARG;
+  *layout = step_layout(batch, num_q_heads, num_kv_heads, head_dim, max_blocks_per_seq);
+  return COOPT_OK;
 }
 
-int coopt_decode_step_host(const coopt_cache* cache, const void* q_host, const void* k_host, const void* v_host,
-                           const int64_t* slot_mapping_host, const int32_t* block_table_host,
-                           int32_t max_blocks_per_seq, const int32_t* context_lens_host, void* out_host,
-                           int32_t batch, int32_t num_q_heads, float sm_scale, void* staging, size_t staging_bytes,
-                           void* workspace, size_t workspace_bytes, void* stream) {
+int coopt_decode_step_host(const coopt_cache* cache, const void* step_inputs_host, void* out_host, int32_t max_blocks_per_seq,
+                           int32_t batch, int32_t num_q_heads, float sm_scale, void* staging, size_t staging_bytes, void* plan,
+                           size_t plan_bytes_given, void* workspace, size_t workspace_bytes, void* stream) {
   int rc = check_cache(cache);
   if (rc != COOPT_OK) return rc;
-  if (!q_host || !k_host || !v_host || !slot_mapping_host || !block_table_host || !context_lens_host || !out_host ||
-      batch < 0 || num_q_heads <= 0 || max_blocks_per_seq <= 0)
-    return COOPT_ERR_INVALID_ARG;
+  if (!step_inputs_host || !out_host || batch < 0 || num_q_heads <= 0 || max_blocks_per_seq <= 0) return COOPT_ERR_INVALID_ARG;
   if (batch == 0) return COOPT_OK;
   const int hkv = cache->num_kv_heads, d = cache->head_dim;
-  const StepStaging s = step_staging(batch, num_q_heads, hkv, d, max_blocks_per_seq);
-  if (!staging || staging_bytes < s.total) return COOPT_ERR_WORKSPACE;
+  const coopt_step_layout s = step_layout(batch, num_q_heads, hkv, d, max_blocks_per_seq);
+  if (!staging || staging_bytes < s.total_bytes) return COOPT_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(staging) % 256 != 0) return COOPT_ERR_INVALID_ARG;
   uint8_t* dev = static_cast<uint8_t*>(staging);
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const size_t qb = static_cast<size_t>(batch) * num_q_heads * d * 2, kb = static_cast<size_t>(batch) * hkv * d * 2;
-  bool ok = true;
-  ok &= cudaMemcpyAsync(dev + s.q, q_host, qb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(dev + s.k, k_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(dev + s.v, v_host, kb, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(dev + s.slots, slot_mapping_host, static_cast<size_t>(batch) * 8, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(dev + s.table, block_table_host, static_cast<size_t>(batch) * max_blocks_per_seq * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  ok &= cudaMemcpyAsync(dev + s.lens, context_lens_host, static_cast<size_t>(batch) * 4, cudaMemcpyHostToDevice, st) == cudaSuccess;
-  if (!ok) return COOPT_ERR_CUDA;
-  rc = coopt_decode_step(cache, dev + s.k, dev + s.v, static_cast<int64_t>(hkv) * d, reinterpret_cast<const int64_t*>(dev + s.slots),
-                         dev + s.q, dev + s.out, reinterpret_cast<const int32_t*>(dev + s.table), max_blocks_per_seq,
-                         reinterpret_cast<const int32_t*>(dev + s.lens), batch, num_q_heads, sm_scale, workspace,
-                         workspace_bytes, stream);
+  // every check of the device part before the first copy is enqueued
+  rc = check_attention_args(cache, dev + s.q, dev + s.out, reinterpret_cast<const int32_t*>(dev + s.block_table), max_blocks_per_seq,
+                            reinterpret_cast<const int32_t*>(dev + s.context_lens), batch, num_q_heads);
   if (rc != COOPT_OK) return rc;
-  return cudaMemcpyAsync(out_host, dev + s.out, qb, cudaMemcpyDeviceToHost, st) == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
+  if (cache->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;
+  rc = check_plan_args(batch, hkv, max_blocks_per_seq, 0, plan, plan_bytes_given);
+  if (rc != COOPT_OK) return rc;
+  if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, hkv, d, max_blocks_per_seq, 0, batch)) return COOPT_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // one copy in, the plan and the fused step, one copy out
+  if (cudaMemcpyAsync(dev, step_inputs_host, s.in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return COOPT_ERR_CUDA;
+  const int P = planned_ctas(batch, hkv, max_blocks_per_seq);
+  rc = launch_decode_plan(reinterpret_cast<const int32_t*>(dev + s.block_table), max_blocks_per_seq,
+                          reinterpret_cast<const int32_t*>(dev + s.context_lens), batch, hkv, cache->num_blocks, 0, P, plan, st);
+  if (rc != COOPT_OK) return rc;
+  rc = launch_decode_planned(cache, plan, dev + s.k_new, dev + s.v_new, static_cast<int64_t>(hkv) * d,
+                             reinterpret_cast<const int64_t*>(dev + s.slot_mapping), dev + s.q, dev + s.out, max_blocks_per_seq, batch,
+                             num_q_heads, sm_scale, 0, nullptr, workspace, P, false, st);
+  if (rc != COOPT_OK) return rc;
+  return cudaMemcpyAsync(out_host, dev + s.out, s.out_bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
 
 const char* coopt_status_string(int status) {

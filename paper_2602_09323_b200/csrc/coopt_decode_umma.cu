@@ -77,6 +77,7 @@ struct UCfg {
   static constexpr int kStageBytes = kHdrOff + kTileBlocks * kFp8Header;
   static constexpr int kGroupBytes = kGatherRows * (2 * kPart + kFp8Header);   // what the three requests of four granules bring
   static constexpr int kQBytes = 2 * 8 * D;                    // 16 rows x D codes
+  static constexpr int kQRawBytes = kGMax * D * 2;             // the bf16 query rows of one (sequence, kv head) as they sit in memory
   static constexpr int kPBytes = NP * kTileTokens;             // NP rows x 128 codes
   static constexpr int kXchFloats = kGMax * kTeamThreads;            // one team's output of a segment: [head][dim]
   static constexpr int kMlFloats = 4 * 8 + 8;                       // one team's sums (per warp) and maxima of a segment
@@ -85,13 +86,14 @@ struct UCfg {
   static constexpr int kQOff = kRingOff + kStages * kStageBytes;
   static constexpr int kPOff = kQOff + 2 * kQBytes;
   static constexpr int kPlanOff = kPOff + 4 * kPBytes;             // one round of the plan: header, segments, block ids
-  static constexpr int kXchOff = kPlanOff + (kPlanRoundMax + 127) / 128 * 128;
+  static constexpr int kQRawOff = kPlanOff + (kPlanRoundMax + 127) / 128 * 128;   // two segments' raw queries
+  static constexpr int kXchOff = kQRawOff + 2 * kQRawBytes;
   static constexpr int kMlOff = kXchOff + 2 * kXchFloats * 4;       // [2 segment parities][2 teams][kMlFloats]
   static constexpr int kRedOff = kMlOff + 2 * 2 * kMlFloats * 4;
   // int red_max [2 teams][4 warps][12], uint red_q [4][8], float qscale [2][8]
   static constexpr int kRedBytes = (2 * 4 * 12 + 4 * 8 + 2 * 8) * 4;
   static constexpr int kBarOff = kRedOff + kRedBytes;
-  static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2 + 2;
+  static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2 + 2 + 2;
   static constexpr int kWriteStage = 4 * kBlockSize * D;       // staging of team 1's four warps for the fused append
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kSmemBytes = kMiscOff + 128;            // 64 bytes of planner words and flags, 64 of the published slice
@@ -190,6 +192,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   uint64_t* bar_efree = bar_efull + 2;              // [2] the epilogue warp has read them
   uint64_t* bar_plan = bar_efree + 2;               // a piece of the plan has landed in shared memory
   uint64_t* bar_wdone = bar_plan + 1;               // team 1 has written the round's new tokens to the cache
+  uint64_t* bar_qraw = bar_wdone + 1;               // [2] the raw query rows of a segment have landed (buffer = segment & 1)
+  uint8_t* qraw = smem + C::kQRawOff;
   volatile int* abort_flag = plan.misc + 4;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(plan.misc + 5);
 
@@ -202,6 +206,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   // engine's view of the cache (fetched on first use otherwise, in front of the first tile)
   COOPT_TRACE_CYCLES(p.trace, kTrEntry, tid == 0);
   COOPT_TRACE_NS(p.trace, kTrEntryNs, tid == 0);
+#ifdef COOPT_TRACE
+  if (tid == 0) { unsigned int smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); trace_put(p.trace, kTrSmId, smid + 1); }
+#endif
   const uint8_t* plan_region = p.plan + static_cast<size_t>(blockIdx.x) * p.plan_cta_stride;
   if (tid == kProducerWarp * 32) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_part) : "memory");
@@ -221,6 +228,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
     for (int i = 0; i < 2; ++i) { mbar_init(&bar_qfull[i], kTeamThreads); mbar_init(&bar_efull[i], kSmThreads); mbar_init(&bar_efree[i], 1); }
     mbar_init(bar_plan, 1);
     mbar_init(bar_wdone, 4);
+    mbar_init(&bar_qraw[0], 1);
+    mbar_init(&bar_qraw[1], 1);
     mbar_fence_init();
     *abort_flag = 0;
     // the first round of this CTA's plan: its size is not known yet, so a fixed first piece is fetched
@@ -243,15 +252,6 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   if (warp != kProducerWarp) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   plan_check_single_query(p, tid, kUmmaThreads);
-  // sequences with an empty context: all-zero output rows (the epilogue warp has nothing else to do yet)
-  if (warp == kEpilogueWarp) {
-    for (int b = blockIdx.x; b < B; b += gridDim.x) {
-      if ((p.plan_header->empty_bits[b >> 5] >> (b & 31)) & 1u) {
-        uint4* row = reinterpret_cast<uint4*>(p.out + static_cast<size_t>(b) * Hq * D);
-        for (int i = lane; i < Hq * D / 8; i += 32) row[i] = make_uint4(0u, 0u, 0u, 0u);
-      }
-    }
-  }
   COOPT_TRACE_CYCLES(p.trace, kTrSetupDone, tid == 0);
   const uint32_t tmem_o = tmem + 64;                           // logits buffer b at column 16 b, output buffer b at 64 + NP b
   const uint32_t lane_base = static_cast<uint32_t>(warp & 3) * 32u << 16;
@@ -276,19 +276,29 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       plan_ok = wait_bar(bar_plan, plan_phase & 1u, abort_flag);
       ++plan_phase;
     }
-    plan_ok = __syncthreads_and(plan_ok);       // one verdict for the whole CTA
-    if (!plan_ok) {
-      if (tid == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+    // A wait that ran out has raised the abort flag: this thread skips the round's work (nseg = 0 below) but
+    // keeps the CTA's barriers company, and everybody leaves behind the round's closing barrier.
+    if (!plan_ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
+    const bool plan_valid = plan_ok && round_hdr->key == p.plan_key && round_hdr->nseg <= kMaxSeg && round_bytes <= kPlanRoundMax &&
+                            round_hdr->n_ids <= kCap;
+    if (plan_ok && !plan_valid) {                                                // not a plan of this problem (the same verdict in every thread)
+      if (tid == 0) atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG);
       break;
     }
-    const int nseg = round_hdr->nseg;
-    if (round_hdr->key != p.plan_key || nseg > kMaxSeg || round_bytes > kPlanRoundMax || round_hdr->n_ids > kCap) {
-      if (tid == 0) atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG);              // not a plan of this problem
-      break;
+    if (plan_ok && tid == 0 && round_hdr->status != 0) atomicCAS(p.status, 0, round_hdr->status);   // what the planner found
+    const int nseg = plan_ok ? round_hdr->nseg : 0;
+    if (warp == kEpilogueWarp && round_no == 0 && plan_ok) {
+      // sequences with an empty context: all-zero output rows (this warp has nothing else to do yet, and no
+      // other role waits for it here)
+      for (int b = blockIdx.x; b < B; b += gridDim.x) {
+        if ((p.plan_header->empty_bits[b >> 5] >> (b & 31)) & 1u) {
+          uint4* row = reinterpret_cast<uint4*>(p.out + static_cast<size_t>(b) * Hq * D);
+          for (int i = lane; i < Hq * D / 8; i += 32) row[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
     }
-    if (tid == 0 && round_hdr->status != 0) atomicCAS(p.status, 0, round_hdr->status);   // what the planner found
-    if (nseg <= 0) break;                                                        // nothing (left) to do
-    const bool last_round = round_hdr->last != 0;
+    if (plan_ok && nseg <= 0) break;                                             // nothing (left) to do
+    const bool last_round = !plan_ok || round_hdr->last != 0;
     plan.ids = reinterpret_cast<int*>(plan_smem + 64 + nseg * 64);
     const uint32_t round_tile0 = tile_no;             // every role's tile counter agrees at the start of a round
     uint8_t* write_stage = ring + ((round_tile0 + C::kStages - 1) % C::kStages) * C::kStageBytes;   // the stage the ring fills last
@@ -344,6 +354,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           if (lane < 3 * ngroups) gather4_g2s(st + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[stage]);
           COOPT_TRACE_CYCLES(p.trace, kTrFirstCopy, lane == 0 && tile_no == 0);
           COOPT_TRACE_CYCLES(p.trace, kTrLastCopy, lane == 0);
+          COOPT_TRACE_CYCLES(p.trace, kTrCopyTileBase + static_cast<int>(tile_no), lane == 0 && tile_no < 32);
           ++tile_no;
         }
       }
@@ -373,6 +384,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
 #pragma unroll
             for (int ks = 0; ks < kKSteps; ++ks) umma_f8(tmem + 16 * buf, dk + ks * 16, dq + ks * 16, umma_idesc(16), ks > 0);
             umma_commit(&bar_sfull[buf]);
+            COOPT_TRACE_CYCLES(p.trace, kTrLogitsTileBase + static_cast<int>(tile_no), tile_no < 32);
           }
         }
         if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
@@ -396,6 +408,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
               umma_f8(tmem_o + NP * buf, dv + ks * ((2 * C::kPart) >> 4), dp + ks * 16, umma_idesc(NP), ks > 0 ? 1u : 0u);
             umma_commit(&bar_empty[stage]);     // the stage is free again and the tile's product is in its output buffer
             COOPT_TRACE_CYCLES(p.trace, kTrLastPv, true);
+            COOPT_TRACE_CYCLES(p.trace, kTrPvTileBase + static_cast<int>(tile_no), tile_no < 32);
           }
         }
         if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
@@ -553,17 +566,26 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       int* my_red_max = red_max + team * 48;
 
       // query operand of a segment (team 0): E4M3 lead term in rows 0..7, remainder term in rows 8..15.
-      // The global loads are started a segment ahead (load_q) and consumed after a tile (publish_q).
-      float xq[kGMax];
-      auto load_q = [&](const Segment& sg) {
-#pragma unroll
-        for (int h = 0; h < kGMax; ++h) {
-          xq[h] = 0.0f;
-          if (h < G && t < D) xq[h] = __bfloat162float(p.q[(static_cast<size_t>(sg.b) * Hq + sg.g * G + h) * D + t]);
-        }
+      // The bf16 rows are brought into shared memory by a small bulk copy two segments ahead (fetch_q, one
+      // thread), so that no thread of the team ever waits on a load from a memory system that the cache stream
+      // keeps saturated; publish_q turns them into the operand behind the team's first tile of the segment before.
+      auto fetch_q = [&](const Segment& sg, uint32_t segc) {
+        const uint32_t bytes = static_cast<uint32_t>(G) * D * 2;
+        fence_proxy_async();
+        mbar_expect_tx(&bar_qraw[segc & 1u], bytes);
+        bulk_copy_g2s(qraw + (segc & 1u) * C::kQRawBytes, p.q + (static_cast<size_t>(sg.b) * Hq + sg.g * G) * D, bytes, &bar_qraw[segc & 1u]);
       };
-      auto publish_q = [&](uint32_t segc) {
+      float xq[kGMax];
+      auto publish_q = [&](uint32_t segc, int si_next2) {
         uint8_t* qb = qbuf + (segc & 1u) * C::kQBytes;
+        {
+          bool ok = !bad && wait_bar(&bar_qraw[segc & 1u], (segc >> 1) & 1u, abort_flag);
+          ok = __all_sync(0xffffffffu, ok);
+          bad = bad || !ok;
+          const __nv_bfloat16* raw = reinterpret_cast<const __nv_bfloat16*>(qraw + (segc & 1u) * C::kQRawBytes);
+#pragma unroll
+          for (int h = 0; h < kGMax; ++h) xq[h] = (!bad && h < G && t < D) ? __bfloat162float(raw[h * D + t]) : 0.0f;
+        }
 #pragma unroll
         for (int h = 0; h < kGMax; ++h) {
           const uint32_t am = __reduce_max_sync(0xffffffffu, __float_as_uint(fabsf(xq[h])));   // non-negative floats order like their bits
@@ -600,6 +622,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         bad = barrier_or(team_bar, kTeamThreads, bad);   // every thread has read the exchange words before the next query reuses them
         fence_proxy_async();
         mbar_arrive(&bar_qfull[segc & 1u]);
+        // the raw buffer is free again: the rows of the segment two further on take its place
+        if (t == 0 && si_next2 < nseg) fetch_q(plan.segs[si_next2], segc + 2);
       };
 
       // The piece of the segment before: its last product is folded in, and the piece handed to the
@@ -640,7 +664,13 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         mbar_arrive(&bar_efull[old_seg & 1u]);
       };
 
-      if (team == 0 && nseg > 0) { load_q(plan.segs[0]); publish_q(seg_no); }
+      if (team == 0 && nseg > 0) {
+        if (t == 0) {
+          fetch_q(plan.segs[0], seg_no);
+          if (nseg > 1) fetch_q(plan.segs[1], seg_no + 1);
+        }
+        publish_q(seg_no, 2);
+      }
       if (team == 1 && has_new) {
         // ---- Algorithm 1 phase 1 inside the step: the new token of every (sequence, kv head) whose last block
         // lies in this round.  Warp wq takes (tail segment, K | V) pairs wq, wq + 4, ..; the scale rule is the
@@ -680,7 +710,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
         const Segment sg = plan.segs[si];
         const bool more = si + 1 < nseg;
         COOPT_TRACE_CYCLES(p.trace, kTrTeamSegBase + static_cast<int>(seg_no), tid == 0 && seg_no < 20);
-        if (team == 0 && more) load_q(plan.segs[si + 1]);
+        COOPT_TRACE_VALUE(p.trace, kTrSegTileBase + static_cast<int>(seg_no), tid == 0 && seg_no < 20, tile_no + 1);
 
         // the team's running softmax over its tiles of this segment
         float m_run[kGMax], l_run[kGMax], o_reg[kGMax];
@@ -811,6 +841,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             fence_proxy_async();
             mbar_arrive(&bar_pfull[buf]);
             COOPT_TRACE_CYCLES(p.trace, kTrFirstProbs, tid == 0 && tile_no == 0);
+            COOPT_TRACE_CYCLES(p.trace, kTrProbsTileBase + static_cast<int>(tile_no), t == 0 && tile_no < 32);
           }
           // the product of the team's previous tile (its own buffers, so nothing above had to wait for it)
           if (pending) {
@@ -822,11 +853,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           for (int h = 0; h < kGMax; ++h) o_reg[h] *= a_o[h];      // what is folded in so far, on the scale of this tile's product
           pending = true;
           pend_tile = tile_no;
-          if (q_due) { publish_q(seg_no + 1); q_due = false; }
+          if (q_due) { publish_q(seg_no + 1, si + 3); q_due = false; }
           if (old_open) flush_old();
         }
         // (a team whose wait ran out keeps company until the next barrier makes it known to everybody)
-        if (q_due) publish_q(seg_no + 1);   // the segment had no tile for this team
+        if (q_due) publish_q(seg_no + 1, si + 3);   // the segment had no tile for this team
 
         // ---- end of segment: the team's sums and maxima go to the epilogue warp now, its output follows
         // once the last product has been folded in (flush_old, behind the next segment's first tile)

@@ -117,6 +117,8 @@ int plan_cta_stride(int planned_ctas, int batch, int num_kv_heads, int max_block
     blocks_max = ((u_max + planned_ctas - 1) / planned_ctas + 1) * chunk_blocks;
   } else {
     blocks_max = (n_max + planned_ctas - 1) / planned_ctas + 1;
+    // few blocks in all: fewer CTAs than planned take part, with at least kMinBlocksPerCta blocks each
+    if (blocks_max < 2 * kMinBlocksPerCta) blocks_max = 2 * kMinBlocksPerCta;
   }
   blocks_max = blocks_max < n_max ? blocks_max : n_max;
   long long segs_max = blocks_max < static_cast<long long>(batch) * num_kv_heads ? blocks_max : static_cast<long long>(batch) * num_kv_heads;

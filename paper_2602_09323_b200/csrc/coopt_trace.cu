@@ -11,7 +11,7 @@ unsigned long long* g_trace_buffer = nullptr;
 unsigned long long* trace_buffer() { return g_trace_buffer; }
 }  // namespace coopt
 
-// DEVICE buffer of kTraceMaxCtas * kTraceSlots uint64 (512 KiB), zeroed by the caller before a launch;
+// DEVICE buffer of kTraceMaxCtas * kTraceSlots uint64 (2 MiB), zeroed by the caller before a launch;
 // NULL switches the stamps off.  Not thread-safe; a tool for one measuring process.
 extern "C" int coopt_trace_set_buffer(void* device_buffer, size_t bytes) {
   if (device_buffer != nullptr && bytes < static_cast<size_t>(coopt::kTraceMaxCtas) * coopt::kTraceSlots * 8) return COOPT_ERR_WORKSPACE;

@@ -29,9 +29,15 @@ enum TraceSlot {
   kTrWriteDone,        // fused step: the new tokens' granules are written
   kTrNumSeg,           // number of segments of the first round (a count, not a time)
   kTrNumTiles,         // tiles of the CTA (a count)
+  kTrSmId,             // the SM the CTA ran on
   kTrSegBase = 24,     // 24 + i: epilogue warp received segment i (i < 20)
   kTrTeamSegBase = 44, // 44 + i: team 0 began segment i (i < 20)
-  kTraceSlots = 64
+  kTrCopyTileBase = 64,    // 64 + i: tile i requested (i < 32)
+  kTrProbsTileBase = 96,   // 96 + i: probabilities of tile i written by its team (i < 32)
+  kTrSegTileBase = 128,    // 128 + i: 1 + number of the first tile of segment i (i < 20; a count)
+  kTrLogitsTileBase = 148, // 148 + i: logits of tile i issued (i < 32)
+  kTrPvTileBase = 180,     // 180 + i: P V of tile i issued (i < 32)
+  kTraceSlots = 256
 };
 constexpr int kTraceMaxCtas = 1024;
 

@@ -17,11 +17,11 @@ import torch
 
 from . import binding, build, workloads
 
-SLOTS = 64
+SLOTS = 256
 MAX_CTAS = 1024
 NAMES = ["entry", "entry_ns", "setup_done", "plan_in_smem", "first_copy", "first_landed", "first_probs", "last_copy",
          "last_landed", "last_pv", "teams_done", "last_hand_off", "piece_stored", "counted", "epilogue_done", "exit",
-         "exit_ns", "write_done", "num_seg", "num_tiles"]
+         "exit_ns", "write_done", "num_seg", "num_tiles", "sm_id"]
 SEG_BASE, TEAM_SEG_BASE = 24, 44
 
 
@@ -30,6 +30,8 @@ def main():
     ap.add_argument("--workload", default="llama13b_decode", choices=["llama13b_decode", "mixed_serving", "long_context"])
     ap.add_argument("--no-append", action="store_true", help="attention only (no new token written in the launch)")
     ap.add_argument("--launches", type=int, default=12)
+    ap.add_argument("--timeline", type=int, nargs="*", default=None, help="CTAs whose tile-by-tile timeline is printed")
+    ap.add_argument("--per-cta", action="store_true", help="also list every CTA: SM, segments, streaming time")
     ap.add_argument("--sm-mhz", type=float, default=1965.0, help="SM clock used to turn cycles into microseconds")
     args = ap.parse_args()
     binding.use_library(build.build(trace=True))
@@ -68,9 +70,35 @@ def main():
         else:
             binding.decode_step_planned(caches[i % 2], plan, q, table.shape[1], w.sm_scale, ws, k_new, v_new, s_new,
                                         chunk_size=chunk, out=out)
+        if i == args.launches - 2:
+            torch.cuda.synchronize()
+            prev = buf.cpu().numpy().reshape(MAX_CTAS, SLOTS).copy()
     torch.cuda.synchronize()
     assert binding.workspace_status(ws) == 0
     t = buf.cpu().numpy().reshape(MAX_CTAS, SLOTS)
+    if args.per_cta:
+        # streaming time (first copy requested to last tile landed) of every CTA in the last two launches, by SM
+        us_ = 1.0 / args.sm_mhz
+        rows = []
+        for rec in (prev, t):
+            r = rec[rec[:, 0] != 0]
+            rows.append({int(x[20]) - 1: ((x[8] - x[4]) * us_, int(x[18]), (x[15] - x[0]) * us_) for x in r})
+        print("sm  launch A: stream_us nseg life_us | launch B: stream_us nseg life_us")
+        for sm in sorted(set(rows[0]) & set(rows[1])):
+            a, b = rows[0][sm], rows[1][sm]
+            print(f"{sm:3d}  {a[0]:6.2f} {a[1]} {a[2]:6.2f} | {b[0]:6.2f} {b[1]} {b[2]:6.2f}")
+    if args.timeline is not None:
+        us_ = 1.0 / args.sm_mhz
+        for cta in (args.timeline or [0, 1, 2, 3]):
+            x = t[cta]
+            seg_first = [int(v) - 1 for v in x[128:148] if v]
+            print(f"CTA {cta}: {int(x[18])} segments starting at tiles {seg_first}; epilogue got them at "
+                  f"{[round(float((v - x[0]) * us_), 2) for v in x[24:44] if v]}")
+            print(" tile   requested  logits_issued  probs_written  pv_issued   (us)")
+            for i in range(32):
+                if x[64 + i]:
+                    f = lambda v: f"{(v - x[0]) * us_:10.2f}" if v else "         -"
+                    print(f"{i:5d} {f(x[64 + i])}    {f(x[148 + i])}     {f(x[96 + i])}  {f(x[180 + i])}{'   <- segment starts' if i in seg_first else ''}")
     t = t[t[:, 0] != 0]
     us = 1.0 / args.sm_mhz
     print(f"workload {args.workload}{' (no append)' if args.no_append else ''}: {t.shape[0]} CTAs, "
@@ -81,7 +109,7 @@ def main():
           f"{(t[:, 1].max() - t[:, 1].min()) / 1e3:.1f} us, exits over {(t[:, 16].max() - t[:, 16].min()) / 1e3:.1f} us")
     print(f"{'milestone':<16}{'median':>9}{'earliest':>10}{'latest':>9}   (us after the CTA's first instruction, {args.sm_mhz:.0f} MHz)")
     for i, name in enumerate(NAMES):
-        if name in ("entry", "entry_ns", "exit_ns", "num_seg", "num_tiles"):
+        if name in ("entry", "entry_ns", "exit_ns", "num_seg", "num_tiles", "sm_id"):
             continue
         col = t[:, i]
         ok = col != 0
