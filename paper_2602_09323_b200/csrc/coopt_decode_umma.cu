@@ -96,7 +96,7 @@ struct UCfg {
   static constexpr int kNumBars = 2 * kStages + 4 * 4 + 3 * 2 + 2 + 2;
   static constexpr int kWriteStage = 4 * kBlockSize * D;       // staging of team 1's four warps for the fused append
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kSmemBytes = kMiscOff + 128;            // 64 bytes of planner words and flags, 64 of the published slice
+  static constexpr int kSmemBytes = kMiscOff + 128;            // flags, the tensor-memory address, the copy warp's first time stamp
   static_assert(kStageBytes % 128 == 0 && kKArea % 128 == 0 && kHdrOff % 128 == 0 && (kGatherRows * kPart) % 128 == 0 &&
                     (kGatherRows * kFp8Header) % 128 == 0, "tensor copies land on 128-byte boundaries");
   static_assert(kPart / 8 <= 256 && kGran % 16 == 0, "one box row is at most 256 eight-byte elements");
@@ -209,7 +209,11 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
 #ifdef COOPT_TRACE
   if (tid == 0) { unsigned int smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); trace_put(p.trace, kTrSmId, smid + 1); }
 #endif
+#ifdef COOPT_TRACE
+  const uint8_t* plan_region = p.plan + static_cast<size_t>((blockIdx.x + p.plan_rotate) % gridDim.x) * p.plan_cta_stride;
+#else
   const uint8_t* plan_region = p.plan + static_cast<size_t>(blockIdx.x) * p.plan_cta_stride;
+#endif
   if (tid == kProducerWarp * 32) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_part) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&map_hdr) : "memory");
@@ -322,6 +326,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
       // A step that appends tokens: the tile that holds a sequence's last block, and the ring stage that
       // team 1 borrows as staging, are not requested before team 1 has written the round's new tokens.
       bool writes_pending = has_new && round_hdr->n_tail > 0;
+      COOPT_TRACE_CYCLES(p.trace, kTrProducerPlan, lane == 0 && round_no == 0);
+
       for (int si = 0; si < nseg && ok; ++si) {
         const int n = plan.segs[si].n, g = plan.segs[si].g;
         const bool seg_tail = (plan.segs[si].run_flags & kSegTail) != 0;
@@ -953,6 +959,7 @@ int launch_umma_one(DecodeParams p, int grid, bool overlap_previous, cudaStream_
   if (!configure_kernel_smem(reinterpret_cast<const void*>(&paged_decode_umma_kernel<D, NP>), C::kSmemBytes)) return COOPT_ERR_CUDA;
 #ifdef COOPT_TRACE
   p.trace = trace_buffer();
+  p.plan_rotate = trace_plan_rotate();
 #endif
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(grid));

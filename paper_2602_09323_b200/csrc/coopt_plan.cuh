@@ -88,6 +88,7 @@ struct DecodeParams {
   const long long* slot_mapping;
   long long kv_token_stride;
   unsigned long long* trace;   // time stamps (trace build only; null otherwise)
+  int plan_rotate;             // trace build only: CTA i works through plan region (i + plan_rotate) mod planned_ctas
   int max_blocks_per_seq;
   int batch, num_q_heads, num_kv_heads, group;
   int num_blocks;

@@ -7,8 +7,10 @@
 namespace coopt {
 namespace {
 unsigned long long* g_trace_buffer = nullptr;
+int g_plan_rotate = 0;
 }
 unsigned long long* trace_buffer() { return g_trace_buffer; }
+int trace_plan_rotate() { return g_plan_rotate; }
 }  // namespace coopt
 
 // DEVICE buffer of kTraceMaxCtas * kTraceSlots uint64 (2 MiB), zeroed by the caller before a launch;
@@ -16,6 +18,13 @@ unsigned long long* trace_buffer() { return g_trace_buffer; }
 extern "C" int coopt_trace_set_buffer(void* device_buffer, size_t bytes) {
   if (device_buffer != nullptr && bytes < static_cast<size_t>(coopt::kTraceMaxCtas) * coopt::kTraceSlots * 8) return COOPT_ERR_WORKSPACE;
   coopt::g_trace_buffer = static_cast<unsigned long long*>(device_buffer);
+  return COOPT_OK;
+}
+
+// CTA i of the decode kernel works through plan region (i + rotate) mod planned CTAs: tells apart what is slow
+// because of its share of the plan from what is slow because of the SM it runs on.
+extern "C" int coopt_trace_set_rotate(int rotate) {
+  coopt::g_plan_rotate = rotate < 0 ? 0 : rotate;
   return COOPT_OK;
 }
 #endif

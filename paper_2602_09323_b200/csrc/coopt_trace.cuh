@@ -30,6 +30,7 @@ enum TraceSlot {
   kTrNumSeg,           // number of segments of the first round (a count, not a time)
   kTrNumTiles,         // tiles of the CTA (a count)
   kTrSmId,             // the SM the CTA ran on
+  kTrProducerPlan,     // the copy warp has seen the plan
   kTrSegBase = 24,     // 24 + i: epilogue warp received segment i (i < 20)
   kTrTeamSegBase = 44, // 44 + i: team 0 began segment i (i < 20)
   kTrCopyTileBase = 64,    // 64 + i: tile i requested (i < 32)
@@ -43,6 +44,7 @@ constexpr int kTraceMaxCtas = 1024;
 
 #ifdef COOPT_TRACE
 unsigned long long* trace_buffer();      // host: what coopt_trace_set_buffer registered (nullptr = none)
+int trace_plan_rotate();                 // host: what coopt_trace_set_rotate registered
 #ifdef __CUDACC__
 __device__ __forceinline__ void trace_put(unsigned long long* buf, int slot, unsigned long long v) {
   if (buf != nullptr && blockIdx.x < kTraceMaxCtas && slot < kTraceSlots) buf[blockIdx.x * kTraceSlots + slot] = v;

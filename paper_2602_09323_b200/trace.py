@@ -21,7 +21,7 @@ SLOTS = 256
 MAX_CTAS = 1024
 NAMES = ["entry", "entry_ns", "setup_done", "plan_in_smem", "first_copy", "first_landed", "first_probs", "last_copy",
          "last_landed", "last_pv", "teams_done", "last_hand_off", "piece_stored", "counted", "epilogue_done", "exit",
-         "exit_ns", "write_done", "num_seg", "num_tiles", "sm_id"]
+         "exit_ns", "write_done", "num_seg", "num_tiles", "sm_id", "producer_plan"]
 SEG_BASE, TEAM_SEG_BASE = 24, 44
 
 
@@ -31,6 +31,8 @@ def main():
     ap.add_argument("--no-append", action="store_true", help="attention only (no new token written in the launch)")
     ap.add_argument("--launches", type=int, default=12)
     ap.add_argument("--timeline", type=int, nargs="*", default=None, help="CTAs whose tile-by-tile timeline is printed")
+    ap.add_argument("--rotate", type=int, default=0, help="with --per-cta: the second listed launch gives CTA i the plan "
+                    "region i + ROTATE, to tell slow shares of the plan from slow SMs")
     ap.add_argument("--per-cta", action="store_true", help="also list every CTA: SM, segments, streaming time")
     ap.add_argument("--sm-mhz", type=float, default=1965.0, help="SM clock used to turn cycles into microseconds")
     args = ap.parse_args()
@@ -63,8 +65,10 @@ def main():
     buf = torch.zeros(MAX_CTAS * SLOTS, dtype=torch.int64, device="cuda")
     assert lib.coopt_trace_set_buffer(ctypes.c_void_p(buf.data_ptr()), buf.numel() * 8) == 0
     out = torch.empty_like(q)
+    lib.coopt_trace_set_rotate.restype, lib.coopt_trace_set_rotate.argtypes = ctypes.c_int, [ctypes.c_int]
     for i in range(args.launches):
         buf.zero_()
+        lib.coopt_trace_set_rotate(args.rotate if i == args.launches - 1 else 0)
         if args.no_append:
             binding.decode_step_planned(caches[i % 2], plan, q, table.shape[1], w.sm_scale, ws, chunk_size=chunk, out=out)
         else:
