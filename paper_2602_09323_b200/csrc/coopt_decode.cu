@@ -85,6 +85,7 @@ __global__ void __launch_bounds__(kThreads, 1) paged_decode_kernel(const DecodeP
   PlanSmem plan;
   plan.pre_blk = pre_blk; plan.pre_unit = pre_unit; plan.segs = segs; plan.ids = ids; plan.misc = misc;
   plan.slice = reinterpret_cast<long long*>(smem + C::kMiscOff + 64);
+  plan.bounds = nullptr;
   int ctx_early[2];
   plan_prefix_load(p, tid, kThreads, ctx_early);
   if (tid == 0) {

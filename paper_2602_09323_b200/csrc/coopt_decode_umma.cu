@@ -175,6 +175,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   plan.pre_blk = plan.pre_unit = nullptr;
   plan.misc = reinterpret_cast<int*>(smem + C::kMiscOff);          // flags and the tensor-memory address
   plan.slice = nullptr;
+  plan.bounds = nullptr;
   float* xch = reinterpret_cast<float*>(smem + C::kXchOff);         // [2 teams][kXchFloats]
   float* mlbuf = reinterpret_cast<float*>(smem + C::kMlOff);        // [2 segment parities][2 teams][kMlFloats]
   int* red_max = reinterpret_cast<int*>(smem + C::kRedOff);         // [2][4][12] per-warp maxima of a tile (ordered ints)

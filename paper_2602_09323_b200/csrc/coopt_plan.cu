@@ -28,15 +28,19 @@ __global__ void __launch_bounds__(kPlanThreads) decode_plan_kernel(const PlanKer
   __shared__ int misc[8];
   __shared__ long long slice[8];
   __shared__ int round_status;     // what the round being planned wants reported (bad block ids)
+  __shared__ long long bounds[kMaxAnchorCtas + 1];
+  __shared__ int budget[kMaxAnchorCtas];
   DecodeParams p = pk.d;
   p.status = &round_status;
   if (threadIdx.x == 0) round_status = 0;
   PlanSmem plan;
   plan.pre_blk = pre_blk; plan.pre_unit = pre_unit; plan.segs = segs; plan.ids = ids; plan.misc = misc; plan.slice = slice;
+  plan.bounds = bounds;
   const int tid = threadIdx.x;
   int ctx_early[2];
   plan_prefix_load(p, tid, kPlanThreads, ctx_early);
   plan_prefix(p, plan, tid, kPlanThreads, ctx_early);
+  if (!plan_anchor_bounds(p, plan, tid, kPlanThreads, budget)) plan.bounds = nullptr;
   if (tid == 0) plan_slice_publish(p, plan);
   __syncthreads();
   PlanSlice sl;
@@ -63,12 +67,41 @@ __global__ void __launch_bounds__(kPlanThreads) decode_plan_kernel(const PlanKer
   long long x = active ? sl.lo : 0;
   const long long x_end = active ? sl.hi : 0;
   bool wrote_last = false;
-  while (x < x_end) {
-    if (tid == 0) plan_round(p, plan, sl, x);
+  // the anchor (anchored split): a whole (sequence, kv head) appended behind the CTA's last round of the remainder
+  const int anchor_blocks = (active && sl.anchor_b >= 0) ? pre_blk[sl.anchor_b + 1] - pre_blk[sl.anchor_b] : 0;
+  bool anchor_pending = anchor_blocks > 0;
+  while (x < x_end || anchor_pending) {
+    if (tid == 0) {
+      if (x < x_end) {
+        plan_round(p, plan, sl, x);
+      } else {
+        misc[0] = 0;
+        misc[1] = static_cast<int>(x & 0xffffffffll);
+        misc[2] = static_cast<int>(x >> 32);
+      }
+    }
     __syncthreads();
-    const int nseg = misc[0];
+    int nseg = misc[0];
     const long long x_next = (static_cast<long long>(misc[2]) << 32) | static_cast<unsigned int>(misc[1]);
     if (tid < nseg) plan_round_finish(p, plan, sl, tid);
+    __syncthreads();
+    if (anchor_pending && x_next >= x_end) {
+      int staged = 0;
+      for (int i = 0; i < nseg; ++i) staged = max(staged, segs[i].list_off + segs[i].n);
+      if (nseg < kMaxSeg && staged + anchor_blocks <= kCap) {      // else: a round of its own, next time round
+        if (tid == 0) {
+          Segment sg = {};
+          sg.b = sl.anchor_b; sg.g = sl.anchor_g; sg.j0 = 0; sg.n = anchor_blocks; sg.list_off = staged;
+          sg.partial = 0; sg.expected = 1; sg.seq_blocks = anchor_blocks;
+          sg.run_flags = kRunFirst | kRunLast | kRunWhole | kSegTail;
+          sg.run_expected = 1; sg.first_cta = static_cast<int>(blockIdx.x);
+          segs[nseg] = sg;
+        }
+        ++nseg;
+        anchor_pending = false;
+      }
+    }
+    __syncthreads();
     plan_stage_ids(p, plan, nseg, tid, kPlanThreads);
     __syncthreads();
     int used = 0, n_tail = 0;
@@ -82,7 +115,7 @@ __global__ void __launch_bounds__(kPlanThreads) decode_plan_kernel(const PlanKer
     PlanRound* hdr = reinterpret_cast<PlanRound*>(region + at);
     if (tid == 0) {
       PlanRound h = {};
-      h.nseg = nseg; h.n_ids = used; h.bytes = bytes; h.last = x_next >= x_end ? 1 : 0; h.n_tail = n_tail; h.key = pk.key;
+      h.nseg = nseg; h.n_ids = used; h.bytes = bytes; h.last = (x_next >= x_end && !anchor_pending) ? 1 : 0; h.n_tail = n_tail; h.key = pk.key;
       h.status = round_status;
       *hdr = h;
       round_status = 0;
@@ -92,7 +125,7 @@ __global__ void __launch_bounds__(kPlanThreads) decode_plan_kernel(const PlanKer
     for (int i = tid; i < nseg * 4; i += kPlanThreads) dseg[i] = sseg[i];
     int* dids = reinterpret_cast<int*>(region + at + 64 + nseg * 64);
     for (int i = tid; i < ((used + 3) / 4) * 4; i += kPlanThreads) dids[i] = i < used ? ids[i] : 0;
-    wrote_last = x_next >= x_end;
+    wrote_last = x_next >= x_end && !anchor_pending;
     at += bytes;
     x = x_next;
     __syncthreads();
@@ -122,7 +155,7 @@ int plan_cta_stride(int planned_ctas, int batch, int num_kv_heads, int max_block
   }
   blocks_max = blocks_max < n_max ? blocks_max : n_max;
   long long segs_max = blocks_max < static_cast<long long>(batch) * num_kv_heads ? blocks_max : static_cast<long long>(batch) * num_kv_heads;
-  segs_max += 2;
+  segs_max += 3;
   if (chunk_blocks > 0) segs_max += blocks_max / chunk_blocks + 1;
   if (segs_max > blocks_max + 2) segs_max = blocks_max + 2;
   const long long rounds_max = (segs_max + kMaxSeg - 1) / kMaxSeg + (blocks_max + kCap / 2 - 1) / (kCap / 2) + 1;

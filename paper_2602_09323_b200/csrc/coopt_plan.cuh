@@ -17,6 +17,7 @@ constexpr int kMinBlocksPerCta = 16;
 constexpr int kMaxGroup = 8;
 constexpr int kCounterSlots = 16384;
 constexpr int kWsHeaderBytes = 256;
+constexpr int kMaxAnchorCtas = 256;   // the anchored split (below) is worked out for at most this many CTAs
 
 struct Segment {
   int b, g;          // sequence, kv head
@@ -116,6 +117,7 @@ struct PlanSmem {
   int* ids;          // [kCap]
   int* misc;         // [4]: nseg, next x (lo, hi), scratch flag
   long long* slice;  // [8]: the CTA's slice as one thread worked it out (plan_slice_publish)
+  long long* bounds; // anchored split: [P + 1] first flat index of every CTA's slice of the remainder (nullptr: equal slices)
 };
 
 // floor(a / b) for 0 <= a < 2^52, 0 < b < 2^31: one double division and a fix-up instead of the
@@ -196,15 +198,28 @@ struct PlanSlice {
   long long lo, hi, N;
   long long ulo, uhi, U;     // chunk mode: the same slice in units of (sequence, kv head, chunk)
   int P;
+  const long long* bounds;   // anchored split: slice i of the remainder is [bounds[i], bounds[i + 1])
+  int anchor_b, anchor_g;    // anchored split: the (sequence, kv head) this CTA also takes whole; -1: none
 };
 __device__ inline bool plan_slice(const DecodeParams& p, const PlanSmem& s, PlanSlice& sl) {
   const int B = p.batch, Hkv = p.num_kv_heads;
   sl.N = static_cast<long long>(Hkv) * s.pre_blk[B];
   sl.ulo = sl.uhi = sl.U = 0;
+  sl.bounds = nullptr;
+  sl.anchor_b = sl.anchor_g = -1;
   if (sl.N == 0) return false;
   if (p.chunk_blocks == 0) {
     sl.P = static_cast<int>(min(static_cast<long long>(p.planned_ctas), max(1ll, sl.N / kMinBlocksPerCta)));
     if (static_cast<int>(blockIdx.x) >= sl.P) return false;
+    if (s.bounds != nullptr && sl.P == p.planned_ctas) {
+      const int u = B * Hkv - sl.P + static_cast<int>(blockIdx.x);
+      sl.bounds = s.bounds;
+      sl.anchor_b = u / Hkv;
+      sl.anchor_g = u - sl.anchor_b * Hkv;
+      sl.lo = s.bounds[blockIdx.x];
+      sl.hi = s.bounds[blockIdx.x + 1];
+      return true;
+    }
     sl.lo = plan_div(blockIdx.x * sl.N, sl.P);
     sl.hi = plan_div((blockIdx.x + 1ll) * sl.N, sl.P);
     return true;
@@ -232,16 +247,65 @@ __device__ inline void plan_slice_publish(const DecodeParams& p, const PlanSmem&
   PlanSlice sl;
   const bool active = plan_slice(p, s, sl);
   s.slice[0] = sl.lo; s.slice[1] = sl.hi; s.slice[2] = sl.N; s.slice[3] = sl.ulo; s.slice[4] = sl.uhi; s.slice[5] = sl.U;
-  s.slice[6] = sl.P; s.slice[7] = active ? 1 : 0;
+  s.slice[6] = sl.P | (static_cast<long long>(sl.anchor_b + 1) << 32);
+  s.slice[7] = (active ? 1 : 0) | (sl.bounds != nullptr ? 2 : 0) | (static_cast<long long>(sl.anchor_g + 1) << 32);
 }
 __device__ inline bool plan_slice_fetch(const PlanSmem& s, PlanSlice& sl) {
   sl.lo = s.slice[0]; sl.hi = s.slice[1]; sl.N = s.slice[2]; sl.ulo = s.slice[3]; sl.uhi = s.slice[4]; sl.U = s.slice[5];
-  sl.P = static_cast<int>(s.slice[6]);
-  return s.slice[7] != 0;
+  sl.P = static_cast<int>(s.slice[6] & 0xffffffffll);
+  sl.anchor_b = static_cast<int>(s.slice[6] >> 32) - 1;
+  sl.anchor_g = static_cast<int>(s.slice[7] >> 32) - 1;
+  sl.bounds = (s.slice[7] & 2) ? s.bounds : nullptr;
+  return (s.slice[7] & 1) != 0;
 }
 // CTA that owns flat block index x (decode mode).
 __device__ __forceinline__ int plan_cta_of(const PlanSlice& sl, long long x) {
+  if (sl.bounds != nullptr) {
+    int lo = 0, hi = sl.P - 1;                       // largest i with bounds[i] <= x among the non-empty slices
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (sl.bounds[mid] <= x) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+  }
   return static_cast<int>(plan_div((x + 1) * sl.P - 1, static_cast<int>(sl.N)));
+}
+
+// Anchored split (decode mode).  With equal slices of the flat list, a CTA whose slice holds no whole
+// (sequence, kv head) ends on a piece of a cut one, and is then usually the last to deliver a piece of it: the
+// launch ends on its trip to the piece counter and its merge.  Here every CTA takes one (sequence, kv head)
+// whole -- its anchor: the last P of them, in order -- and the others (the remainder, a prefix of the flat
+// list) are cut so that every CTA still gets the same number of blocks: slice i of the remainder has the equal
+// share minus the anchor's blocks.  A CTA works through its pieces of the remainder first and its anchor last,
+// so every merge happens while the stream still runs and every CTA ends on a plain store.  Needs as many
+// (sequence, kv head) pairs as CTAs and no anchor larger than the equal share; false otherwise.
+__device__ inline bool plan_anchor_bounds(const DecodeParams& p, const PlanSmem& s, int tid, int nthreads, int* budget /* shared, [P] */) {
+  const int B = p.batch, Hkv = p.num_kv_heads, P = p.planned_ctas;
+  const long long N = static_cast<long long>(Hkv) * s.pre_blk[B];
+  const long long U = static_cast<long long>(B) * Hkv;
+  if (s.bounds == nullptr || p.chunk_blocks != 0 || P > kMaxAnchorCtas || U < P || N / kMinBlocksPerCta < P) return false;
+  for (int i = tid; i < P; i += nthreads) {
+    const int u = static_cast<int>(U) - P + i, b = u / Hkv;
+    const int a = s.pre_blk[b + 1] - s.pre_blk[b];
+    const long long share = plan_div((i + 1ll) * N, P) - plan_div(static_cast<long long>(i) * N, P);
+    budget[i] = static_cast<int>(share) - a;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    long long at = 0;
+    bool ok = true, none = true, all = true;
+    for (int i = 0; i < P; ++i) {
+      s.bounds[i] = at;
+      ok = ok && budget[i] >= 0;
+      none = none && budget[i] == 0;
+      all = all && budget[i] > 0;
+      at += budget[i];
+    }
+    // the pieces of a cut (sequence, kv head) must sit in consecutive CTAs: no empty slice between two others
+    s.bounds[P] = (ok && (none || all)) ? at : -1;
+  }
+  __syncthreads();
+  return s.bounds[P] >= 0;
 }
 
 // One thread plans the next round starting at flat index x: fills the geometry of segs (plan_round_finish
