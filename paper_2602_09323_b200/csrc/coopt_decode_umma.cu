@@ -206,6 +206,9 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
   // two trips to memory start before anything else: the context lengths for the planner, and the copy
   // engine's view of the cache (fetched on first use otherwise, in front of the first tile)
   COOPT_TRACE_CYCLES(p.trace, kTrEntry, tid == 0);
+#ifdef COOPT_TRACE
+  if (tid == 0 && p.trace != nullptr && blockIdx.x < kTraceMaxCtas) trace_put(p.trace, kTrPrevExitNs, p.trace[blockIdx.x * kTraceSlots + kTrExitNs]);
+#endif
   COOPT_TRACE_NS(p.trace, kTrEntryNs, tid == 0);
 #ifdef COOPT_TRACE
   if (tid == 0) { unsigned int smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); trace_put(p.trace, kTrSmId, smid + 1); }

@@ -21,7 +21,7 @@ SLOTS = 256
 MAX_CTAS = 1024
 NAMES = ["entry", "entry_ns", "setup_done", "plan_in_smem", "first_copy", "first_landed", "first_probs", "last_copy",
          "last_landed", "last_pv", "teams_done", "last_hand_off", "piece_stored", "counted", "epilogue_done", "exit",
-         "exit_ns", "write_done", "num_seg", "num_tiles", "sm_id", "producer_plan"]
+         "exit_ns", "write_done", "num_seg", "num_tiles", "sm_id", "producer_plan", "prev_exit_ns"]
 SEG_BASE, TEAM_SEG_BASE = 24, 44
 
 
@@ -67,14 +67,15 @@ def main():
     out = torch.empty_like(q)
     lib.coopt_trace_set_rotate.restype, lib.coopt_trace_set_rotate.argtypes = ctypes.c_int, [ctypes.c_int]
     for i in range(args.launches):
-        buf.zero_()
+        if i != args.launches - 1:
+            buf.zero_()                     # (the last launch follows its predecessor directly and keeps its exit times)
         lib.coopt_trace_set_rotate(args.rotate if i == args.launches - 1 else 0)
         if args.no_append:
             binding.decode_step_planned(caches[i % 2], plan, q, table.shape[1], w.sm_scale, ws, chunk_size=chunk, out=out)
         else:
             binding.decode_step_planned(caches[i % 2], plan, q, table.shape[1], w.sm_scale, ws, k_new, v_new, s_new,
                                         chunk_size=chunk, out=out)
-        if i == args.launches - 2:
+        if i == args.launches - 3:
             torch.cuda.synchronize()
             prev = buf.cpu().numpy().reshape(MAX_CTAS, SLOTS).copy()
     torch.cuda.synchronize()
@@ -111,9 +112,11 @@ def main():
     span = (t[:, 16].max() - t[:, 1].min()) / 1e3
     print(f"launch span on the global timer: {span:.1f} us (first entry to last exit); entries spread over "
           f"{(t[:, 1].max() - t[:, 1].min()) / 1e3:.1f} us, exits over {(t[:, 16].max() - t[:, 16].min()) / 1e3:.1f} us")
+    if t[:, 22].min() > 0:
+        print(f"gap to the launch before (its last exit to this one's first entry): {(t[:, 1].min() - t[:, 22].max()) / 1e3:.2f} us")
     print(f"{'milestone':<16}{'median':>9}{'earliest':>10}{'latest':>9}   (us after the CTA's first instruction, {args.sm_mhz:.0f} MHz)")
     for i, name in enumerate(NAMES):
-        if name in ("entry", "entry_ns", "exit_ns", "num_seg", "num_tiles", "sm_id"):
+        if name in ("entry", "entry_ns", "exit_ns", "num_seg", "num_tiles", "sm_id", "prev_exit_ns"):
             continue
         col = t[:, i]
         ok = col != 0
