@@ -5,10 +5,13 @@
 // A CTA owns one (sequence, kv head, tile of consecutive query tokens).  Its 128 rows are the (query
 // token, query head of the group) pairs of the tile, so the K/V stream of the kv head is fetched once
 // for all G heads (Algorithm 2).  The E4M3 codes of the cache feed tcgen05.mma kind::f8f6f4 as they are:
-//     S [128 rows x 128 keys] = Q  [128 x D] . Ktile^T      Q as two exact E4M3 terms of the bf16 query
-//     O [128 rows x D]       += P  [128 x 128 keys] . Vtile  P as three E4M3 terms of the probabilities
+//     S [128 rows x 128 keys] = Q  [128 x D] . Ktile^T      kind::f8f6f4: Q as two exact E4M3 terms of the bf16 query
+//     O [128 rows x D]       += P  [128 x 128 keys] . Vtile  kind::f16: P rounded once to f16, the V codes widened to f16 (exact)
 // with fp32 accumulators in tensor memory.  The K scale of a block multiplies the logits of its 16 keys,
-// the V scale is folded into the probabilities.
+// the V scale is folded into the probabilities.  (Carrying P as E4M3 terms instead, three per probability for
+// the same 11 bits, kept the V codes as they are but cost five conversions per pair of probabilities on the
+// SM's conversion pipe, which then bounded the kernel; widening V costs one conversion per pair of codes and
+// a tile of V is a sixteenth of a tile of P per query row.)
 //
 // The context is walked twice, 128 keys (eight cache blocks) at a time.  The first walk fetches K only and
 // leaves every row's maximum logit (and the largest V scale); the second recomputes the logits, so every
@@ -22,9 +25,10 @@
 //               row's logits from tensor memory 16 at a time (one cache block: one pair of scales), and
 //               maxima and sums are exchanged only at the end of a walk;
 //   warp 16     copies: gather requests over the tensor map of the cache (K parts, V parts, headers of
-//               four granules each) into six slots of 16 KB + 256 B.  The first walk uses all six for K
+//               four granules each) into four slots of 16 KB + 256 B.  The first walk uses all four for K
 //               tiles (and their scales); in the second walk two take K tiles, freed as soon as the logits
-//               are computed, and four take V tiles and the scales, held until the P V instructions are done;
+//               are computed, and two take V tiles and the scales, freed as soon as the tile's team has widened
+//               the codes into its f16 operand;
 //   warp 17     one lane issues the S instructions; warp 18 one lane issues the P V instructions.
 // Every wait is bounded; a wait that runs out is reported in the status word and all roles leave through
 // the common exit, which frees the tensor memory.
@@ -42,8 +46,8 @@ constexpr int kPuThreads = 608;
 constexpr int kPuTileBlocks = 8;
 constexpr int kPuTileKeys = kPuTileBlocks * kBlockSize;   // 128
 constexpr int kPuD = 128;
-constexpr int kPuSlots = 6;                                // of the copy ring
-constexpr int kPuKSlots = 2, kPuVSlots = 4;               // second walk: slots 0-1 take K tiles, slots 2-5 V tiles and scales
+constexpr int kPuSlots = 4;                                // of the copy ring
+constexpr int kPuKSlots = 2, kPuVSlots = 2;               // second walk: slots 0-1 take K tiles, slots 2-3 V tiles and scales
 constexpr float kPuLog2e = 1.4426950408889634f;
 constexpr float kPuGain = 256.0f;                          // probabilities are carried times 2^8 (at most 256 < 448)
 
@@ -71,10 +75,11 @@ struct PuCfg {
   static constexpr int kOperand = 128 * 128;                      // one 128 x 128 operand of codes
   static constexpr int kRingOff = 0;
   static constexpr int kQOff = kRingOff + kPuSlots * kSlot;          // Q: lead term, remainder term
-  static constexpr int kPOff = kQOff + 2 * kOperand;                 // P: [team][term], three terms (12 bits) per probability
-  static constexpr int kPTerms = 3;
-  static constexpr int kBarOff = kPOff + 2 * kPTerms * kOperand;
-  static constexpr int kNumBars = 2 * kPuSlots + kPuKSlots + kPuVSlots + 2 + 2 + 2;   // full, free1, kdone, vdone, sfull, sfree, pfull
+  static constexpr int kOperand16 = 128 * 128 * 2;                   // one 128 x 128 operand of f16 values
+  static constexpr int kPOff = kQOff + 2 * kOperand;                 // P: [team], f16
+  static constexpr int kV16Off = kPOff + 2 * kOperand16;             // V^T of a tile widened to f16: [team]
+  static constexpr int kBarOff = kV16Off + 2 * kOperand16;
+  static constexpr int kNumBars = 2 * kPuSlots + kPuKSlots + 2 * kPuVSlots + 2 + 2 + 2;   // full, free1, kdone, vdone, vread, sfull, sfree, pfull
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kSmemBytes = kMiscOff + 64;
   static_assert(kSlot % 128 == 0 && kSmemBytes <= 232448, "shared memory of one CTA");
@@ -88,6 +93,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   uint8_t* ring = smem + C::kRingOff;
   uint8_t* qbuf = smem + C::kQOff;
   uint8_t* pbuf = smem + C::kPOff;
+  uint8_t* v16buf = smem + C::kV16Off;
   // float [4 parts of a row][128] maxima and [4][128] sums share the probability operands' memory: the maxima are
   // exchanged before the first probability is written, the sums after the last P V instruction has finished
   float* xch = reinterpret_cast<float*>(smem + C::kPOff);
@@ -98,7 +104,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   uint64_t* bar_free1 = bar_full + kPuSlots;         // [kPuSlots] first walk: the tile's team has read its logits and scales
   uint64_t* bar_kdone = bar_free1 + kPuSlots;        // [kPuKSlots] second walk: the logits of the K tile in the slot are computed
   uint64_t* bar_vdone = bar_kdone + kPuKSlots;       // [kPuVSlots] second walk: the P V instructions of the V tile in the slot are done
-  uint64_t* bar_sfull = bar_vdone + kPuVSlots;       // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
+  uint64_t* bar_vread = bar_vdone + kPuVSlots;       // [kPuVSlots] second walk: the tile's team has widened the V tile in the slot
+  uint64_t* bar_sfull = bar_vread + kPuVSlots;       // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
   uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's eight warps have read them (and the tile's scales)
   uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's probabilities of a tile are in shared memory
   int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory, [4..7] V scale maxima
@@ -124,7 +131,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     *abort_flag = 0;
     for (int i = 0; i < kPuSlots; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_free1[i], 8); }
     for (int i = 0; i < kPuKSlots; ++i) mbar_init(&bar_kdone[i], 1);
-    for (int i = 0; i < kPuVSlots; ++i) mbar_init(&bar_vdone[i], 1);
+    for (int i = 0; i < kPuVSlots; ++i) { mbar_init(&bar_vdone[i], 1); mbar_init(&bar_vread[i], 8); }
     for (int i = 0; i < 2; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 8); mbar_init(&bar_pfull[i], kPuTeam); }
     mbar_fence_init();
   }
@@ -282,7 +289,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
           if (t >= kPuKSlots) ok = wait_bar(&bar_kdone[ks], static_cast<uint32_t>(t / kPuKSlots - 1) & 1u, abort_flag);
           else if (uses1(ks) > 0) ok = wait_bar(&bar_free1[ks], static_cast<uint32_t>(uses1(ks) - 1) & 1u, abort_flag);
           if (ok) {
-            if (t >= kPuVSlots) ok = wait_bar(&bar_vdone[vq], static_cast<uint32_t>(t / kPuVSlots - 1) & 1u, abort_flag);
+            if (t >= kPuVSlots) ok = wait_bar(&bar_vread[vq], static_cast<uint32_t>(t / kPuVSlots - 1) & 1u, abort_flag);
             else if (uses1(vs) > 0) ok = wait_bar(&bar_free1[vs], static_cast<uint32_t>(uses1(vs) - 1) & 1u, abort_flag);
           }
           if (ok) {
@@ -329,7 +336,9 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     // ================= outputs: O += P . Vtile, both terms of P (one lane) ===================================
     if (lane == 0) {
       bool ok = true;
-      const uint64_t desc_v = umma_desc(smem_u32(ring), C::kPart, 128), desc_p = umma_desc(smem_u32(pbuf), 128, 1024);
+      // both operands of P V are f16, K-major: 8 rows x 16 bytes (8 values) per core matrix, cores of a row group 128 bytes
+      // apart along the keys, row groups 2048 bytes apart
+      const uint64_t desc_v = umma_desc(smem_u32(v16buf), 128, 2048), desc_p = umma_desc(smem_u32(pbuf), 128, 2048);
       for (int T = n_tiles; T < total && ok; ++T) {
         const int t = T - n_tiles;
         const uint32_t vq = t % kPuVSlots, team = T & 1u;
@@ -339,14 +348,10 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         ok = wait_bar(&bar_pfull[team], use & 1u, abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
-        const int nks = (nb + 1) >> 1;                // 32 keys (two granules) per instruction
-        const uint64_t dv = desc_v + (((kPuKSlots + vq) * C::kSlot) >> 4), dp = desc_p + ((team * C::kPTerms * C::kOperand) >> 4);
-#pragma unroll
-        for (int term = 0; term < C::kPTerms; ++term)
-          for (int ks = 0; ks < nks; ++ks)
-            umma_f8(tmem_o, dp + ((term * C::kOperand) >> 4) + ks * 16, dv + ks * ((2 * C::kPart) >> 4), umma_idesc(D), (t | term | ks) != 0);
-        umma_commit(&bar_vdone[vq]);        // the V slot and the team's probability operand are free again
+        const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);      // 16 keys (one cache block) per instruction
+        const uint64_t dv = desc_v + ((team * C::kOperand16) >> 4), dp = desc_p + ((team * C::kOperand16) >> 4);
+        for (int ks = 0; ks < nb; ++ks) umma_f16(tmem_o, dp + ks * 16, dv + ks * 16, umma_idesc(D), (t | ks) != 0);
+        umma_commit(&bar_vdone[vq]);        // the team's two f16 operands are free again
       }
       if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     }
@@ -356,7 +361,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     const int c_lo = half * (kPuTileBlocks / 2), c_hi = c_lo + kPuTileBlocks / 2;   // this thread's cache blocks of a tile
     bool bad = false;
     float m_row = -INFINITY, l_row = 0.0f, v_max = 0.0f;
-    uint8_t* prow = pbuf + team * C::kPTerms * C::kOperand + (r >> 3) * 1024 + (r & 7) * 16;
+    uint8_t* prow = pbuf + team * C::kOperand16 + (r >> 3) * 2048 + (r & 7) * 16;      // row r of the team's P operand
+    uint8_t* vrow = v16buf + team * C::kOperand16 + (r >> 3) * 2048 + (r & 7) * 16;    // dim r of the team's V^T operand
 
     // ---- first walk: the row's maximum logit, and the largest V scale ------------------------------------
     for (int T = team; T < n_tiles; T += 2) {
@@ -402,12 +408,12 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     const float m_use = m_row == -INFINITY ? 0.0f : m_row;
     const float v_inv = v_max > 0.0f ? kPuGain / v_max : 0.0f;
 
-    // ---- second walk: probabilities against the final maximum, two E4M3 terms each -----------------------
+    // ---- second walk: probabilities against the final maximum (f16), the V tile widened to f16 -----------
     int mine = 0;                                                  // this team's tiles of the second walk so far
     for (int T = n_tiles + ((team - n_tiles % 2) + 2) % 2; T < total && !bad; T += 2, ++mine) {
       const int t = T - n_tiles;
       const uint32_t vq = t % kPuVSlots, buf = T & 1u;
-      uint8_t* st = ring + (kPuKSlots + vq) * C::kSlot;            // the tile's V parts, and behind them its scales
+      const uint8_t* st = ring + (kPuKSlots + vq) * C::kSlot;      // the tile's V parts, and behind them its scales
       bool ok = wait_bar(&bar_full[kPuKSlots + vq], vslot_par(t), abort_flag);
       ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
       // the logits are computed: the tile's K slot can be refilled
@@ -423,70 +429,58 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       const int nb = (nkeys + kBlockSize - 1) / kBlockSize;
 #pragma unroll 2
       for (int c = c_lo; c < c_hi; ++c) {
-        uint4 lead4 = make_uint4(0u, 0u, 0u, 0u), rest4 = make_uint4(0u, 0u, 0u, 0u), last4 = make_uint4(0u, 0u, 0u, 0u);
-        if (c < nb) {
-          uint32_t s[16];
-          tmem_ld16_issue(tmem + 128 * buf + 16 * c + lane_base, s);
-          const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + c * kFp8Header);
-          const float sk = hdr[0] * qscale;
-          const float pv = hdr[1] * v_inv;
-          const int visible = lim - (key0 + c * kBlockSize);
-          tmem_ld_wait(s);
-          uint32_t lw[4], rw[4], tw[4];
+        if (c >= nb) break;                               // uniform over the warp: the P V instructions stop at block nb
+        uint32_t s[16];
+        tmem_ld16_issue(tmem + 128 * buf + 16 * c + lane_base, s);
+        const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + c * kFp8Header);
+        const float sk = hdr[0] * qscale;
+        const float pv = hdr[1] * v_inv;
+        const int visible = lim - (key0 + c * kBlockSize);
+        // dim r of V^T, the 16 tokens of block c: widened to f16 (exact) while the logits are on their way
+        const uint4 vc = *reinterpret_cast<const uint4*>(st + c * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
+        const int keep = nkeys - c * kBlockSize;          // tokens of the block inside the context (Eq. 9)
+        uint32_t vw[8];
+        {
+          const uint32_t cw[4] = {vc.x, vc.y, vc.z, vc.w};
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            float pe[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float x = ex2(__uint_as_float(s[4 * e + j]) * sk - m_use);
-              pe[j] = (4 * e + j <= visible) ? x : 0.0f;
-              l_row += pe[j];
-            }
-            uint32_t h0 = pack_f16x2(pe[0] * pv, pe[1] * pv), h1 = pack_f16x2(pe[2] * pv, pe[3] * pv);
-            // each term is the E4M3 value nearest to what the earlier ones left over (the differences are exact)
-            const uint32_t l0 = e4m3_term(h0, 1.0f), l1 = e4m3_term(h1, 1.0f);
-            const uint32_t r0 = e4m3_term(h0, 1.0f), r1 = e4m3_term(h1, 1.0f);
-            lw[e] = l0 | (l1 << 16);
-            rw[e] = r0 | (r1 << 16);
-            tw[e] = f16x2_to_e4m3x2(h0) | (f16x2_to_e4m3x2(h1) << 16);
+          for (int j = 0; j < 4; ++j) {
+            const int left = keep - 4 * j;
+            const uint32_t w = cw[j] & (left >= 4 ? 0xFFFFFFFFu : (left <= 0 ? 0u : (1u << (8 * left)) - 1u));
+            vw[2 * j] = e4m3x2_to_f16x2_lo(w);
+            vw[2 * j + 1] = e4m3x2_to_f16x2_hi(w);
           }
-          lead4 = make_uint4(lw[0], lw[1], lw[2], lw[3]);
-          rest4 = make_uint4(rw[0], rw[1], rw[2], rw[3]);
-          last4 = make_uint4(tw[0], tw[1], tw[2], tw[3]);
         }
-        if (c < 2 * ((nb + 1) >> 1)) {                 // what the P V instructions of this tile read
-          *reinterpret_cast<uint4*>(prow + c * 128) = lead4;
-          *reinterpret_cast<uint4*>(prow + C::kOperand + c * 128) = rest4;
-          *reinterpret_cast<uint4*>(prow + 2 * C::kOperand + c * 128) = last4;
+        *reinterpret_cast<uint4*>(vrow + (2 * c) * 128) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
+        *reinterpret_cast<uint4*>(vrow + (2 * c + 1) * 128) = make_uint4(vw[4], vw[5], vw[6], vw[7]);
+        tmem_ld_wait(s);
+        uint32_t pw[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float x0 = ex2(__uint_as_float(s[2 * e]) * sk - m_use), x1 = ex2(__uint_as_float(s[2 * e + 1]) * sk - m_use);
+          const float p0 = (2 * e <= visible) ? x0 : 0.0f, p1 = (2 * e + 1 <= visible) ? x1 : 0.0f;
+          l_row += p0 + p1;
+          pw[e] = pack_f16x2(p0 * pv, p1 * pv);           // at most 256: probabilities are carried times 2^8
         }
+        *reinterpret_cast<uint4*>(prow + (2 * c) * 128) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+        *reinterpret_cast<uint4*>(prow + (2 * c + 1) * 128) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&bar_sfree[buf]);
-      // V codes of slots past the context inside the last block are cleared (row r = dim r of V^T), and
-      // so is the slot behind an odd number of blocks, which the last instruction also reads
-      if (half == 0 && (nkeys & 15) != 0) {
-        uint4* row = reinterpret_cast<uint4*>(st + (nkeys >> 4) * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
-        const int keep = nkeys & 15;
-        uint4 w = *row;
-        uint32_t* ww = reinterpret_cast<uint32_t*>(&w);
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const int left = keep - 4 * j;
-          ww[j] &= left >= 4 ? 0xFFFFFFFFu : (left <= 0 ? 0u : (1u << (8 * left)) - 1u);
-        }
-        *row = w;
-      }
-      if (half == 0 && (nb & 1) != 0)
-        *reinterpret_cast<uint4*>(st + nb * C::kPart + (r >> 3) * 128 + (r & 7) * 16) = make_uint4(0u, 0u, 0u, 0u);
+      if (lane == 0) { mbar_arrive(&bar_sfree[buf]); mbar_arrive(&bar_vread[vq]); }
       fence_proxy_async();
       mbar_arrive(&bar_pfull[team]);
     }
 
     // ---- the last P V instruction has finished: normalise and store ---------------------------------------
     if (!bad) {
+      // A wait names a phase by its parity, which only tells the phase before from the one in progress: a team
+      // that is done a tile early must not ask for the last tile's phase while the phase before it on the same
+      // barrier is still open.  The last two tiles' instructions are waited for in order (the one before them
+      // is finished: the team waited for it, or for a later one, inside its loop).
       const int tl = n_tiles - 1;
-      bool ok = wait_bar(&bar_vdone[tl % kPuVSlots], static_cast<uint32_t>(tl / kPuVSlots) & 1u, abort_flag);
+      bool ok = true;
+      if (tl >= 1) ok = wait_bar(&bar_vdone[(tl - 1) % kPuVSlots], static_cast<uint32_t>((tl - 1) / kPuVSlots) & 1u, abort_flag);
+      ok = ok && wait_bar(&bar_vdone[tl % kPuVSlots], static_cast<uint32_t>(tl / kPuVSlots) & 1u, abort_flag);
       ok = __all_sync(0xffffffffu, ok);
       bad = !ok;
     }
