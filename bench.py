@@ -335,7 +335,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--workload", default="llama13b_decode",
                     choices=["llama13b_decode", "llama13b_40layers", "mha_bf16_ablation", "mixed_serving", "long_context",
-                             "chunked_prefill"],
+                             "chunked_prefill", "kv_write_fill"],
                     help="llama13b_decode is the benchmark; llama13b_40layers runs the 40 layers of one model step through "
                          "coopt_decode_layers; the others time the remaining configurations (1 GPU, kernel-level line "
                          "without the end-to-end and CPU legs)")
@@ -344,6 +344,8 @@ def main():
         return run_reference(args)
     if args.workload == "llama13b_40layers":
         return run_layers(args)
+    if args.workload == "kv_write_fill":
+        return run_kv_write_fill(args)
     if args.workload != "llama13b_decode":
         return run_other_workload(args)
 
@@ -517,6 +519,47 @@ def main():
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def run_kv_write_fill(args):
+    """coopt_kv_write on a bulk fill: the 32 x 2048 tokens of the LLaMA-13B-shaped workload written in one call into an
+    empty FP8 cache (whole blocks: one scale per block, no resident codes), caches visited in turn."""
+    import torch
+    from paper_2602_09323_b200 import binding, build, workloads
+    torch.cuda.set_device(0)
+    build.build()
+    binding.load_library()
+    w = workloads.config_llama13b_decode()
+    k, v, slots = w.k.cuda(), w.v.cuda(), w.slot_mapping.cuda()
+    caches = [binding.Cache(w.num_blocks, HKV, D) for _ in range(4)]
+    steps, warmup = max(1, min(args.steps, 400)), max(3, min(args.warmup, 20))
+    for i in range(warmup):
+        binding.kv_write(caches[i % 4], k, v, slots)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(torch.cuda.current_device(), period_s=0.002)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(steps):
+        binding.kv_write(caches[i % 4], k, v, slots)
+    e1.record()
+    torch.cuda.synchronize()
+    sampler.stop_flag = True
+    ms = e0.elapsed_time(e1) / steps
+    T = k.shape[0]
+    algo = T * HKV * D * 2 * 2 + T * HKV * D * 2 + T * 8 + (T // 16) * HKV * 32      # bf16 K and V read, codes and headers written
+    peaks_path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    peak = float(json.load(open(peaks_path))["hbm_gbs"]) if os.path.exists(peaks_path) else FALLBACK_HBM_GBS
+    achieved = algo / (ms * 1e-3) / 1e9
+    line = {"metric": "Opt-KV write tokens/s", "value": T / (ms * 1e-3), "unit": "attention-layer tokens/s", "n_gpus": 1, "steps": steps,
+            "warmup": warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16 in, fp8_e4m3 codes and fp32 scales out", "data": "synthetic",
+            "config": {"workload": "kv_write_fill: %d tokens, Hkv 8, head_dim 128, one call" % T, "l2": "four caches of 138 MB visited in turn"},
+            "gpu_launches": steps, "clocks": sampler.summary(), "e2e": None,
+            "roofline": {"bound": "hbm", "kernel": "kv_write_fp8_span_kernel<128>", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "algorithmic_bytes_per_launch": algo, "kernel_us": ms * 1e3, "traffic": None},
+            "cpu_baseline": None}
+    print(json.dumps(line), flush=True)
 
 
 def run_layers(args):

@@ -24,6 +24,8 @@
  *       bytes 16*D..32*D-1     V codes, transposed: token t, dim d at (d/8)*128 + (d%8)*16 + t
  *       bytes 32*D..32*D+3     fp32 K scale of the granule     bytes 32*D+4..32*D+7  fp32 V scale
  *       bytes 32*D+8..32*D+31  zero
+ *       bytes 32*D+32..32*D+127 padding (never read, never written: a granule is 32*D + 128 bytes, so that
+ *                              granules start on 128-byte lines)
  *   A dequantised element is decode_e4m3(code) * scale (Eq. 6).  A scale of 0 marks a
  *   granule that holds only zeros.  Both parts are laid out as the tensor cores read matrix
  *   operands from shared memory (8 rows x 16 bytes form one contiguous 128-byte unit), so a part

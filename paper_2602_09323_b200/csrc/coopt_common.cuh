@@ -11,7 +11,9 @@
 namespace coopt {
 
 constexpr int kBlockSize = 16;     // tokens per physical block
-constexpr int kFp8Header = 32;     // bytes behind the codes of an FP8 granule: K scale, V scale, zeros
+constexpr int kFp8Header = 32;     // bytes behind the codes of an FP8 granule that are read: K scale, V scale, zeros
+constexpr int kFp8Tail = 128;      // bytes behind the codes that the granule occupies: the header and padding, so that
+                                   // granules start on 128-byte lines and no line is shared by two writers
 constexpr float kE4m3Max = 448.0f;
 
 // ---- cache layout ---------------------------------------------------------------------------
@@ -31,11 +33,11 @@ constexpr float kE4m3Max = 448.0f;
 // a chunk holds two k-steps (K) or two n-tiles (V) of two registers each.
 
 __host__ __device__ constexpr int granule_bytes(int D, bool fp8) {
-  return fp8 ? kFp8Header + 2 * kBlockSize * D : 2 * kBlockSize * D * 2;
+  return fp8 ? kFp8Tail + 2 * kBlockSize * D : 2 * kBlockSize * D * 2;
 }
 __host__ __device__ constexpr int part_bytes(int D, bool fp8) { return kBlockSize * D * (fp8 ? 1 : 2); }
 __host__ __device__ constexpr int part_offset(int D, bool fp8, int which) { return which * part_bytes(D, fp8); }
-// FP8 granule: [K codes 16D][V codes 16D][fp32 K scale, fp32 V scale, 24 zero bytes]
+// FP8 granule: [K codes 16D][V codes 16D][fp32 K scale, fp32 V scale, 24 zero bytes][96 bytes of padding]
 __host__ __device__ constexpr int header_offset(int D) { return 2 * kBlockSize * D; }
 
 // Byte offset of K element (token t, dim d) inside the K part.

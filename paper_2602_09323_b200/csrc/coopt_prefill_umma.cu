@@ -68,7 +68,7 @@ struct PrefillUmmaParams {
 
 struct PuCfg {
   static constexpr int kPart = kBlockSize * kPuD;                 // 2048: K (or V) codes of one granule
-  static constexpr int kGran = 2 * kPart + kFp8Header;
+  static constexpr int kGran = granule_bytes(kPuD, true);
   static constexpr int kKArea = kPuTileBlocks * kPart;            // 16 KB: the K parts, or the V parts, of a tile
   static constexpr int kHdrOff = kKArea;                          // behind them the eight headers (scales) of the tile
   static constexpr int kSlot = kHdrOff + kPuTileBlocks * kFp8Header;   // 16,640

@@ -29,17 +29,17 @@ __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WritePar
 // FP8, many tokens (prefill chunks, bulk fills): one CTA per (kSpan consecutive tokens, kWriteHeads
 // kv heads).  Every warp settles one token of the span in the same memory trip; the groups found
 // (one per 16 tokens in a contiguous fill) are then served by all warps.
-constexpr int kSpan = kWriteWarps;
+constexpr int kSpan = 4 * kWriteWarps;  // a contiguous fill starts a group every 16 tokens: every CTA finds one
 constexpr int kSpanThreshold = 512;     // calls with more tokens than this take the span kernel
 template <int D>
-__global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_span_kernel(WriteParams p) {
+__global__ void __launch_bounds__(kWriteWarps * 32, 3) kv_write_fp8_span_kernel(WriteParams p) {
   __shared__ __align__(16) uint8_t stage[kWriteWarps][part_bytes(D, true)];
   __shared__ Group groups[kSpan];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  {
-    const int tok = blockIdx.x * kSpan + warp;
-    if (tok < p.num_tokens) find_group_warp(p, tok, groups[warp], lane);
-    else if (lane == 0) groups[warp].n = 0;
+  for (int w = warp; w < kSpan; w += kWriteWarps) {
+    const int tok = blockIdx.x * kSpan + w;
+    if (tok < p.num_tokens) find_group_warp(p, tok, groups[w], lane);
+    else if (lane == 0) groups[w].n = 0;
   }
   __syncthreads();
   unsigned leaders = 0;

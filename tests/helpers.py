@@ -81,7 +81,7 @@ def cache_to_logical(cache: binding.Cache, heads=None):
         so = binding.scale_offset(cache, 0, 0, 0)                # the 32-byte header: two fp32 scales, 24 zero bytes
         assert binding.scale_offset(cache, 0, 0, 1) == so + 4
         scales = raw[:, :, so:so + 8].copy().view(np.float32)    # [NB, H, 2]
-        return codes, scales, raw[:, :, so + 8:so + 32]
+        return codes, scales, raw[:, :, so + 8:]                  # rest of the header and the granule's padding
     lo = raw[:, :, idx].astype(np.uint32)
     hi = raw[:, :, idx + 1].astype(np.uint32)
     bits = ((hi << 8) | lo) << 16

@@ -52,7 +52,7 @@ def test_layout_is_a_bijection_inside_each_granule(lib, head_dim, dtype):
     gran = lib.coopt_granule_bytes(head_dim, dtype)
     esize = 1 if dtype == binding.KV_FP8_E4M3 else 2
     header = 0                                   # the FP8 header sits behind the codes
-    assert gran == (32 if dtype == binding.KV_FP8_E4M3 else 0) + 2 * 16 * head_dim * esize
+    assert gran == (128 if dtype == binding.KV_FP8_E4M3 else 0) + 2 * 16 * head_dim * esize
     assert lib.coopt_cache_bytes(3, 2, head_dim, dtype) == 3 * 2 * gran
     for blk, h in [(0, 0), (2, 1)]:
         base = (blk * 2 + h) * gran
