@@ -6,7 +6,8 @@ package; the CUDA path shares no code with it.
 Inputs are the cache in logical order plus the block table.  The cache ``kv`` is either
 an array of values [num_blocks, Hkv, 2, 16, D] (the bf16 ablation cache, or an FP8 cache
 already passed through ``kv_cache.dequantise``) or the pair ``(codes, scales)`` of an FP8
-cache, which is dequantised (Eq. 6: dec(code) * scale, exact in float64) as it is read.
+cache (a third entry names the format module when it is not ``e4m3``), which is dequantised
+(Eq. 6: dec(code) * scale, exact in float64) as it is read.
 The computation is the definition, written out per (sequence, query head):
 
   * Eq. 9 / Algorithm 3 phase 1: only blocks 0 .. ceil(t/B)-1 of the sequence are read,
@@ -33,8 +34,9 @@ def gather_kv(kv: np.ndarray, table_row: np.ndarray, length: int, kv_head: int):
     blk = np.asarray(table_row)[pos // BLOCK_SIZE].astype(np.int64)     # Eq. 9: valid blocks only
     off = pos % BLOCK_SIZE
     if isinstance(kv, tuple):                                           # FP8: Eq. 6 on the fly
-        codes, scales = kv
-        return tuple(e4m3.decode(codes[blk, kv_head, w, off, :])
+        codes, scales = kv[0], kv[1]
+        fmt = kv[2] if len(kv) > 2 else e4m3                            # (codes, scales[, format module])
+        return tuple(fmt.decode(codes[blk, kv_head, w, off, :])
                      * scales[blk, kv_head, w].astype(np.float64)[:, None] for w in (0, 1))
     return (kv[blk, kv_head, 0, off, :].astype(np.float64),
             kv[blk, kv_head, 1, off, :].astype(np.float64))

@@ -44,17 +44,20 @@ def new_cache(num_blocks: int, num_kv_heads: int, head_dim: int):
     return codes, scales
 
 
-def _quantise(x: np.ndarray, scale: np.float32) -> np.ndarray:
+def _quantise(x: np.ndarray, scale: np.float32, fmt=e4m3) -> np.ndarray:
     """enc(x / scale) with an fp32 division; a zero scale gives signed zeros."""
     x = x.astype(_F32)
     if not scale > 0:
-        return e4m3.encode(np.copysign(_F32(0.0), x))
-    return e4m3.encode((x / _F32(scale)).astype(_F32))
+        return fmt.encode(np.copysign(_F32(0.0), x))
+    return fmt.encode((x / _F32(scale)).astype(_F32))
 
 
 def kv_write(codes: np.ndarray, scales: np.ndarray, k: np.ndarray, v: np.ndarray,
-             slot_mapping: np.ndarray, heads=None) -> None:
+             slot_mapping: np.ndarray, heads=None, fmt=e4m3) -> None:
     """Apply one write call in place.
+
+    ``fmt`` is the 8-bit format of the codes: ``e4m3`` (the reading the build takes), or ``e5m2``
+    as an ablation of the format the paper leaves open; the scale is amax / fmt.MAX either way.
 
     ``k``, ``v``: float32 [T, Hkv, D] holding bf16-representable values; ``slot_mapping``
     int64 [T].  ``heads`` restricts the work to some kv heads (used to check samples of a
@@ -75,14 +78,14 @@ def kv_write(codes: np.ndarray, scales: np.ndarray, k: np.ndarray, v: np.ndarray
                 x = kv[w][tok, h, :]                              # [n, D]
                 amax = _F32(np.max(np.abs(x)))
                 s_old = _F32(0.0) if fresh else _F32(scales[blk, h, w])
-                s_new = max(s_old, _F32(amax / _F32(e4m3.E4M3_MAX)))
+                s_new = max(s_old, _F32(amax / _F32(fmt.MAX)))
                 if fresh:
                     codes[blk, h, w, others, :] = 0
                 elif s_new > s_old and s_old > 0:
-                    resident = e4m3.decode(codes[blk, h, w, others, :]).astype(_F32)
+                    resident = fmt.decode(codes[blk, h, w, others, :]).astype(_F32)
                     resident = (resident * s_old).astype(_F32)
-                    codes[blk, h, w, others, :] = _quantise(resident, s_new)
-                codes[blk, h, w, off, :] = _quantise(x, s_new)
+                    codes[blk, h, w, others, :] = _quantise(resident, s_new, fmt)
+                codes[blk, h, w, off, :] = _quantise(x, s_new, fmt)
                 scales[blk, h, w] = s_new
 
 
@@ -101,6 +104,6 @@ def kv_write_bf16(values: np.ndarray, k: np.ndarray, v: np.ndarray, slot_mapping
         values[blk, :, w, off, :] = np.asarray(x, dtype=np.float32)[keep]
 
 
-def dequantise(codes: np.ndarray, scales: np.ndarray) -> np.ndarray:
+def dequantise(codes: np.ndarray, scales: np.ndarray, fmt=e4m3) -> np.ndarray:
     """Eq. 6: float64 values of a whole FP8 cache, dec(code) * scale (exact in float64)."""
-    return e4m3.decode(codes) * scales.astype(np.float64)[..., None, None]
+    return fmt.decode(codes) * scales.astype(np.float64)[..., None, None]
