@@ -55,7 +55,10 @@ typedef enum {
   COOPT_ERR_TIMEOUT = -5      /* device side: a bounded wait ran out (workspace word 0)  */
 } coopt_status;
 
-typedef enum { COOPT_KV_FP8_E4M3 = 0, COOPT_KV_BF16 = 1 } coopt_kv_dtype;
+/* COOPT_KV_FP8_E5M2 is an ablation of the FP8 format, which Section 3.1 leaves open: the same granule layout and the
+ * same scale rule with codes in the OCP E5M2 format (5 exponent bits, 2 mantissa bits, saturating at +-57344:
+ * scale = amax / 57344).  Supported by every call except chunked prefill at head_dim 64. */
+typedef enum { COOPT_KV_FP8_E4M3 = 0, COOPT_KV_BF16 = 1, COOPT_KV_FP8_E5M2 = 2 } coopt_kv_dtype;
 
 typedef struct coopt_cache {
   void* data;           /* DEVICE, coopt_cache_bytes() bytes, 32-byte aligned, layout above */

@@ -15,6 +15,7 @@ import torch
 
 KV_FP8_E4M3 = 0
 KV_BF16 = 1
+KV_FP8_E5M2 = 2
 BLOCK_SIZE = 16
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libcoopt.so")

@@ -69,7 +69,7 @@ namespace {
 
 bool cache_shape_ok(int head_dim, int block_size, int dtype) {
   return (head_dim == 64 || head_dim == 128) && block_size == kBlockSize &&
-         (dtype == COOPT_KV_FP8_E4M3 || dtype == COOPT_KV_BF16);
+         (is_fp8(dtype) || dtype == COOPT_KV_BF16);
 }
 
 int check_cache(const coopt_cache* c) {
@@ -127,7 +127,7 @@ extern "C" {
 
 size_t coopt_granule_bytes(int32_t head_dim, int32_t dtype) {
   if (!cache_shape_ok(head_dim, kBlockSize, dtype)) return 0;
-  return granule_bytes(head_dim, dtype == COOPT_KV_FP8_E4M3);
+  return granule_bytes(head_dim, is_fp8(dtype));
 }
 
 size_t coopt_cache_bytes(int32_t num_blocks, int32_t num_kv_heads, int32_t head_dim, int32_t dtype) {
@@ -141,14 +141,14 @@ int64_t coopt_cache_offset(const coopt_cache* c, int32_t block, int32_t kv_head,
   if (block < 0 || block >= c->num_blocks || kv_head < 0 || kv_head >= c->num_kv_heads || which < 0 || which > 1 ||
       token < 0 || token >= kBlockSize || dim < 0 || dim >= c->head_dim)
     return -1;
-  const bool fp8 = c->dtype == COOPT_KV_FP8_E4M3;
+  const bool fp8 = is_fp8(c->dtype);
   const int64_t gran = (static_cast<int64_t>(block) * c->num_kv_heads + kv_head) * granule_bytes(c->head_dim, fp8);
   const int inner = which == 0 ? k_elem_offset(c->head_dim, fp8, token, dim) : v_elem_offset(c->head_dim, fp8, token, dim);
   return gran + part_offset(c->head_dim, fp8, which) + inner;
 }
 
 int64_t coopt_scale_offset(const coopt_cache* c, int32_t block, int32_t kv_head, int32_t which) {
-  if (!c || !cache_shape_ok(c->head_dim, c->block_size, c->dtype) || c->dtype != COOPT_KV_FP8_E4M3) return -1;
+  if (!c || !cache_shape_ok(c->head_dim, c->block_size, c->dtype) || !is_fp8(c->dtype)) return -1;
   if (block < 0 || block >= c->num_blocks || kv_head < 0 || kv_head >= c->num_kv_heads || which < 0 || which > 1) return -1;
   return (static_cast<int64_t>(block) * c->num_kv_heads + kv_head) * granule_bytes(c->head_dim, true) + header_offset(c->head_dim) + 4 * which;
 }
@@ -260,7 +260,7 @@ int coopt_decode_step_planned(const coopt_cache* cache, const void* plan, size_t
                               void* workspace, size_t workspace_bytes, uint32_t flags, void* stream) {
   int rc = check_attention_shapes(cache, q, out, max_blocks_per_seq, batch, num_q_heads);
   if (rc != COOPT_OK) return rc;
-  if (cache->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;         // the bf16 ablation kernel plans for itself
+  if (!is_fp8(cache->dtype)) return COOPT_ERR_UNSUPPORTED;                     // the bf16 ablation kernel plans for itself
   rc = check_plan_args(batch, cache->num_kv_heads, max_blocks_per_seq, chunk_size, plan, plan_bytes_given);
   if (rc != COOPT_OK) return rc;
   const bool append = k_new || v_new || slot_mapping;
@@ -288,7 +288,7 @@ int coopt_decode_layers(const coopt_layer_io* layers, int32_t num_layers, int64_
     const coopt_layer_io& io = layers[l];
     const int rc = check_attention_shapes(io.cache, io.q, io.out, max_blocks_per_seq, batch, num_q_heads);
     if (rc != COOPT_OK) return rc;
-    if (io.cache->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;
+    if (!is_fp8(io.cache->dtype) || io.cache->dtype != c0->dtype) return COOPT_ERR_UNSUPPORTED;
     if (io.cache->num_kv_heads != c0->num_kv_heads || io.cache->head_dim != c0->head_dim || io.cache->num_blocks != c0->num_blocks)
       return COOPT_ERR_INVALID_ARG;                                             // one plan serves every layer
     const bool append = io.k_new || io.v_new || io.slot_mapping;
@@ -380,7 +380,7 @@ int coopt_decode_step_host(const coopt_cache* cache, const void* step_inputs_hos
   rc = check_attention_args(cache, dev + s.q, dev + s.out, reinterpret_cast<const int32_t*>(dev + s.block_table), max_blocks_per_seq,
                             reinterpret_cast<const int32_t*>(dev + s.context_lens), batch, num_q_heads);
   if (rc != COOPT_OK) return rc;
-  if (cache->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;
+  if (!is_fp8(cache->dtype)) return COOPT_ERR_UNSUPPORTED;
   rc = check_plan_args(batch, hkv, max_blocks_per_seq, 0, plan, plan_bytes_given);
   if (rc != COOPT_OK) return rc;
   if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, hkv, d, max_blocks_per_seq, 0, batch)) return COOPT_ERR_WORKSPACE;

@@ -15,6 +15,8 @@ constexpr int kFp8Header = 32;     // bytes behind the codes of an FP8 granule t
 constexpr int kFp8Tail = 128;      // bytes behind the codes that the granule occupies: the header and padding, so that
                                    // granules start on 128-byte lines and no line is shared by two writers
 constexpr float kE4m3Max = 448.0f;
+constexpr float kE5m2Max = 57344.0f;
+inline bool is_fp8(int dtype) { return dtype == COOPT_KV_FP8_E4M3 || dtype == COOPT_KV_FP8_E5M2; }
 
 // ---- cache layout ---------------------------------------------------------------------------
 // A granule holds 16 tokens x D of K and of V for one (block, kv head).
@@ -84,6 +86,20 @@ __device__ __forceinline__ uint32_t f32_to_e4m3(float x) {
   asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(0.0f), "f"(x));
   return d & 0xFFu;
 }
+
+// fp32 -> one E5M2 code, round to nearest even, saturating to +-57344.
+__device__ __forceinline__ uint32_t f32_to_e5m2(float x) {
+  uint16_t d;
+  asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(0.0f), "f"(x));
+  return d & 0xFFu;
+}
+// An E5M2 code is the upper byte of the half-precision number of the same value.
+__device__ __forceinline__ float e5m2_to_f32(uint32_t code) {
+  return __half2float(__ushort_as_half(static_cast<unsigned short>((code & 0xFFu) << 8)));
+}
+// Two E5M2 codes (bytes 0, 1 of `w`, or bytes 2, 3) -> two f16 (exact).
+__device__ __forceinline__ uint32_t e5m2x2_to_f16x2_lo(uint32_t w) { return __byte_perm(w, 0u, 0x1404); }
+__device__ __forceinline__ uint32_t e5m2x2_to_f16x2_hi(uint32_t w) { return __byte_perm(w, 0u, 0x3424); }
 
 __device__ __forceinline__ float e4m3_to_f32(uint32_t code) {
   const uint32_t h2 = e4m3x2_to_f16x2_lo(code & 0xFFu);

@@ -432,6 +432,7 @@ static void fill_decode_params(DecodeParams& p, const coopt_cache* c, const void
   p.num_kv_heads = c->num_kv_heads;
   p.group = num_q_heads / c->num_kv_heads;
   p.num_blocks = c->num_blocks;
+  p.kv_e5m2 = c->dtype == COOPT_KV_FP8_E5M2 ? 1 : 0;
   p.sm_scale_log2 = sm_scale * kLog2e;
   p.planned_ctas = planned_ctas;
   p.chunk_blocks = chunk_size / kBlockSize;
@@ -479,7 +480,7 @@ int launch_paged_decode(const coopt_cache* c, const void* q, void* out, const in
   DecodeParams p;
   fill_decode_params(p, c, q, out, block_table, max_blocks_per_seq, context_lens, batch, num_q_heads, sm_scale, chunk_size,
                      cu_q_lens, workspace, planned_ctas);
-  if (c->dtype != COOPT_KV_FP8_E4M3)
+  if (!is_fp8(c->dtype))
     return c->head_dim == 128 ? launch_one<128>(p, planned_ctas, stream) : launch_one<64>(p, planned_ctas, stream);
   void* plan = static_cast<uint8_t*>(workspace) + partials_bytes(planned_ctas, p.group, c->head_dim, batch, num_q_heads, p.max_chunks);
   const int rc = launch_decode_plan(block_table, max_blocks_per_seq, context_lens, batch, c->num_kv_heads, c->num_blocks, chunk_size,

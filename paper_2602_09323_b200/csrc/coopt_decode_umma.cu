@@ -392,7 +392,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             tc_fence_after();
             const uint64_t dk = desc_k + ((stage * C::kStageBytes) >> 4);
 #pragma unroll
-            for (int ks = 0; ks < kKSteps; ++ks) umma_f8(tmem + 16 * buf, dk + ks * 16, dq + ks * 16, umma_idesc(16), ks > 0);
+            for (int ks = 0; ks < kKSteps; ++ks) umma_f8(tmem + 16 * buf, dk + ks * 16, dq + ks * 16, umma_idesc(16, p.kv_e5m2), ks > 0);
             umma_commit(&bar_sfull[buf]);
             COOPT_TRACE_CYCLES(p.trace, kTrLogitsTileBase + static_cast<int>(tile_no), tile_no < 32);
           }
@@ -415,7 +415,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             const uint64_t dv = desc_v + ((stage * C::kStageBytes) >> 4), dp = desc_p + ((buf * C::kPBytes) >> 4);
             const int nks = (min(kTileBlocks, n - k0) + 1) >> 1;      // 32 tokens (two granules) per instruction
             for (int ks = 0; ks < nks; ++ks)
-              umma_f8(tmem_o + NP * buf, dv + ks * ((2 * C::kPart) >> 4), dp + ks * 16, umma_idesc(NP), ks > 0 ? 1u : 0u);
+              umma_f8(tmem_o + NP * buf, dv + ks * ((2 * C::kPart) >> 4), dp + ks * 16, umma_idesc(NP, p.kv_e5m2), ks > 0 ? 1u : 0u);
             umma_commit(&bar_empty[stage]);     // the stage is free again and the tile's product is in its output buffer
             COOPT_TRACE_CYCLES(p.trace, kTrLastPv, true);
             COOPT_TRACE_CYCLES(p.trace, kTrPvTileBase + static_cast<int>(tile_no), tile_no < 32);
@@ -707,7 +707,8 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
             if (blk >= p.num_blocks) continue;
             Group gr;
             gr.n = 1; gr.blk = static_cast<int>(blk); gr.tok[0] = sg.b; gr.off[0] = static_cast<int>(slot % kBlockSize);
-            write_part<D, 1>(wp, gr, sg.g, which, write_stage + wq * (kBlockSize * D), lane);
+            if (p.kv_e5m2) write_part<D, 1, true>(wp, gr, sg.g, which, write_stage + wq * (kBlockSize * D), lane);
+            else write_part<D, 1, false>(wp, gr, sg.g, which, write_stage + wq * (kBlockSize * D), lane);
           }
         }
         // the granules are read next by the copy engine: order this warp's global (and staging) writes before it

@@ -93,6 +93,7 @@ struct DecodeParams {
   int max_blocks_per_seq;
   int batch, num_q_heads, num_kv_heads, group;
   int num_blocks;
+  int kv_e5m2;             // 1: the cache codes are E5M2 (the format ablation), 0: E4M3
   float sm_scale_log2;     // sm_scale * log2(e)
   int planned_ctas;        // P
   int chunk_blocks;        // 0 = decode mode

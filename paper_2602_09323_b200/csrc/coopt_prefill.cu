@@ -414,7 +414,8 @@ int launch_paged_prefill(const coopt_cache* c, const void* q, void* out, const i
                          const int32_t* block_table, int32_t max_blocks_per_seq, const int32_t* context_lens,
                          int32_t batch, int32_t num_q_heads, int32_t total_q, int32_t causal, float sm_scale,
                          void* workspace, cudaStream_t stream) {
-  if (c->dtype != COOPT_KV_FP8_E4M3) return COOPT_ERR_UNSUPPORTED;
+  if (!is_fp8(c->dtype)) return COOPT_ERR_UNSUPPORTED;
+  if (c->dtype == COOPT_KV_FP8_E5M2 && c->head_dim != 128) return COOPT_ERR_UNSUPPORTED;   // the E5M2 ablation: tcgen05 kernel only
   if (num_q_heads / c->num_kv_heads > kPfRows) return COOPT_ERR_UNSUPPORTED;   // a tile holds at least one query token of every head of the group
   // head_dim 128: the tcgen05 kernel; head_dim 64: the mma.sync kernel of this file
   if (c->head_dim == 128)

@@ -62,6 +62,7 @@ struct PrefillUmmaParams {
   int num_blocks;
   int tile_queries;        // query tokens per CTA = 128 / group
   int causal;
+  int kv_e5m2;             // the cache codes are E5M2 (the format ablation)
   float sm_scale_log2;
   int* status;
 };
@@ -327,7 +328,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         for (int term = 0; term < 2; ++term)
 #pragma unroll
           for (int ks = 0; ks < D / 32; ++ks)
-            umma_f8(tmem + 128 * buf, desc_q + ((term * C::kOperand) >> 4) + ks * 16, dk + ks * 16, umma_idesc(128), (term | ks) != 0);
+            umma_f8(tmem + 128 * buf, desc_q + ((term * C::kOperand) >> 4) + ks * 16, dk + ks * 16, umma_idesc(128, 0, p.kv_e5m2), (term | ks) != 0);
         umma_commit(&bar_sfull[buf]);
       }
       if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
@@ -446,8 +447,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
           for (int j = 0; j < 4; ++j) {
             const int left = keep - 4 * j;
             const uint32_t w = cw[j] & (left >= 4 ? 0xFFFFFFFFu : (left <= 0 ? 0u : (1u << (8 * left)) - 1u));
-            vw[2 * j] = e4m3x2_to_f16x2_lo(w);
-            vw[2 * j + 1] = e4m3x2_to_f16x2_hi(w);
+            vw[2 * j] = p.kv_e5m2 ? e5m2x2_to_f16x2_lo(w) : e4m3x2_to_f16x2_lo(w);
+            vw[2 * j + 1] = p.kv_e5m2 ? e5m2x2_to_f16x2_hi(w) : e4m3x2_to_f16x2_hi(w);
           }
         }
         *reinterpret_cast<uint4*>(vrow + (2 * c) * 128) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
@@ -540,6 +541,7 @@ int launch_paged_prefill_umma(const coopt_cache* c, const void* q, void* out, co
   p.num_blocks = c->num_blocks;
   p.tile_queries = 128 / p.group;
   p.causal = causal;
+  p.kv_e5m2 = c->dtype == COOPT_KV_FP8_E5M2 ? 1 : 0;
   p.sm_scale_log2 = sm_scale * kPuLog2e;
   p.status = static_cast<int*>(workspace);
   const long long tiles = static_cast<long long>(total_q) / p.tile_queries + batch;   // every sequence adds at most one partly filled tile

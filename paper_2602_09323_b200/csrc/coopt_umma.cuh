@@ -19,8 +19,10 @@ __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo, uint
          (static_cast<uint64_t>(sbo >> 4) << 32) | (1ull << 46);
 }
 // Instruction descriptor: E4M3 x E4M3 -> fp32, both operands K-major, M = 128, N = n.
-__device__ __forceinline__ constexpr uint32_t umma_idesc(int n) {
-  return (1u << 4) | (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
+// a_e5m2 / b_e5m2: the A (B) operand holds E5M2 codes instead (kind::f8f6f4 takes a format per operand).
+__device__ __forceinline__ constexpr uint32_t umma_idesc(int n, int a_e5m2 = 0, int b_e5m2 = 0) {
+  return (1u << 4) | (static_cast<uint32_t>(a_e5m2) << 7) | (static_cast<uint32_t>(b_e5m2) << 10) |
+         (static_cast<uint32_t>(n >> 3) << 17) | (static_cast<uint32_t>(128 >> 4) << 24);
 }
 __device__ __forceinline__ void umma_f8(uint32_t d_tmem, uint64_t a, uint64_t b, uint32_t idesc, uint32_t accumulate) {
   asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p;\n}"

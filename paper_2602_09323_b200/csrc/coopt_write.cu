@@ -13,7 +13,7 @@ constexpr int kWriteWarps = 2 * kWriteHeads;   // FP8: one warp per (kv head, K 
 
 // FP8, few tokens (decode steps): one CTA per (token, kWriteHeads kv heads), one warp per
 // (kv head, K | V); CTAs whose token leads no group leave at once.
-template <int D>
+template <int D, bool kE5m2>
 __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WriteParams p) {
   __shared__ __align__(16) uint8_t stage[kWriteWarps][part_bytes(D, true)];
   __shared__ Group group;
@@ -23,7 +23,7 @@ __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WritePar
   if (group.n == 0) return;
   const int h = blockIdx.y * kWriteHeads + (warp >> 1);
   if (h >= p.num_kv_heads) return;
-  write_part<D>(p, group, h, warp & 1, stage[warp], lane);
+  write_part<D, kBlockSize, kE5m2>(p, group, h, warp & 1, stage[warp], lane);
 }
 
 // FP8, many tokens (prefill chunks, bulk fills): one CTA per (kSpan consecutive tokens, kWriteHeads
@@ -31,7 +31,7 @@ __global__ void __launch_bounds__(kWriteWarps * 32) kv_write_fp8_kernel(WritePar
 // (one per 16 tokens in a contiguous fill) are then served by all warps.
 constexpr int kSpan = 4 * kWriteWarps;  // a contiguous fill starts a group every 16 tokens: every CTA finds one
 constexpr int kSpanThreshold = 512;     // calls with more tokens than this take the span kernel
-template <int D>
+template <int D, bool kE5m2>
 __global__ void __launch_bounds__(kWriteWarps * 32, 3) kv_write_fp8_span_kernel(WriteParams p) {
   __shared__ __align__(16) uint8_t stage[kWriteWarps][part_bytes(D, true)];
   __shared__ Group groups[kSpan];
@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(kWriteWarps * 32, 3) kv_write_fp8_span_kernel(
   while (leaders) {
     const int w = __ffs(leaders) - 1;
     leaders &= leaders - 1;
-    write_part<D>(p, groups[w], h, warp & 1, stage[warp], lane);
+    write_part<D, kBlockSize, kE5m2>(p, groups[w], h, warp & 1, stage[warp], lane);
   }
 }
 
@@ -95,7 +95,7 @@ int launch_kv_write(const coopt_cache* c, const void* k, const void* v, int64_t 
   p.num_kv_heads = c->num_kv_heads;
   p.num_blocks = c->num_blocks;
   const dim3 block(kWriteWarps * 32);
-  const bool fp8 = c->dtype == COOPT_KV_FP8_E4M3;
+  const bool fp8 = is_fp8(c->dtype), e5m2 = c->dtype == COOPT_KV_FP8_E5M2;
   // FP8: a CTA serves kWriteHeads kv heads (two warps each); bf16: kWriteWarps heads (one warp each)
   const int heads_per_cta = fp8 ? kWriteHeads : kWriteWarps;
   const int head_ctas = (c->num_kv_heads + heads_per_cta - 1) / heads_per_cta;
@@ -103,12 +103,16 @@ int launch_kv_write(const coopt_cache* c, const void* k, const void* v, int64_t 
   const dim3 span_grid((num_tokens + kSpan - 1) / kSpan, head_ctas);
   const bool span = fp8 && num_tokens > kSpanThreshold;
   if (c->head_dim == 128) {
-    if (span) kv_write_fp8_span_kernel<128><<<span_grid, block, 0, stream>>>(p);
-    else if (fp8) kv_write_fp8_kernel<128><<<grid, block, 0, stream>>>(p);
+    if (span && e5m2) kv_write_fp8_span_kernel<128, true><<<span_grid, block, 0, stream>>>(p);
+    else if (span) kv_write_fp8_span_kernel<128, false><<<span_grid, block, 0, stream>>>(p);
+    else if (e5m2) kv_write_fp8_kernel<128, true><<<grid, block, 0, stream>>>(p);
+    else if (fp8) kv_write_fp8_kernel<128, false><<<grid, block, 0, stream>>>(p);
     else kv_write_bf16_kernel<128><<<grid, block, 0, stream>>>(p);
   } else {
-    if (span) kv_write_fp8_span_kernel<64><<<span_grid, block, 0, stream>>>(p);
-    else if (fp8) kv_write_fp8_kernel<64><<<grid, block, 0, stream>>>(p);
+    if (span && e5m2) kv_write_fp8_span_kernel<64, true><<<span_grid, block, 0, stream>>>(p);
+    else if (span) kv_write_fp8_span_kernel<64, false><<<span_grid, block, 0, stream>>>(p);
+    else if (e5m2) kv_write_fp8_kernel<64, true><<<grid, block, 0, stream>>>(p);
+    else if (fp8) kv_write_fp8_kernel<64, false><<<grid, block, 0, stream>>>(p);
     else kv_write_bf16_kernel<64><<<grid, block, 0, stream>>>(p);
   }
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;

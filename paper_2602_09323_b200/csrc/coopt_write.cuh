@@ -97,6 +97,17 @@ __device__ __forceinline__ uint32_t f32x2_to_e4m3x2(float lo, float hi) {
   return d;
 }
 
+// Two fp32 values -> two E5M2 codes (lo in the low byte), round to nearest even, saturating.
+__device__ __forceinline__ uint32_t f32x2_to_e5m2x2(float lo, float hi) {
+  uint16_t d;
+  asm("cvt.rn.satfinite.e5m2x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+template <bool kE5m2>
+__device__ __forceinline__ uint32_t f32x2_to_codes(float lo, float hi) {
+  return kE5m2 ? f32x2_to_e5m2x2(lo, hi) : f32x2_to_e4m3x2(lo, hi);
+}
+
 // kPerLane consecutive bf16 values of one row as packed pairs; one load when the row is aligned for it.
 template <int kPerLane, bool kVec>
 __device__ __forceinline__ void load_row(const __nv_bfloat16* row, uint32_t (&w)[kPerLane / 2]) {
@@ -125,7 +136,8 @@ __device__ __forceinline__ float row_elem(const uint32_t (&w)[kWords], int e) {
 // resident codes; its V part goes from registers straight to memory.
 // kTok bounds the group's size: 16 for the write kernels, 1 for the fused decode step (one new token per
 // sequence); the arithmetic is the same instruction for instruction, so both give the same bytes.
-template <int D, int kTok = kBlockSize>
+// kE5m2 selects the code format (the E5M2 ablation): encoder, decoder and the format's largest value.
+template <int D, int kTok = kBlockSize, bool kE5m2 = false>
 __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g, int h, int which, uint8_t* st, int lane) {
   constexpr int kPart = part_bytes(D, true);          // 16 * D bytes
   constexpr int kPerLane = D / 32;                    // dims handled by one lane
@@ -173,14 +185,14 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
 #pragma unroll
     for (int e = 0; e < kPerLane; ++e) amax = fmaxf(amax, t < n ? fabsf(row_elem(raw[t], e)) : 0.0f);
   amax = warp_max(amax);
-  const float s_new = fmaxf(s_old, __fdiv_rn(amax, kE4m3Max));
+  const float s_new = fmaxf(s_old, __fdiv_rn(amax, kE5m2 ? kE5m2Max : kE4m3Max));
   __syncwarp();
 
   // scale grew on a block that already holds tokens: re-express every resident code
   if (!fresh && s_new > s_old && s_old > 0.0f) {
     for (int i = lane; i < kPart; i += 32) {
-      const float val = __fmul_rn(e4m3_to_f32(st[i]), s_old);
-      st[i] = static_cast<uint8_t>(f32_to_e4m3(__fdiv_rn(val, s_new)));
+      const float val = __fmul_rn(kE5m2 ? e5m2_to_f32(st[i]) : e4m3_to_f32(st[i]), s_old);
+      st[i] = static_cast<uint8_t>(kE5m2 ? f32_to_e5m2(__fdiv_rn(val, s_new)) : f32_to_e4m3(__fdiv_rn(val, s_new)));
     }
     __syncwarp();
   }
@@ -211,8 +223,8 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
         uint32_t w[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
-          w[q] = f32x2_to_e4m3x2(scaled((4 * q) % kTok, e), scaled((4 * q + 1) % kTok, e)) |
-                 (f32x2_to_e4m3x2(scaled((4 * q + 2) % kTok, e), scaled((4 * q + 3) % kTok, e)) << 16);
+          w[q] = f32x2_to_codes<kE5m2>(scaled((4 * q) % kTok, e), scaled((4 * q + 1) % kTok, e)) |
+                 (f32x2_to_codes<kE5m2>(scaled((4 * q + 2) % kTok, e), scaled((4 * q + 3) % kTok, e)) << 16);
         *reinterpret_cast<uint4*>(part + v_elem_offset(D, true, 0, lane * kPerLane + e)) = make_uint4(w[0], w[1], w[2], w[3]);
       }
     } else {
@@ -225,13 +237,13 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
             // the lane's dims are consecutive bytes of a K row
             uint8_t* dst = st + k_elem_offset(D, true, off, lane * kPerLane);
             if constexpr (kPerLane == 4)
-              *reinterpret_cast<uint32_t*>(dst) = f32x2_to_e4m3x2(scaled(t, 0), scaled(t, 1)) | (f32x2_to_e4m3x2(scaled(t, 2), scaled(t, 3)) << 16);
+              *reinterpret_cast<uint32_t*>(dst) = f32x2_to_codes<kE5m2>(scaled(t, 0), scaled(t, 1)) | (f32x2_to_codes<kE5m2>(scaled(t, 2), scaled(t, 3)) << 16);
             else
-              *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(f32x2_to_e4m3x2(scaled(t, 0), scaled(t, 1)));
+              *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(f32x2_to_codes<kE5m2>(scaled(t, 0), scaled(t, 1)));
           } else {
 #pragma unroll
             for (int e = 0; e < kPerLane; ++e)
-              st[v_elem_offset(D, true, off, lane * kPerLane + e)] = static_cast<uint8_t>(f32_to_e4m3(scaled(t, e)));
+              st[v_elem_offset(D, true, off, lane * kPerLane + e)] = static_cast<uint8_t>(kE5m2 ? f32_to_e5m2(scaled(t, e)) : f32_to_e4m3(scaled(t, e)));
           }
         }
       }

@@ -167,6 +167,37 @@ def uniform_lengths(batch: int, lo: int, hi: int, seed: int) -> List[int]:
     return [int(x) for x in torch.randint(lo, hi + 1, (batch,), generator=gen)]
 
 
+# --- SkipSet policies (Eq. 5): which tokens of a write call the caller marks as skipped ---------------------
+# The paper filters tokens whose slot is negative or in a SkipSet of "redundant" slots and never says how
+# the set is built.  Two policies that a serving stack meets are given here as slot-mapping generators; a
+# skipped token is a negative slot, which is all the library ever tests.
+
+def skip_padding(slot_mapping: torch.Tensor, row_lens: Sequence[int], padded_len: int) -> torch.Tensor:
+    """Padding tokens: a batch of write rows laid out as ``len(row_lens)`` sequences of ``padded_len`` rows
+    each, of which only the first ``row_lens[b]`` are real.  The padding rows get slot -1."""
+    out = slot_mapping.clone()
+    for b, n in enumerate(row_lens):
+        out[b * padded_len + n:(b + 1) * padded_len] = -1
+    return out
+
+
+def share_prefix(w: Workload, donor: int, taker: int, prefix_tokens: int) -> Workload:
+    """Duplicate prefix tokens: sequence ``taker`` starts with the same ``prefix_tokens`` tokens (a multiple of the
+    block size) as sequence ``donor``, whose blocks already hold them.  The taker's block table points at the
+    donor's blocks for the prefix, its own K/V rows of the prefix are made equal to the donor's, and their
+    slots become -1: writing them again would be redundant."""
+    assert prefix_tokens % BLOCK_SIZE == 0 and prefix_tokens <= min(w.context_lens[donor], w.context_lens[taker])
+    nb = prefix_tokens // BLOCK_SIZE
+    table = w.block_table.clone()
+    table[taker, :nb] = table[donor, :nb]
+    k, v, slots = w.k.clone(), w.v.clone(), w.slot_mapping.clone()
+    d0, t0 = w.kv_offsets[donor], w.kv_offsets[taker]
+    k[t0:t0 + prefix_tokens] = k[d0:d0 + prefix_tokens]
+    v[t0:t0 + prefix_tokens] = v[d0:d0 + prefix_tokens]
+    slots[t0:t0 + prefix_tokens] = -1
+    return dataclasses.replace(w, block_table=table, k=k, v=v, slot_mapping=slots)
+
+
 # --- the five named configurations -------------------------------------------------------------
 
 def config_tiny(seed: int = 0, **kw) -> Workload:

@@ -76,7 +76,7 @@ def cache_to_logical(cache: binding.Cache, heads=None):
     if heads is not None:
         raw = raw[:, heads]
     idx = granule_index_map(cache)
-    if cache.dtype == binding.KV_FP8_E4M3:
+    if cache.dtype in (binding.KV_FP8_E4M3, binding.KV_FP8_E5M2):
         codes = raw[:, :, idx]                                   # [NB, H, 2, 16, D]
         so = binding.scale_offset(cache, 0, 0, 0)                # the 32-byte header: two fp32 scales, 24 zero bytes
         assert binding.scale_offset(cache, 0, 0, 1) == so + 4
@@ -88,14 +88,17 @@ def cache_to_logical(cache: binding.Cache, heads=None):
     return bits.view(np.float32)
 
 
-def oracle_fp8_cache(w, calls=None, heads=None):
+def oracle_fp8_cache(w, calls=None, heads=None, fmt=None):
     """Oracle cache for workload ``w`` filled by the given list of calls, each a (row_start, row_stop)
     pair or an array of row indices (default: one call with every token)."""
     codes, scales = kv_cache.new_cache(w.num_blocks, w.num_kv_heads, w.head_dim)
     k, v, slots = w.k.float().numpy(), w.v.float().numpy(), w.slot_mapping.numpy()
     for call in (calls or [(0, k.shape[0])]):
         rows = slice(*call) if isinstance(call, tuple) else np.asarray(call, dtype=np.int64)
-        kv_cache.kv_write(codes, scales, k[rows], v[rows], slots[rows], heads=heads)
+        if fmt is None:
+            kv_cache.kv_write(codes, scales, k[rows], v[rows], slots[rows], heads=heads)
+        else:
+            kv_cache.kv_write(codes, scales, k[rows], v[rows], slots[rows], heads=heads, fmt=fmt)
     return codes, scales
 
 
