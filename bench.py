@@ -211,13 +211,24 @@ def run_other_workload(args):
     ws = binding.new_workspace(B, Hq, Hkv, Dh, w.block_table.shape[1], chunk, total_q)
     out = torch.empty_like(q)
 
+    # FP8 decode-style configurations go through the planned calls, as a serving loop would: one plan per layer here
+    # (every layer cache of this benchmark has a block placement of its own), made outside the timed launches' event
+    # pairs; the append of a serving step rides in the attention launch.
+    planned = dtype == binding.KV_FP8_E4M3 and name != "chunked_prefill"
+    plans = [binding.decode_plan(t, lens, Hkv, c.num_blocks, chunk if name == "long_context" else 0) for c, t, _ in layers] if planned else None
+    fused = planned and new_per_seq == 1
+
     def step(i, ev=None):
         cache, table, slots_new = layers[i % n_layers]
-        if new_per_seq:
+        if new_per_seq and not fused:
             binding.kv_write(cache, k_new, v_new, slots_new)
         if ev:
             ev[0].record()
-        if chunk:
+        if planned:
+            binding.decode_step_planned(cache, plans[i % n_layers], q, table.shape[1], w.sm_scale, ws,
+                                        k_new if fused else None, v_new if fused else None, slots_new if fused else None,
+                                        chunk_size=chunk if name == "long_context" else 0, out=out)
+        elif chunk:
             binding.paged_chunked(cache, q, cu, table, lens, chunk, True, w.sm_scale, ws, out=out)
         else:
             binding.paged_decode(cache, q, table, lens, w.sm_scale, ws, out=out)
@@ -280,7 +291,7 @@ def run_other_workload(args):
             "dtype": "bf16" if esize == 2 else "fp8_e4m3 cache, fp32 accumulate", "data": "synthetic",
             "config": {"workload": name, "batch": B, "context_tokens": tokens, "layers_rotated": n_layers,
                        "l2": "layer caches visited round-robin"},
-            "gpu_launches": steps * (2 if new_per_seq else 1), "clocks": sampler.summary(), "e2e": None, "roofline": roofline,
+            "gpu_launches": steps * (2 if new_per_seq and not fused else 1), "clocks": sampler.summary(), "e2e": None, "roofline": roofline,
             "cpu_baseline": None}
     print(json.dumps(line), flush=True)
 
@@ -333,6 +344,10 @@ def main():
     ap.add_argument("--layers", type=int, default=8, help="layer caches the steps rotate over (one plan per pass over them)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="budget of the CPU-baseline leg")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-graph", action="store_true",
+                    help="launch every step from the host instead of replaying a CUDA graph of one pass over the layer caches")
+    ap.add_argument("--roofline-launches", type=int, default=2000,
+                    help="launches of the kernel-timing loop behind the timed region (fewer under a profiler)")
     ap.add_argument("--workload", default="llama13b_decode",
                     choices=["llama13b_decode", "llama13b_40layers", "mha_bf16_ablation", "mixed_serving", "long_context",
                              "chunked_prefill", "kv_write_fill"],
@@ -404,6 +419,36 @@ def main():
     torch.cuda.synchronize()
     assert binding.workspace_status(ws) == 0
 
+    # One pass over the layer caches (the plan, then one fused step per cache) as a CUDA graph: what a serving loop
+    # replays every model step.  Steps that do not fill a whole pass are launched from the host.
+    graph = None
+    if not args.no_graph:
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            for i in range(NL):
+                step(i)                                   # first use on this stream, outside the capture
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for i in range(NL):
+                    step(i)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        assert binding.workspace_status(ws) == 0
+
+    def run_steps(n):
+        done = 0
+        if graph is not None:
+            while done + NL <= n:
+                graph.replay()
+                done += NL
+        for i in range(done, n):
+            step(i)
+
     # ---- timed region: exactly K steps between one pair of CUDA events on the launching stream ------------
     start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local, period_s=0.002)
@@ -412,8 +457,7 @@ def main():
     torch.cuda.synchronize()
     sampler.start()
     start.record()
-    for i in range(args.steps):
-        step(i)
+    run_steps(args.steps)
     stop.record()
     torch.cuda.synchronize()
     if world > 1:
@@ -424,7 +468,7 @@ def main():
 
     # ---- the dominant kernel, timed live (the clock sampler keeps running): the fused step's launches back to
     # back between one pair of events (no plan launches in between), and one launch at a time between event pairs
-    n_b2b = 2000
+    n_b2b = max(8, args.roofline_launches)
     b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     binding.decode_plan(table, lens, HKV, base.num_blocks, plan=plan)
     torch.cuda.synchronize()
@@ -434,7 +478,7 @@ def main():
     b1.record()
     torch.cuda.synchronize()
     kernel_b2b_ms = b0.elapsed_time(b1) / n_b2b
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(200)]
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(max(4, n_b2b // 10))]
     for i, (e0, e1) in enumerate(pairs):
         e0.record()
         binding.decode_step_planned(caches[i % NL], plan, q, max_blocks, base.sm_scale, ws, k_new, v_new, s_new, out=out)
@@ -513,7 +557,9 @@ def main():
             "config": {"workload": WORKLOAD, "layers_rotated": NL,
                        "l2": "inputs larger than L2: %d layer caches of %.0f MB visited round-robin" % (NL, algo / 1e6),
                        "step": "coopt_decode_step_planned (one launch: the new token of every sequence written, then attention); "
-                               "coopt_decode_plan once per pass over the layer caches, inside the timed region"},
+                               "coopt_decode_plan once per pass over the layer caches, inside the timed region",
+                       "launch": "host launches" if graph is None else
+                                 "a CUDA graph of one pass over the layer caches (plan + %d steps) replayed; the remainder from the host" % NL},
             "gpu_launches": args.steps + (args.steps + NL - 1) // NL, "clocks": clocks, "clocks_timed_region": region_clocks,
             "e2e": e2e, "roofline": roofline, "cpu_baseline": cpu}
     print(json.dumps(line), flush=True)

@@ -4,34 +4,42 @@
 //
 // A CTA owns one (sequence, kv head, tile of consecutive query tokens).  Its 128 rows are the (query
 // token, query head of the group) pairs of the tile, so the K/V stream of the kv head is fetched once
-// for all G heads (Algorithm 2).  The E4M3 codes of the cache feed tcgen05.mma kind::f8f6f4 as they are:
-//     S [128 rows x 128 keys] = Q  [128 x D] . Ktile^T      kind::f8f6f4: Q as two exact E4M3 terms of the bf16 query
+// for all G heads (Algorithm 2).
+//     S [128 rows x 128 keys] = Q  [128 x D] . Ktile^T      kind::f8f6f4: the cache codes as they are, Q as two exact
+//                                                            E4M3 terms of the bf16 query
 //     O [128 rows x D]       += P  [128 x 128 keys] . Vtile  kind::f16: P rounded once to f16, the V codes widened to f16 (exact)
 // with fp32 accumulators in tensor memory.  The K scale of a block multiplies the logits of its 16 keys,
 // the V scale is folded into the probabilities.  (Carrying P as E4M3 terms instead, three per probability for
 // the same 11 bits, kept the V codes as they are but cost five conversions per pair of probabilities on the
-// SM's conversion pipe, which then bounded the kernel; widening V costs one conversion per pair of codes and
-// a tile of V is a sixteenth of a tile of P per query row.)
+// SM's conversion pipe; widening V costs one conversion per pair of codes, and a tile of V is a sixteenth of a
+// tile of P per query row.)
 //
-// The context is walked twice, 128 keys (eight cache blocks) at a time.  The first walk fetches K only and
-// leaves every row's maximum logit (and the largest V scale); the second recomputes the logits, so every
-// probability is exp(s - final maximum) <= 1 and the output accumulator in tensor memory is never
-// rescaled.  The second product over K costs a third more tensor work and K traffic (out of L2), and
-// removes the read-modify-write of 128 x 128 accumulators whenever a maximum moves.
+// The context is walked once, 128 keys (eight cache blocks) at a time; even tiles go to softmax team 0, odd
+// tiles to team 1, and each team keeps an online softmax of its own for all 128 rows: a reference maximum per
+// row, the sum of the exponentials taken against it, and an output accumulator of its own in tensor memory.
+// The reference is lazy: a probability may exceed one by up to 2^8 before its row's reference is moved up to
+// the row's maximum (and a V scale may exceed the team's reference scale by up to 2^4), because moving a
+// reference means reading, scaling and writing back the row's 128 accumulators; f16 probabilities have room
+// for that factor, and after the first tiles a reference hardly ever moves.  At the end the two teams'
+// results are merged like two split-KV pieces.  Per tile the tensor core does 8 instructions for the logits
+// and 8 for P V; nothing is computed twice.  (An earlier version walked the context twice, row maxima first,
+// so that nothing was ever rescaled: a third more tensor work, every tile's logits read and scaled twice by
+// the teams, and a team idle while its own P V instructions ran.)
 //
 // Warp roles (608 threads):
-//   warps 0-7, 8-15  two softmax teams, even and odd tiles.  Two threads of a team share row r: warps 0-3 of
-//               the team take the tile's first four cache blocks, warps 4-7 the last four; a thread reads its
-//               row's logits from tensor memory 16 at a time (one cache block: one pair of scales), and
-//               maxima and sums are exchanged only at the end of a walk;
-//   warp 16     copies: gather requests over the tensor map of the cache (K parts, V parts, headers of
-//               four granules each) into four slots of 16 KB + 256 B.  The first walk uses all four for K
-//               tiles (and their scales); in the second walk two take K tiles, freed as soon as the logits
-//               are computed, and two take V tiles and the scales, freed as soon as the tile's team has widened
-//               the codes into its f16 operand;
+//   warps 0-7, 8-15  two softmax teams.  Two threads of a team share row r: warps 0-3 of the team take the
+//               tile's first four cache blocks, warps 4-7 the last four.  A tile's logits are read from tensor
+//               memory twice: a first pass for the row's maximum, which both threads of a row make over the whole
+//               row (so that they agree on the reference without meeting) and which touches none of the team's
+//               operand buffers, so it runs while the P V instructions of the team's tile before are still in
+//               flight; and a second pass for the probabilities of the thread's own blocks;
+//   warp 16     copies: gather requests over the tensor map of the cache into two slots for K tiles, freed as
+//               soon as the logits are computed, and two slots for V tiles with the tile's scales, freed as
+//               soon as the team has widened the codes into its f16 operand;
 //   warp 17     one lane issues the S instructions; warp 18 one lane issues the P V instructions.
 // Every wait is bounded; a wait that runs out is reported in the status word and all roles leave through
 // the common exit, which frees the tensor memory.
+#include "coopt_trace.cuh"
 #include "coopt_umma.cuh"
 
 namespace coopt {
@@ -46,10 +54,10 @@ constexpr int kPuThreads = 608;
 constexpr int kPuTileBlocks = 8;
 constexpr int kPuTileKeys = kPuTileBlocks * kBlockSize;   // 128
 constexpr int kPuD = 128;
-constexpr int kPuSlots = 4;                                // of the copy ring
-constexpr int kPuKSlots = 2, kPuVSlots = 2;               // second walk: slots 0-1 take K tiles, slots 2-3 V tiles and scales
+constexpr int kPuSlots = 4;                                // of the copy ring: slots 0-1 take K tiles, slots 2-3 V tiles and scales
 constexpr float kPuLog2e = 1.4426950408889634f;
-constexpr float kPuGain = 256.0f;                          // probabilities are carried times 2^8 (at most 256 < 448)
+constexpr float kPuMaxLag = 8.0f;                          // a row's reference may lag its maximum by this much (base-2 logarithm units)
+constexpr float kPuScaleLag = 16.0f;                       // a V scale may exceed the team's reference scale by this factor
 
 struct PrefillUmmaParams {
   const __nv_bfloat16* q;
@@ -65,51 +73,57 @@ struct PrefillUmmaParams {
   int kv_e5m2;             // the cache codes are E5M2 (the format ablation)
   float sm_scale_log2;
   int* status;
+  unsigned long long* trace;   // trace build only: per CTA the cycles team 0's first thread spent in each phase
 };
 
 struct PuCfg {
   static constexpr int kPart = kBlockSize * kPuD;                 // 2048: K (or V) codes of one granule
   static constexpr int kGran = granule_bytes(kPuD, true);
   static constexpr int kKArea = kPuTileBlocks * kPart;            // 16 KB: the K parts, or the V parts, of a tile
-  static constexpr int kHdrOff = kKArea;                          // behind them the eight headers (scales) of the tile
-  static constexpr int kSlot = kHdrOff + kPuTileBlocks * kFp8Header;   // 16,640
+  static constexpr int kHdrOff = kKArea;                          // V slots: behind the parts the eight headers (scales) of the tile
+  static constexpr int kKSlot = kKArea;
+  static constexpr int kVSlot = kKArea + kPuTileBlocks * kFp8Header;   // 16,640
   static constexpr int kOperand = 128 * 128;                      // one 128 x 128 operand of codes
-  static constexpr int kRingOff = 0;
-  static constexpr int kQOff = kRingOff + kPuSlots * kSlot;          // Q: lead term, remainder term
-  static constexpr int kOperand16 = 128 * 128 * 2;                   // one 128 x 128 operand of f16 values
-  static constexpr int kPOff = kQOff + 2 * kOperand;                 // P: [team], f16
-  static constexpr int kV16Off = kPOff + 2 * kOperand16;             // V^T of a tile widened to f16: [team]
+  static constexpr int kOperand16 = 128 * 128 * 2;                // one 128 x 128 operand of f16 values
+  static constexpr int kRingOff = 0;                              // K slot 0, K slot 1, V slot 0, V slot 1
+  static constexpr int kVRingOff = kRingOff + 2 * kKSlot;
+  static constexpr int kQOff = kVRingOff + 2 * kVSlot;            // Q: lead term, remainder term
+  static constexpr int kPOff = kQOff + 2 * kOperand;              // P: [team], f16
+  static constexpr int kV16Off = kPOff + 2 * kOperand16;          // V^T of a tile widened to f16: [team]
   static constexpr int kBarOff = kV16Off + 2 * kOperand16;
-  static constexpr int kNumBars = 2 * kPuSlots + kPuKSlots + 2 * kPuVSlots + 2 + 2 + 2;   // full, free1, kdone, vdone, vread, sfull, sfree, pfull
+  static constexpr int kNumBars = kPuSlots + 2 + 2 + 2 + 2 + 2 + 2;   // full, kdone, vdone, vread, sfull, sfree, pfull
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kSmemBytes = kMiscOff + 64;
-  static_assert(kSlot % 128 == 0 && kSmemBytes <= 232448, "shared memory of one CTA");
+  static_assert(kVSlot % 128 == 0 && kQOff % 128 == 0 && kSmemBytes <= 232448, "shared memory of one CTA");
 };
+
+// 16 consecutive fp32 columns of this thread's tensor-memory lane, written back.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+                 "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const PrefillUmmaParams p, const __grid_constant__ CUtensorMap map_part,
                                                                           const __grid_constant__ CUtensorMap map_hdr) {
   using C = PuCfg;
   constexpr int D = kPuD;
   extern __shared__ __align__(128) uint8_t smem[];
-  uint8_t* ring = smem + C::kRingOff;
+  uint8_t* kring = smem + C::kRingOff;
+  uint8_t* vring = smem + C::kVRingOff;
   uint8_t* qbuf = smem + C::kQOff;
   uint8_t* pbuf = smem + C::kPOff;
   uint8_t* v16buf = smem + C::kV16Off;
-  // float [4 parts of a row][128] maxima and [4][128] sums share the probability operands' memory: the maxima are
-  // exchanged before the first probability is written, the sums after the last P V instruction has finished
-  float* xch = reinterpret_cast<float*>(smem + C::kPOff);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
-  // Every signal that frees a slot is per slot: its next phase cannot complete before the slot has been
-  // refilled, so the parity a waiter looks for is never overtaken.
-  uint64_t* bar_full = bars;                         // [kPuSlots] the copies into the slot have landed
-  uint64_t* bar_free1 = bar_full + kPuSlots;         // [kPuSlots] first walk: the tile's team has read its logits and scales
-  uint64_t* bar_kdone = bar_free1 + kPuSlots;        // [kPuKSlots] second walk: the logits of the K tile in the slot are computed
-  uint64_t* bar_vdone = bar_kdone + kPuKSlots;       // [kPuVSlots] second walk: the P V instructions of the V tile in the slot are done
-  uint64_t* bar_vread = bar_vdone + kPuVSlots;       // [kPuVSlots] second walk: the tile's team has widened the V tile in the slot
-  uint64_t* bar_sfull = bar_vread + kPuVSlots;       // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
-  uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's eight warps have read them (and the tile's scales)
-  uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's probabilities of a tile are in shared memory
-  int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory, [4..7] V scale maxima
+  uint64_t* bar_full = bars;                         // [4] the copies into the slot have landed (K slots 0-1, V slots 2-3)
+  uint64_t* bar_kdone = bar_full + kPuSlots;         // [2] the logits of the K tile in the slot are computed
+  uint64_t* bar_vdone = bar_kdone + 2;               // [2] the P V instructions of the team's tile are done
+  uint64_t* bar_vread = bar_vdone + 2;               // [2] the team has widened the V tile in the slot (and read its scales)
+  uint64_t* bar_sfull = bar_vread + 2;               // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
+  uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's eight warps have read them for the last time
+  uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's two f16 operands of a tile are in shared memory
+  int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory
   volatile int* abort_flag = misc + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 3);
 
@@ -130,10 +144,11 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     misc[0] = found;
     misc[1] = q0;
     *abort_flag = 0;
-    for (int i = 0; i < kPuSlots; ++i) { mbar_init(&bar_full[i], 1); mbar_init(&bar_free1[i], 8); }
-    for (int i = 0; i < kPuKSlots; ++i) mbar_init(&bar_kdone[i], 1);
-    for (int i = 0; i < kPuVSlots; ++i) { mbar_init(&bar_vdone[i], 1); mbar_init(&bar_vread[i], 8); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 8); mbar_init(&bar_pfull[i], kPuTeam); }
+    for (int i = 0; i < kPuSlots; ++i) mbar_init(&bar_full[i], 1);
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&bar_kdone[i], 1); mbar_init(&bar_vdone[i], 1); mbar_init(&bar_vread[i], 8);
+      mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 8); mbar_init(&bar_pfull[i], kPuTeam);
+    }
     mbar_fence_init();
   }
   if (tid == kPuProducer * 32) {
@@ -159,8 +174,9 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   const int qi = r / G;
   const bool live = tid < kPuSm && qi < nq;
   const size_t grow = static_cast<size_t>(row_base + q0 + (live ? qi : 0)) * Hq + g * G + (live ? r % G : 0);
-  // index of the last visible key of the row; -1 hides everything
-  const int lim = live ? (p.causal ? min(L - 1, L - n_new + q0 + qi) : L - 1) : -1;
+  // index of the last visible key of the row.  Rows past the tile's last query (their query operand is zero and
+  // they are never stored) see everything, so that their warp takes the same unmasked path as its live rows.
+  const int lim = live ? (p.causal ? min(L - 1, L - n_new + q0 + qi) : L - 1) : (1 << 30);
 
   if (n_tiles == 0) {
     // nothing visible: all-zero rows
@@ -222,19 +238,12 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t tmem_o = tmem + 256;                 // logits buffer b at column 128 b, output at 256
+  const uint32_t tmem_o = tmem + 256;                 // logits buffer b at column 128 b, team b's output at 256 + 128 b
   const uint32_t lane_base = static_cast<uint32_t>(warp & 3) * 32u << 16;
-  const int total = 2 * n_tiles;                      // tiles of both walks, numbered in order of use
-  // Slots and the phase of a slot's "landed" barrier.  First walk: tile T lands in slot T % 6 (its use
-  // T / 6 of that slot).  Second walk: the K parts of tile t land in slot t % 2 (use t / 2 after the slot's
-  // first-walk uses), its V parts and scales in slot 2 + t % 4 (use t / 4 after the first-walk uses).
-  auto uses1 = [&](int slot) { return n_tiles > slot ? (n_tiles - slot + kPuSlots - 1) / kPuSlots : 0; };
-  auto kslot_par = [&](int t) { return static_cast<uint32_t>(uses1(t % kPuKSlots) + t / kPuKSlots) & 1u; };
-  auto vslot_par = [&](int t) { return static_cast<uint32_t>(uses1(kPuKSlots + t % kPuVSlots) + t / kPuVSlots) & 1u; };
   uint32_t pend_mask = 0, pend_par = 0;               // copy lane: the latest phase expected of every slot it has filled
 
   if (warp == kPuProducer) {
-    // ================= copies: first walk K parts and headers, second walk V parts as well ================
+    // ================= copies: the K parts of tile t into K slot t % 2, its V parts and headers into V slot t % 2 ====
     // Lane 3 q + w (q = 0, 1; w = 0, 1, 2) fetches the K parts (w = 0), the V parts (w = 1) or the headers
     // (w = 2) of granules 4 q .. 4 q + 3 of the tile.  Rows past the last block repeat the tile's first one.
     bool ok = true;
@@ -244,24 +253,22 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     const CUtensorMap* map = what == 2 ? &map_hdr : &map_part;
     // The physical blocks are looked up 32 at a time (four tiles, one per lane), a batch ahead of their use, so
     // that the copy lane never waits for the block table (range-checked: a bad id is reported in the status
-    // word and replaced by block 0, never dereferenced).  Batches are numbered through both walks.
+    // word and replaced by block 0, never dereferenced).
     const int* trow = p.block_table + static_cast<size_t>(b) * p.max_blocks_per_seq;
     const int nbatch = (n_tiles + 3) / 4;
     auto load_batch = [&](int lb) -> int {
-      if (lb >= 2 * nbatch) return 0;
-      const int j = (lb >= nbatch ? lb - nbatch : lb) * 32 + lane;
+      if (lb >= nbatch) return 0;
+      const int j = lb * 32 + lane;
       int id = j < n_blocks ? trow[j] : 0;
       if (id < 0 || id >= p.num_blocks) { atomicCAS(p.status, 0, COOPT_ERR_INVALID_ARG); id = 0; }
       return id;
     };
     int cur_lb = 0;
     int ids_cur = load_batch(0), ids_next = load_batch(1);
-    for (int T = 0; T < total; ++T) {
-      const bool second = T >= n_tiles;
-      const int t = second ? T - n_tiles : T;
+    for (int t = 0; t < n_tiles; ++t) {
       const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);
       const int ngroups = (nb + 3) / 4;
-      const int lb = (second ? nbatch : 0) + (t >> 2);
+      const int lb = t >> 2;
       if (lb != cur_lb) { ids_cur = ids_next; cur_lb = lb; ids_next = load_batch(lb + 1); }
       int rows[4];
 #pragma unroll
@@ -269,43 +276,23 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         const int j = (q4 & 1) * 4 + i;                             // block of the tile (lanes past the six copy lanes fetch along)
         rows[i] = __shfl_sync(0xffffffffu, ids_cur, (t & 3) * 8 + (j < nb ? j : 0)) * Hkv + g;
       }
-      if (!second) {
-        const int slot = T % kPuSlots;
-        if (lane == 0) {
-          if (T >= kPuSlots) ok = wait_bar(&bar_free1[slot], static_cast<uint32_t>(T / kPuSlots - 1) & 1u, abort_flag);
-          if (ok) {
-            mbar_expect_tx(&bar_full[slot], ngroups * 4 * (C::kPart + kFp8Header));
-            pend_mask |= 1u << slot;
-            pend_par = (pend_par & ~(1u << slot)) | ((static_cast<uint32_t>(T / kPuSlots) & 1u) << slot);
-          }
+      const int sl = t & 1;
+      const uint32_t use = static_cast<uint32_t>(t >> 1);
+      if (lane == 0) {
+        // the slots' users before: the team's tile two back (a wait for phase k follows the one for phase k - 1)
+        if (t >= 2) ok = wait_bar(&bar_kdone[sl], (use - 1) & 1u, abort_flag) && wait_bar(&bar_vread[sl], (use - 1) & 1u, abort_flag);
+        if (ok) {
+          mbar_expect_tx(&bar_full[sl], ngroups * 4 * C::kPart);
+          mbar_expect_tx(&bar_full[2 + sl], ngroups * 4 * (C::kPart + kFp8Header));
+          pend_mask |= (1u << sl) | (4u << sl);
+          pend_par = (pend_par & ~((1u << sl) | (4u << sl))) | ((use & 1u) << sl) | ((use & 1u) << (2 + sl));
         }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) break;
-        if (lane < 3 * ngroups && what != 1)
-          gather4_g2s(ring + slot * C::kSlot + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[slot]);
-      } else {
-        const int ks = t % kPuKSlots, vq = t % kPuVSlots, vs = kPuKSlots + vq;
-        if (lane == 0) {
-          // who used the slots before: the second walk's tile two (K) or four (V) back, else the slot's last tile of the first walk
-          if (t >= kPuKSlots) ok = wait_bar(&bar_kdone[ks], static_cast<uint32_t>(t / kPuKSlots - 1) & 1u, abort_flag);
-          else if (uses1(ks) > 0) ok = wait_bar(&bar_free1[ks], static_cast<uint32_t>(uses1(ks) - 1) & 1u, abort_flag);
-          if (ok) {
-            if (t >= kPuVSlots) ok = wait_bar(&bar_vread[vq], static_cast<uint32_t>(t / kPuVSlots - 1) & 1u, abort_flag);
-            else if (uses1(vs) > 0) ok = wait_bar(&bar_free1[vs], static_cast<uint32_t>(uses1(vs) - 1) & 1u, abort_flag);
-          }
-          if (ok) {
-            mbar_expect_tx(&bar_full[ks], ngroups * 4 * C::kPart);
-            mbar_expect_tx(&bar_full[vs], ngroups * 4 * (C::kPart + kFp8Header));
-            pend_mask |= (1u << ks) | (1u << vs);
-            pend_par = (pend_par & ~((1u << ks) | (1u << vs))) | (kslot_par(t) << ks) | (vslot_par(t) << vs);
-          }
-        }
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) break;
-        if (lane < 3 * ngroups) {
-          const int slot = what == 0 ? ks : vs;
-          gather4_g2s(ring + slot * C::kSlot + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[slot]);
-        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane < 3 * ngroups) {
+        uint8_t* dst = what == 0 ? kring + sl * C::kKSlot : vring + sl * C::kVSlot;
+        gather4_g2s(dst + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[what == 0 ? sl : 2 + sl]);
       }
     }
     if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
@@ -313,17 +300,26 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     // ================= logits: S = Q . Ktile^T, both terms of Q (one lane) ====================================
     if (lane == 0) {
       bool ok = true;
-      const uint64_t desc_k = umma_desc(smem_u32(ring), 128, 8 * D), desc_q = umma_desc(smem_u32(qbuf), 128, 1024);
-      for (int T = 0; T < total && ok; ++T) {
-        const uint32_t buf = T & 1u, use = T >> 1;
-        const bool second = T >= n_tiles;
-        const int t = second ? T - n_tiles : T;
-        const uint32_t slot = second ? t % kPuKSlots : T % kPuSlots;
-        ok = wait_bar(&bar_full[slot], second ? kslot_par(t) : static_cast<uint32_t>(T / kPuSlots) & 1u, abort_flag);
+      const uint64_t desc_k = umma_desc(smem_u32(kring), 128, 8 * D), desc_q = umma_desc(smem_u32(qbuf), 128, 1024);
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const uint32_t buf = t & 1u, use = static_cast<uint32_t>(t >> 1);
+#ifdef COOPT_TRACE
+        const long long ts0 = clock64();
+#endif
+        ok = wait_bar(&bar_full[buf], use & 1u, abort_flag);
+#ifdef COOPT_TRACE
+        const long long ts1 = clock64();
+#endif
         if (ok && use > 0) ok = wait_bar(&bar_sfree[buf], (use - 1) & 1u, abort_flag);
         if (!ok) break;
+#ifdef COOPT_TRACE
+        if (p.trace != nullptr && blockIdx.y * gridDim.x + blockIdx.x < kTraceMaxCtas) {
+          unsigned long long* out = p.trace + static_cast<size_t>(blockIdx.y * gridDim.x + blockIdx.x) * kTraceSlots;
+          out[8] += ts1 - ts0; out[9] += clock64() - ts1;
+        }
+#endif
         tc_fence_after();
-        const uint64_t dk = desc_k + ((slot * C::kSlot) >> 4);
+        const uint64_t dk = desc_k + ((buf * C::kKSlot) >> 4);
 #pragma unroll
         for (int term = 0; term < 2; ++term)
 #pragma unroll
@@ -334,25 +330,39 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     }
   } else if (warp == kPuPvWarp) {
-    // ================= outputs: O += P . Vtile, both terms of P (one lane) ===================================
+    // ================= outputs: O_team += P . Vtile (one lane) ===============================================
     if (lane == 0) {
       bool ok = true;
       // both operands of P V are f16, K-major: 8 rows x 16 bytes (8 values) per core matrix, cores of a row group 128 bytes
       // apart along the keys, row groups 2048 bytes apart
       const uint64_t desc_v = umma_desc(smem_u32(v16buf), 128, 2048), desc_p = umma_desc(smem_u32(pbuf), 128, 2048);
-      for (int T = n_tiles; T < total && ok; ++T) {
-        const int t = T - n_tiles;
-        const uint32_t vq = t % kPuVSlots, team = T & 1u;
-        // the team's tiles of the second walk so far
-        const int first = n_tiles + ((static_cast<int>(team) - n_tiles % 2) + 2) % 2;
-        const uint32_t use = (T - first) >> 1;
+      for (int t = 0; t < n_tiles && ok; ++t) {
+        const uint32_t team = t & 1u, use = static_cast<uint32_t>(t >> 1);
+#ifdef COOPT_TRACE
+        const long long tp0 = clock64();
+#endif
         ok = wait_bar(&bar_pfull[team], use & 1u, abort_flag);
         if (!ok) break;
+#ifdef COOPT_TRACE
+        if (p.trace != nullptr && blockIdx.y * gridDim.x + blockIdx.x < kTraceMaxCtas)
+          p.trace[static_cast<size_t>(blockIdx.y * gridDim.x + blockIdx.x) * kTraceSlots + 10] += clock64() - tp0;
+        const long long tp1 = clock64();
+#endif
         tc_fence_after();
         const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);      // 16 keys (one cache block) per instruction
         const uint64_t dv = desc_v + ((team * C::kOperand16) >> 4), dp = desc_p + ((team * C::kOperand16) >> 4);
-        for (int ks = 0; ks < nb; ++ks) umma_f16(tmem_o, dp + ks * 16, dv + ks * 16, umma_idesc(D), (t | ks) != 0);
-        umma_commit(&bar_vdone[vq]);        // the team's two f16 operands are free again
+        for (int ks = 0; ks < nb; ++ks) umma_f16(tmem_o + 128 * team, dp + ks * 16, dv + ks * 16, umma_idesc(D), (use | ks) != 0);
+        umma_commit(&bar_vdone[team]);      // the team's two f16 operands are free again, its accumulator is at rest
+#ifdef COOPT_TRACE
+        {
+          const long long ti = clock64();
+          wait_bar(&bar_vdone[team], use & 1u, abort_flag);          // (measuring only: how long the instructions take to finish)
+          if (p.trace != nullptr && blockIdx.y * gridDim.x + blockIdx.x < kTraceMaxCtas) {
+            unsigned long long* out = p.trace + static_cast<size_t>(blockIdx.y * gridDim.x + blockIdx.x) * kTraceSlots;
+            out[11] += ti - tp1; out[12] += clock64() - ti;
+          }
+        }
+#endif
       }
       if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
     }
@@ -361,146 +371,255 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     const int team = warp >> 3;
     const int c_lo = half * (kPuTileBlocks / 2), c_hi = c_lo + kPuTileBlocks / 2;   // this thread's cache blocks of a tile
     bool bad = false;
-    float m_row = -INFINITY, l_row = 0.0f, v_max = 0.0f;
+    float m_ref = -INFINITY;     // the row's reference maximum (the same in both threads of the row)
+    float l_row = 0.0f;          // this thread's share of the row's sum of exponentials, against m_ref
+    float v_ref = 0.0f;          // the team's reference V scale (uniform over the team)
     uint8_t* prow = pbuf + team * C::kOperand16 + (r >> 3) * 2048 + (r & 7) * 16;      // row r of the team's P operand
     uint8_t* vrow = v16buf + team * C::kOperand16 + (r >> 3) * 2048 + (r & 7) * 16;    // dim r of the team's V^T operand
+    const uint32_t o_cols = tmem_o + 128 * team + 64 * half + lane_base;               // this thread's 64 of the row's accumulators
+    const uint8_t* st = vring + team * C::kVSlot;                                      // the team's V slot: V parts, then the scales
+    const uint32_t s_cols = tmem + 128 * team + lane_base;                             // the team's logits buffer
 
-    // ---- first walk: the row's maximum logit, and the largest V scale ------------------------------------
-    for (int T = team; T < n_tiles; T += 2) {
-      const uint32_t slot = T % kPuSlots, buf = T & 1u;
-      const uint8_t* st = ring + slot * C::kSlot;
-      bool ok = !bad && wait_bar(&bar_full[slot], static_cast<uint32_t>(T / kPuSlots) & 1u, abort_flag);
-      ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      bad = bad || !ok;
-      if (bad) break;
-      tc_fence_after();
-      const int key0 = T * kPuTileKeys;
-      const int nkeys = min(kPuTileKeys, kv_end - key0);
-#pragma unroll 2
-      for (int c = c_lo; c < c_hi; ++c) {
-        if (c * kBlockSize >= nkeys) break;                       // uniform over the warp
-        uint32_t s[16];
-        tmem_ld16_issue(tmem + 128 * buf + 16 * c + lane_base, s);
-        const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + c * kFp8Header);
-        const float sk = hdr[0] * qscale;
-        v_max = fmaxf(v_max, hdr[1]);
-        const int visible = lim - (key0 + c * kBlockSize);         // keys 0 .. visible of this block are seen by the row
-        tmem_ld_wait(s);
-#pragma unroll
-        for (int j = 0; j < 16; ++j)
-          if (j <= visible) m_row = fmaxf(m_row, __uint_as_float(s[j]) * sk);
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) { mbar_arrive(&bar_sfree[buf]); mbar_arrive(&bar_free1[slot]); }
-    }
-    // the maxima of the four threads that saw part of row r (two teams x two halves of the columns)
-    const int part = team * 2 + half;
-    xch[part * kPuRows + r] = m_row;
-    if (r == 0) reinterpret_cast<float*>(misc + 4)[part] = v_max;
-    bad = barrier_or(1, kPuSm, bad);
-    if (!bad) {
-      m_row = fmaxf(fmaxf(xch[r], xch[kPuRows + r]), fmaxf(xch[2 * kPuRows + r], xch[3 * kPuRows + r]));
-      const float* vm = reinterpret_cast<const float*>(misc + 4);
-      v_max = fmaxf(fmaxf(vm[0], vm[1]), fmaxf(vm[2], vm[3]));
-    }
-    bad = barrier_or(1, kPuSm, bad);          // everybody has read the maxima: their memory may take probabilities
-    const float m_use = m_row == -INFINITY ? 0.0f : m_row;
-    const float v_inv = v_max > 0.0f ? kPuGain / v_max : 0.0f;
-
-    // ---- second walk: probabilities against the final maximum (f16), the V tile widened to f16 -----------
-    int mine = 0;                                                  // this team's tiles of the second walk so far
-    for (int T = n_tiles + ((team - n_tiles % 2) + 2) % 2; T < total && !bad; T += 2, ++mine) {
-      const int t = T - n_tiles;
-      const uint32_t vq = t % kPuVSlots, buf = T & 1u;
-      const uint8_t* st = ring + (kPuKSlots + vq) * C::kSlot;      // the tile's V parts, and behind them its scales
-      bool ok = wait_bar(&bar_full[kPuKSlots + vq], vslot_par(t), abort_flag);
-      ok = ok && wait_bar(&bar_sfull[buf], (T >> 1) & 1u, abort_flag);
-      // the logits are computed: the tile's K slot can be refilled
-      if (ok && (warp & 7) == 0 && lane == 0) mbar_arrive(&bar_kdone[t % kPuKSlots]);
-      // the team's previous tile must have left the probability operand
-      if (ok && mine > 0) ok = wait_bar(&bar_vdone[(t - 2) % kPuVSlots], static_cast<uint32_t>((t - 2) / kPuVSlots) & 1u, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      bad = bad || !ok;
-      if (bad) break;
-      tc_fence_after();
+    // A wait that runs out is made known to the whole team by the named barrier behind it, and the team leaves
+    // the loop together; the other roles give up on their own waits once the abort flag is up.
+#ifdef COOPT_TRACE
+    long long tr_wait_in = 0, tr_pass_a = 0, tr_wait_pv = 0, tr_pass_b = 0, tr_wait_s = 0, tr_wait_v = 0, tr_skew = 0, tr_t = clock64();
+    const long long tr_start = tr_t;
+#define PF_TRACE(acc) do { const long long now_ = clock64(); acc += now_ - tr_t; tr_t = now_; } while (0)
+#else
+#define PF_TRACE(acc) do { } while (0)
+#endif
+    for (int t = team; t < n_tiles && !bad; t += 2) {
+      const uint32_t use = static_cast<uint32_t>(t >> 1);
       const int key0 = t * kPuTileKeys;
       const int nkeys = min(kPuTileKeys, kv_end - key0);
       const int nb = (nkeys + kBlockSize - 1) / kBlockSize;
-#pragma unroll 2
-      for (int c = c_lo; c < c_hi; ++c) {
+      // ---- the tile's scales (they arrive with its V parts) and its logits -------------------------------------
+      // One warp of the team watches the barriers; the other seven wait for it on a named barrier, where the
+      // hardware parks them, instead of polling along with it.
+      if ((warp & 7) == 0) {
+        bool ok = wait_bar(&bar_full[2 + team], use & 1u, abort_flag);
+        ok = ok && wait_bar(&bar_sfull[team], use & 1u, abort_flag);
+        // the logits are computed: the tile's K slot can be refilled
+        if (ok && lane == 0) mbar_arrive(&bar_kdone[team]);
+        bad = !__all_sync(0xffffffffu, ok);
+      }
+      bad = barrier_or(1 + team, kPuTeam, bad);           // uniform over the team from here
+      if (bad) break;
+      tc_fence_after();
+      PF_TRACE(tr_wait_in);
+      float sk8[kPuTileBlocks], sv8[kPuTileBlocks];
+      float v_tile = 0.0f;
+#pragma unroll
+      for (int c = 0; c < kPuTileBlocks; ++c) {
+        const float2 h = *reinterpret_cast<const float2*>(st + C::kHdrOff + c * kFp8Header);
+        sk8[c] = c < nb ? h.x * qscale : 0.0f;
+        sv8[c] = c < nb ? h.y : 0.0f;
+        v_tile = fmaxf(v_tile, sv8[c]);
+      }
+
+      // ---- first pass: the row's maximum over the whole tile -------------------------------------------------
+      float m_tile = -INFINITY;
+#pragma unroll
+      for (int c2 = 0; c2 < kPuTileBlocks; c2 += 2) {             // two cache blocks (32 logits) per trip to tensor memory
+        if (c2 >= nb) break;                              // uniform over the warp
+        uint32_t s[32];
+        tmem_ld32_issue(s_cols + 16 * c2, s);
+        const int visible = lim - (key0 + c2 * kBlockSize);        // keys 0 .. visible of these blocks are seen by the row
+        tmem_ld_wait32(s);
+        if (visible >= 2 * kBlockSize - 1 && c2 + 1 < nb) {
+          // both blocks wholly visible (all but those on the causal diagonal and the tile's last): a K scale is
+          // not negative, so a block's largest logit is its largest accumulator times the scale
+          float mx_a = __uint_as_float(s[0]), mx_b = __uint_as_float(s[16]);
+#pragma unroll
+          for (int j = 1; j < 16; ++j) { mx_a = fmaxf(mx_a, __uint_as_float(s[j])); mx_b = fmaxf(mx_b, __uint_as_float(s[16 + j])); }
+          m_tile = fmaxf(m_tile, fmaxf(mx_a * sk8[c2], mx_b * sk8[c2 + 1]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (j <= visible && (j < 16 || c2 + 1 < nb)) m_tile = fmaxf(m_tile, __uint_as_float(s[j]) * (j < 16 ? sk8[c2] : sk8[c2 + 1]));
+        }
+      }
+      // lazy references: moved only when the tile would push a probability (or a scale ratio) past the margin
+      const bool move_m = m_tile > m_ref + kPuMaxLag;             // also true for the row's first visible key (m_ref = -inf)
+      const bool move_v = v_tile > v_ref * kPuScaleLag;           // uniform over the team; true for the first non-zero scale
+      const float m_new = move_m ? m_tile : m_ref;
+      const float v_new = move_v ? v_tile : v_ref;
+      // the factor that brings what has been accumulated so far onto the new references
+      float factor = 1.0f;
+      if (move_m) factor = m_ref == -INFINITY ? 0.0f : ex2(m_ref - m_new);
+      if (move_v) factor *= v_ref > 0.0f ? __fdividef(v_ref, v_new) : 0.0f;
+      // tensor-memory accesses are warp-wide: the warp rescales if any of its rows has to (the others by 1)
+      const bool rescale = __any_sync(0xffffffffu, move_m || move_v) && use > 0;
+      PF_TRACE(tr_pass_a);
+      // the P V instructions of the team's tile before must have left the team's operands (and its accumulator);
+      // they ran while the first pass was made
+      if (use > 0) {
+        if ((warp & 7) == 0) {
+          const bool ok = wait_bar(&bar_vdone[team], (use - 1) & 1u, abort_flag);
+          bad = !__all_sync(0xffffffffu, ok);
+        }
+        bad = barrier_or(1 + team, kPuTeam, bad);
+        if (bad) break;
+        tc_fence_after();
+      }
+      PF_TRACE(tr_wait_pv);
+      if (rescale) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          uint32_t o[16];
+          tmem_ld16_issue(o_cols + 16 * i, o);
+          tmem_ld_wait(o);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
+          tmem_st16(o_cols + 16 * i, o);
+        }
+        tmem_st_wait();
+      }
+      if (move_m) l_row *= m_ref == -INFINITY ? 0.0f : ex2(m_ref - m_new);
+      m_ref = m_new;
+      v_ref = v_new;
+      const float m_use = m_ref == -INFINITY ? 0.0f : m_ref;
+      const float v_inv = v_ref > 0.0f ? 1.0f / v_ref : 0.0f;
+      // ---- the V tile widened into the team's f16 operand; the copy slot is then free for the team's next tile ---
+#pragma unroll
+      for (int ci = 0; ci < kPuTileBlocks / 2; ++ci) {
+        const int c = c_lo + ci;
         if (c >= nb) break;                               // uniform over the warp: the P V instructions stop at block nb
-        uint32_t s[16];
-        tmem_ld16_issue(tmem + 128 * buf + 16 * c + lane_base, s);
-        const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff + c * kFp8Header);
-        const float sk = hdr[0] * qscale;
-        const float pv = hdr[1] * v_inv;
-        const int visible = lim - (key0 + c * kBlockSize);
-        // dim r of V^T, the 16 tokens of block c: widened to f16 (exact) while the logits are on their way
+        // dim r of V^T, the 16 tokens of block c: widened to f16 (exact)
         const uint4 vc = *reinterpret_cast<const uint4*>(st + c * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
         const int keep = nkeys - c * kBlockSize;          // tokens of the block inside the context (Eq. 9)
-        uint32_t vw[8];
-        {
-          const uint32_t cw[4] = {vc.x, vc.y, vc.z, vc.w};
+        uint32_t cw[4] = {vc.x, vc.y, vc.z, vc.w}, vw[8];
+        if (keep < kBlockSize) {                          // the context ends inside this block: codes past it are cleared
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const int left = keep - 4 * j;
-            const uint32_t w = cw[j] & (left >= 4 ? 0xFFFFFFFFu : (left <= 0 ? 0u : (1u << (8 * left)) - 1u));
-            vw[2 * j] = p.kv_e5m2 ? e5m2x2_to_f16x2_lo(w) : e4m3x2_to_f16x2_lo(w);
-            vw[2 * j + 1] = p.kv_e5m2 ? e5m2x2_to_f16x2_hi(w) : e4m3x2_to_f16x2_hi(w);
+            cw[j] &= left >= 4 ? 0xFFFFFFFFu : (left <= 0 ? 0u : (1u << (8 * left)) - 1u);
           }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          vw[2 * j] = p.kv_e5m2 ? e5m2x2_to_f16x2_lo(cw[j]) : e4m3x2_to_f16x2_lo(cw[j]);
+          vw[2 * j + 1] = p.kv_e5m2 ? e5m2x2_to_f16x2_hi(cw[j]) : e4m3x2_to_f16x2_hi(cw[j]);
         }
         *reinterpret_cast<uint4*>(vrow + (2 * c) * 128) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
         *reinterpret_cast<uint4*>(vrow + (2 * c + 1) * 128) = make_uint4(vw[4], vw[5], vw[6], vw[7]);
-        tmem_ld_wait(s);
-        uint32_t pw[8];
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&bar_vread[team]);       // the V slot may take the team's next tile
+      PF_TRACE(tr_pass_b);
+
+
+      // ---- second pass: probabilities of this thread's blocks against the reference (f16) ----------------------
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-          const float x0 = ex2(__uint_as_float(s[2 * e]) * sk - m_use), x1 = ex2(__uint_as_float(s[2 * e + 1]) * sk - m_use);
-          const float p0 = (2 * e <= visible) ? x0 : 0.0f, p1 = (2 * e + 1 <= visible) ? x1 : 0.0f;
-          l_row += p0 + p1;
-          pw[e] = pack_f16x2(p0 * pv, p1 * pv);           // at most 256: probabilities are carried times 2^8
+      for (int ci = 0; ci < kPuTileBlocks / 2; ci += 2) {         // two cache blocks per trip to tensor memory
+        const int c = c_lo + ci;
+        if (c >= nb) break;                               // uniform over the warp
+        uint32_t s[32];
+        tmem_ld32_issue(s_cols + 16 * c, s);
+        const float sk_a = half ? sk8[4 + ci] : sk8[ci], sk_b = half ? sk8[5 + ci] : sk8[1 + ci];
+        const float pv_a = (half ? sv8[4 + ci] : sv8[ci]) * v_inv, pv_b = (half ? sv8[5 + ci] : sv8[1 + ci]) * v_inv;   // at most 2^4
+        const int visible = lim - (key0 + c * kBlockSize);
+        tmem_ld_wait32(s);
+#pragma unroll
+        for (int blk = 0; blk < 2; ++blk) {
+          if (c + blk >= nb) break;                       // uniform
+          const float sk = blk ? sk_b : sk_a, pv = blk ? pv_b : pv_a;
+          uint32_t pw[8];
+          if (visible >= 16 * blk + kBlockSize - 1 && pv > 0.0f) {
+            // the block is wholly visible: the V scale rides in the exponent, p * pv = 2^(s * sk - m + log2 pv),
+            // and the block's sum of p is recovered from the sum of p * pv with one division
+            float lg;
+            asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(pv));
+            const float shift = lg - m_use;
+            float l_blk = 0.0f;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int j = 16 * blk + 2 * e;
+              const float y0 = ex2(fmaf(__uint_as_float(s[j]), sk, shift)), y1 = ex2(fmaf(__uint_as_float(s[j + 1]), sk, shift));
+              l_blk += y0 + y1;
+              pw[e] = pack_f16x2(y0, y1);                 // at most 2^8 * 2^4: well inside f16
+            }
+            l_row += __fdividef(l_blk, pv);
+          } else {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) {
+              const int j = 16 * blk + 2 * e;
+              const float x0 = ex2(__uint_as_float(s[j]) * sk - m_use), x1 = ex2(__uint_as_float(s[j + 1]) * sk - m_use);
+              const float p0 = (j <= visible) ? x0 : 0.0f, p1 = (j + 1 <= visible) ? x1 : 0.0f;
+              l_row += p0 + p1;
+              pw[e] = pack_f16x2(p0 * pv, p1 * pv);
+            }
+          }
+          *reinterpret_cast<uint4*>(prow + (2 * (c + blk)) * 128) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+          *reinterpret_cast<uint4*>(prow + (2 * (c + blk) + 1) * 128) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
         }
-        *reinterpret_cast<uint4*>(prow + (2 * c) * 128) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
-        *reinterpret_cast<uint4*>(prow + (2 * c + 1) * 128) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
       }
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) { mbar_arrive(&bar_sfree[buf]); mbar_arrive(&bar_vread[vq]); }
+      if (lane == 0) mbar_arrive(&bar_sfree[team]);
       fence_proxy_async();
       mbar_arrive(&bar_pfull[team]);
+      PF_TRACE(tr_pass_b);
+#ifdef COOPT_TRACE
+      if (tid == 0) { wait_bar(&bar_pfull[team], use & 1u, abort_flag); PF_TRACE(tr_skew); }   // (measuring only: until the team's last thread has arrived)
+#endif
     }
+#ifdef COOPT_TRACE
+    if (tid == 0 && p.trace != nullptr) {
+      const int rec = blockIdx.y * gridDim.x + blockIdx.x;
+      if (rec < kTraceMaxCtas) {
+        unsigned long long* out = p.trace + static_cast<size_t>(rec) * kTraceSlots;
+        out[0] = n_tiles; out[1] = tr_wait_in; out[2] = tr_pass_a; out[3] = tr_wait_pv; out[4] = tr_pass_b; out[5] = clock64() - tr_start; out[6] = tr_wait_s; out[7] = tr_wait_v; out[13] = tr_skew;
+      }
+    }
+#endif
 
-    // ---- the last P V instruction has finished: normalise and store ---------------------------------------
-    if (!bad) {
-      // A wait names a phase by its parity, which only tells the phase before from the one in progress: a team
-      // that is done a tile early must not ask for the last tile's phase while the phase before it on the same
-      // barrier is still open.  The last two tiles' instructions are waited for in order (the one before them
-      // is finished: the team waited for it, or for a later one, inside its loop).
-      const int tl = n_tiles - 1;
-      bool ok = true;
-      if (tl >= 1) ok = wait_bar(&bar_vdone[(tl - 1) % kPuVSlots], static_cast<uint32_t>((tl - 1) / kPuVSlots) & 1u, abort_flag);
-      ok = ok && wait_bar(&bar_vdone[tl % kPuVSlots], static_cast<uint32_t>(tl / kPuVSlots) & 1u, abort_flag);
-      ok = __all_sync(0xffffffffu, ok);
-      bad = !ok;
+    // ---- the team's last P V instruction has finished: the two teams' results are merged and stored ------------
+    const int my_tiles = n_tiles > team ? (n_tiles - team + 1) / 2 : 0;
+    if (!bad && my_tiles > 0 && (warp & 7) == 0) {
+      bool ok = wait_bar(&bar_vdone[team], static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag);
+      bad = !__all_sync(0xffffffffu, ok);
     }
-    xch[4 * kPuRows + part * kPuRows + r] = l_row;
-    bad = barrier_or(1, kPuSm, bad);
+    bad = barrier_or(1 + team, kPuTeam, bad);
+    // what the other team needs of this one, in this team's own (now idle) P operand: per row its reference and
+    // the two halves' sums, and the team's reference scale
+    float* mine = reinterpret_cast<float*>(pbuf + team * C::kOperand16);
+    const float* theirs = reinterpret_cast<const float*>(pbuf + (team ^ 1) * C::kOperand16);
+    mine[half * kPuRows + r] = l_row;
+    if (half == 0) mine[2 * kPuRows + r] = m_ref;
+    if (tid == team * kPuTeam) mine[3 * kPuRows] = v_ref;
+    bad = barrier_or(3, kPuSm, bad);
     if (!bad) {
       tc_fence_after();
-      const float l_all = (xch[4 * kPuRows + r] + xch[5 * kPuRows + r]) + (xch[6 * kPuRows + r] + xch[7 * kPuRows + r]);
-      const float k = l_all > 0.0f ? v_max / (kPuGain * l_all) : 0.0f;
+      const float l_me = mine[r] + mine[kPuRows + r], l_ot = theirs[r] + theirs[kPuRows + r];
+      const float m_ot = theirs[2 * kPuRows + r], v_ot = theirs[3 * kPuRows];
+      const float M = fmaxf(l_me > 0.0f ? m_ref : -INFINITY, l_ot > 0.0f ? m_ot : -INFINITY);
+      const float w_me = l_me > 0.0f ? ex2(m_ref - M) : 0.0f, w_ot = l_ot > 0.0f ? ex2(m_ot - M) : 0.0f;
+      const float den = w_me * l_me + w_ot * l_ot;
+      const float inv = den > 0.0f ? 1.0f / den : 0.0f;
+      const float k_me = w_me * v_ref * inv, k_ot = w_ot * v_ot * inv;
+      const bool other_ran = n_tiles > (team ^ 1);
       // the four threads of row r store 32 dims each
+      const int part = team * 2 + half;
 #pragma unroll
       for (int c = 0; c < 2; ++c) {
-        uint32_t o[16];
-        tmem_ld16_issue(tmem_o + part * 32 + 16 * c + lane_base, o);
-        tmem_ld_wait(o);
+        uint32_t oa[16], ob[16];
+        tmem_ld16_issue(tmem_o + 128 * team + part * 32 + 16 * c + lane_base, oa);
+        tmem_ld_wait(oa);
+        if (other_ran) {                                   // uniform; an accumulator that was never written holds anything
+          tmem_ld16_issue(tmem_o + 128 * (team ^ 1) + part * 32 + 16 * c + lane_base, ob);
+          tmem_ld_wait(ob);
+        }
         if (live) {
           uint32_t w[8];
 #pragma unroll
-          for (int j = 0; j < 8; ++j) w[j] = pack_bf16x2(__uint_as_float(o[2 * j]) * k, __uint_as_float(o[2 * j + 1]) * k);
+          for (int j = 0; j < 8; ++j) {
+            float y0 = my_tiles > 0 && w_me > 0.0f ? __uint_as_float(oa[2 * j]) * k_me : 0.0f;
+            float y1 = my_tiles > 0 && w_me > 0.0f ? __uint_as_float(oa[2 * j + 1]) * k_me : 0.0f;
+            if (other_ran && w_ot > 0.0f) { y0 += __uint_as_float(ob[2 * j]) * k_ot; y1 += __uint_as_float(ob[2 * j + 1]) * k_ot; }
+            w[j] = pack_bf16x2(y0, y1);
+          }
           uint4* dst = reinterpret_cast<uint4*>(p.out + grow * D + part * 32 + 16 * c);
           dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
           dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
@@ -544,6 +663,10 @@ int launch_paged_prefill_umma(const coopt_cache* c, const void* q, void* out, co
   p.kv_e5m2 = c->dtype == COOPT_KV_FP8_E5M2 ? 1 : 0;
   p.sm_scale_log2 = sm_scale * kPuLog2e;
   p.status = static_cast<int*>(workspace);
+  p.trace = nullptr;
+#ifdef COOPT_TRACE
+  p.trace = trace_buffer();
+#endif
   const long long tiles = static_cast<long long>(total_q) / p.tile_queries + batch;   // every sequence adds at most one partly filled tile
   if (tiles > 0x7fffffffll) return COOPT_ERR_UNSUPPORTED;
   CUtensorMap map_part, map_hdr;
