@@ -346,6 +346,9 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true",
                     help="launch every step from the host instead of replaying a CUDA graph of one pass over the layer caches")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="do not let a step's prologue start while the step before it drains (COOPT_FLAG_OVERLAP_PREVIOUS "
+                         "is otherwise given to every step of a pass over the layer caches but the first)")
     ap.add_argument("--roofline-launches", type=int, default=2000,
                     help="launches of the kernel-timing loop behind the timed region (fewer under a profiler)")
     ap.add_argument("--workload", default="llama13b_decode",
@@ -408,11 +411,16 @@ def main():
     out = torch.empty_like(q)
     torch.cuda.synchronize()
 
+    overlap = 0 if args.no_overlap else binding.FLAG_OVERLAP_PREVIOUS
+
     def step(i):
-        """One layer's step; the plan is renewed once per pass over the layers, as it is once per model step."""
+        """One layer's step; the plan is renewed once per pass over the layers, as it is once per model step.  As in
+        coopt_decode_layers, a step behind another step may set up (barriers, tensor memory, its plan) while that one
+        drains; it touches the cache, the workspace and the output only after the earlier launch has completed."""
         if i % NL == 0:
             binding.decode_plan(table, lens, HKV, base.num_blocks, plan=plan)
-        binding.decode_step_planned(caches[i % NL], plan, q, max_blocks, base.sm_scale, ws, k_new, v_new, s_new, out=out)
+        binding.decode_step_planned(caches[i % NL], plan, q, max_blocks, base.sm_scale, ws, k_new, v_new, s_new,
+                                    flags=overlap if i % NL else 0, out=out)
 
     for i in range(warmup):
         step(i)
@@ -472,12 +480,17 @@ def main():
     b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     binding.decode_plan(table, lens, HKV, base.num_blocks, plan=plan)
     torch.cuda.synchronize()
-    b0.record()
-    for i in range(n_b2b):
-        binding.decode_step_planned(caches[i % NL], plan, q, max_blocks, base.sm_scale, ws, k_new, v_new, s_new, out=out)
-    b1.record()
-    torch.cuda.synchronize()
-    kernel_b2b_ms = b0.elapsed_time(b1) / n_b2b
+    def back_to_back(flags):
+        b0.record()
+        for i in range(n_b2b):
+            binding.decode_step_planned(caches[i % NL], plan, q, max_blocks, base.sm_scale, ws, k_new, v_new, s_new,
+                                        flags=flags if i else 0, out=out)
+        b1.record()
+        torch.cuda.synchronize()
+        return b0.elapsed_time(b1) / n_b2b
+
+    kernel_serial_ms = back_to_back(0)
+    kernel_b2b_ms = back_to_back(overlap) if overlap else kernel_serial_ms
     pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(max(4, n_b2b // 10))]
     for i, (e0, e1) in enumerate(pairs):
         e0.record()
@@ -487,7 +500,7 @@ def main():
     sampler.stop_flag = True
     kernel_pair_ms = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs)
     assert binding.workspace_status(ws) == 0
-    ms, kernel_b2b_ms, kernel_pair_ms = max_over_ranks([ms, kernel_b2b_ms, kernel_pair_ms], device="cuda")
+    ms, kernel_b2b_ms, kernel_pair_ms, kernel_serial_ms = max_over_ranks([ms, kernel_b2b_ms, kernel_pair_ms, kernel_serial_ms], device="cuda")
     value = job_tokens_per_second(world, BATCH, args.steps, ms)
 
     # ---- end to end: host buffers in, host result out, through coopt_decode_step_host ----------
@@ -545,7 +558,9 @@ def main():
                 "frac_of_nominal_8TBs": achieved / 8000.0,
                 "algorithmic_bytes_per_launch": algo, "kernel_us": kernel_ms * 1e3,
                 "timing": "average over %d launches of the kernel back to back between one pair of CUDA events on the "
-                          "launching stream, layer caches visited round-robin" % n_b2b,
+                          "launching stream, layer caches visited round-robin, launched as the timed region launches them (%s)"
+                          % (n_b2b, "each launch may set up while the one before it drains" if overlap else "serial"),
+                "kernel_us_back_to_back_serial": kernel_serial_ms * 1e3,
                 "kernel_us_event_pair_per_launch": kernel_pair_ms * 1e3,
                 "kernel_us_timed_region_per_step": ms / args.steps * 1e3,
                 "kernel_us_x_sm_mhz": kernel_ms * 1e3 * (clocks["sm_mhz"] or 0),
@@ -557,7 +572,8 @@ def main():
             "config": {"workload": WORKLOAD, "layers_rotated": NL,
                        "l2": "inputs larger than L2: %d layer caches of %.0f MB visited round-robin" % (NL, algo / 1e6),
                        "step": "coopt_decode_step_planned (one launch: the new token of every sequence written, then attention); "
-                               "coopt_decode_plan once per pass over the layer caches, inside the timed region",
+                               "coopt_decode_plan once per pass over the layer caches, inside the timed region; "
+                               + ("steps of a pass behind the first carry COOPT_FLAG_OVERLAP_PREVIOUS" if overlap else "no overlap of consecutive steps"),
                        "launch": "host launches" if graph is None else
                                  "a CUDA graph of one pass over the layer caches (plan + %d steps) replayed; the remainder from the host" % NL},
             "gpu_launches": args.steps + (args.steps + NL - 1) // NL, "clocks": clocks, "clocks_timed_region": region_clocks,

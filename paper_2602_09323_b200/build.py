@@ -4,7 +4,7 @@
 is compiled to an object of its own (in parallel) under ``_build/`` and the objects are linked into
 the shared library.  ``--trace`` builds ``libcoopt_trace.so`` instead: the same sources with
 ``-DCOOPT_TRACE``, whose tcgen05 kernels also write time stamps of their roles into a caller-supplied
-buffer (see ``coopt_trace.h``); the ordinary library contains none of that code.
+buffer (``csrc/coopt_trace.cuh``, read by ``python -m paper_2602_09323_b200.trace``); the ordinary library contains none of that code.
 """
 from __future__ import annotations
 

@@ -103,6 +103,15 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
                ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
                  "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
 }
+// Two E4M3 codes (bytes of `w` picked by `sel`: 0x1404 the low two, 0x3424 the high two) as two f16 holding the
+// codes' values divided by 2^8, exactly: with the code in the upper byte of a half, its exponent and mantissa
+// bits are moved down one place into the f16 fields (bias 7 against 15; a subnormal code becomes a subnormal
+// f16 of the same proportion), the sign stays.  Integer instructions only: the conversion instruction shares
+// the unit that takes the exponentials.
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2_small(uint32_t w, uint32_t sel) {
+  const uint32_t x = __byte_perm(w, 0u, sel);
+  return ((x >> 1) & 0x3F803F80u) | (x & 0x80008000u);
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const PrefillUmmaParams p, const __grid_constant__ CUtensorMap map_part,
@@ -369,7 +378,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   } else {
     // ================= softmax teams ================================================================================
     const int team = warp >> 3;
-    const int c_lo = half * (kPuTileBlocks / 2), c_hi = c_lo + kPuTileBlocks / 2;   // this thread's cache blocks of a tile
+    const int c_lo = half * (kPuTileBlocks / 2);            // the first of this thread's four cache blocks of a tile
     bool bad = false;
     float m_ref = -INFINITY;     // the row's reference maximum (the same in both threads of the row)
     float l_row = 0.0f;          // this thread's share of the row's sum of exponentials, against m_ref
@@ -486,7 +495,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       for (int ci = 0; ci < kPuTileBlocks / 2; ++ci) {
         const int c = c_lo + ci;
         if (c >= nb) break;                               // uniform over the warp: the P V instructions stop at block nb
-        // dim r of V^T, the 16 tokens of block c: widened to f16 (exact)
+        // dim r of V^T, the 16 tokens of block c: widened to f16 (exact; E4M3 codes come out divided by 2^8)
         const uint4 vc = *reinterpret_cast<const uint4*>(st + c * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
         const int keep = nkeys - c * kBlockSize;          // tokens of the block inside the context (Eq. 9)
         uint32_t cw[4] = {vc.x, vc.y, vc.z, vc.w}, vw[8];
@@ -499,8 +508,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          vw[2 * j] = p.kv_e5m2 ? e5m2x2_to_f16x2_lo(cw[j]) : e4m3x2_to_f16x2_lo(cw[j]);
-          vw[2 * j + 1] = p.kv_e5m2 ? e5m2x2_to_f16x2_hi(cw[j]) : e4m3x2_to_f16x2_hi(cw[j]);
+          vw[2 * j] = p.kv_e5m2 ? e5m2x2_to_f16x2_lo(cw[j]) : e4m3x2_to_f16x2_small(cw[j], 0x1404u);
+          vw[2 * j + 1] = p.kv_e5m2 ? e5m2x2_to_f16x2_hi(cw[j]) : e4m3x2_to_f16x2_small(cw[j], 0x3424u);
         }
         *reinterpret_cast<uint4*>(vrow + (2 * c) * 128) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
         *reinterpret_cast<uint4*>(vrow + (2 * c + 1) * 128) = make_uint4(vw[4], vw[5], vw[6], vw[7]);
@@ -511,6 +520,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
 
 
       // ---- second pass: probabilities of this thread's blocks against the reference (f16) ----------------------
+      bool s_freed = false;
 #pragma unroll
       for (int ci = 0; ci < kPuTileBlocks / 2; ci += 2) {         // two cache blocks per trip to tensor memory
         const int c = c_lo + ci;
@@ -521,6 +531,14 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         const float pv_a = (half ? sv8[4 + ci] : sv8[ci]) * v_inv, pv_b = (half ? sv8[5 + ci] : sv8[1 + ci]) * v_inv;   // at most 2^4
         const int visible = lim - (key0 + c * kBlockSize);
         tmem_ld_wait32(s);
+        if (ci + 2 >= kPuTileBlocks / 2 || c + 2 >= nb) {
+          // the thread's last logits of the tile are in registers: the buffer goes back before the probabilities
+          // are made, so that the tile after next is multiplied meanwhile
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&bar_sfree[team]);
+          s_freed = true;
+        }
 #pragma unroll
         for (int blk = 0; blk < 2; ++blk) {
           if (c + blk >= nb) break;                       // uniform
@@ -555,9 +573,11 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
           *reinterpret_cast<uint4*>(prow + (2 * (c + blk) + 1) * 128) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
         }
       }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&bar_sfree[team]);
+      if (!s_freed) {                                     // a warp whose blocks lie past the end of the context
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&bar_sfree[team]);
+      }
       fence_proxy_async();
       mbar_arrive(&bar_pfull[team]);
       PF_TRACE(tr_pass_b);
@@ -598,7 +618,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       const float w_me = l_me > 0.0f ? ex2(m_ref - M) : 0.0f, w_ot = l_ot > 0.0f ? ex2(m_ot - M) : 0.0f;
       const float den = w_me * l_me + w_ot * l_ot;
       const float inv = den > 0.0f ? 1.0f / den : 0.0f;
-      const float k_me = w_me * v_ref * inv, k_ot = w_ot * v_ot * inv;
+      const float unit = p.kv_e5m2 ? 1.0f : 256.0f;        // the widened E4M3 codes carry their values / 2^8
+      const float k_me = w_me * v_ref * inv * unit, k_ot = w_ot * v_ot * inv * unit;
       const bool other_ran = n_tiles > (team ^ 1);
       // the four threads of row r store 32 dims each
       const int part = team * 2 + half;

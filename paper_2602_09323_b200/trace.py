@@ -1,11 +1,12 @@
-"""Where the time of one decode launch goes: ``python -m paper_2602_09323_b200.trace [--workload ...]``.
+"""Where the time of one launch goes: ``python -m paper_2602_09323_b200.trace [--workload ...]``.
 
 Builds ``libcoopt_trace.so`` (the library's sources with ``-DCOOPT_TRACE``), runs the fused decode step of a
 workload a few times and prints, for the last launch, when each role of the tcgen05 kernel reached its
 milestones: per milestone the median, the earliest and the latest CTA, in microseconds from that CTA's own
 first instruction, and the span of the whole launch on the global timer.  The stamps cost a few stores per
 tile; the launch is a few per cent slower than in the ordinary library, so this is a breakdown, not a
-benchmark.
+benchmark.  ``--workload chunked_prefill`` prints instead, for the tcgen05 prefill kernel, the cycles that the
+first thread of softmax team 0 and the two instruction-issuing lanes spend in each phase of a tile.
 """
 from __future__ import annotations
 
@@ -27,7 +28,7 @@ SEG_BASE, TEAM_SEG_BASE = 24, 44
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--workload", default="llama13b_decode", choices=["llama13b_decode", "mixed_serving", "long_context"])
+    ap.add_argument("--workload", default="llama13b_decode", choices=["llama13b_decode", "mixed_serving", "long_context", "chunked_prefill"])
     ap.add_argument("--no-append", action="store_true", help="attention only (no new token written in the launch)")
     ap.add_argument("--launches", type=int, default=12)
     ap.add_argument("--timeline", type=int, nargs="*", default=None, help="CTAs whose tile-by-tile timeline is printed")
@@ -40,6 +41,8 @@ def main():
     lib = binding.load_library()
     lib.coopt_trace_set_buffer.restype, lib.coopt_trace_set_buffer.argtypes = ctypes.c_int, [ctypes.c_void_p, ctypes.c_size_t]
     torch.cuda.set_device(0)
+    if args.workload == "chunked_prefill":
+        return prefill_trace(lib)
     chunk = 0
     if args.workload == "llama13b_decode":
         w = workloads.config_llama13b_decode()
@@ -131,6 +134,40 @@ def main():
             if ok.any():
                 rel = (col[ok] - t[ok, 0]) * us
                 print(f"{label + ' ' + str(i):<26}{np.median(rel):9.2f}{rel.min():10.2f}{rel.max():9.2f}   ({int(ok.sum())} CTAs)")
+
+
+PREFILL_PHASES = (
+    (1, "team: waits for the tile's V part, scales and logits"), (2, "team: first pass (row maxima, references)"),
+    (3, "team: waits for its previous P V product"), (4, "team: rescale, V widened to f16, second pass (probabilities)"),
+    (13, "team: first thread done -> whole team arrived"), (5, "team: whole loop"),
+    (8, "logits lane: waits for the K tile"), (9, "logits lane: waits for the team to free the logits buffer"),
+    (10, "P V lane: waits for the probabilities"), (11, "P V lane: issues 8 instructions + commit"),
+    (12, "P V lane: commit -> completion"))
+
+
+def prefill_trace(lib):
+    """Cycles per tile of team 0 in the phases of the tcgen05 prefill kernel (configuration: 8 sequences of 4096
+    cached + 512 new tokens).  The lanes' figures are sums over both teams' tiles, divided by team 0's tile count."""
+    w = workloads.config_chunked_prefill()
+    cache = binding.Cache(w.num_blocks, w.num_kv_heads, w.head_dim)
+    binding.kv_write(cache, w.k.cuda(), w.v.cuda(), w.slot_mapping.cuda())
+    ws = binding.new_workspace(w.batch, w.num_q_heads, w.num_kv_heads, w.head_dim, w.block_table.shape[1], 2048, sum(w.q_lens))
+    buf = torch.zeros(MAX_CTAS * SLOTS, dtype=torch.int64, device="cuda")
+    assert lib.coopt_trace_set_buffer(ctypes.c_void_p(buf.data_ptr()), buf.numel() * 8) == 0
+    q, cu, table, lens = w.q.cuda(), w.cu_q_lens.cuda(), w.block_table.cuda(), w.context_lens_tensor.cuda()
+    for _ in range(3):
+        buf.zero_()
+        binding.paged_chunked(cache, q, cu, table, lens, 2048, True, w.sm_scale, ws)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    t = buf.cpu().numpy().reshape(MAX_CTAS, SLOTS)
+    t = t[t[:, 0] > 0]
+    own = t[:, 0].astype(float) / 2                      # team 0's tiles of the CTA
+    print(f"workload chunked_prefill: {len(t)} CTAs recorded (the first {MAX_CTAS} of the grid), tiles per CTA median {np.median(t[:, 0]):.0f}")
+    print(f"{'phase':<62}{'median':>8}{'min':>8}{'max':>8}   (cycles per tile of team 0)")
+    for i, name in PREFILL_PHASES:
+        per = t[:, i] / own
+        print(f"{name:<62}{np.median(per):8.0f}{per.min():8.0f}{per.max():8.0f}")
 
 
 if __name__ == "__main__":
