@@ -341,7 +341,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20000)
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--layers", type=int, default=8, help="layer caches the steps rotate over (one plan per pass over them)")
+    ap.add_argument("--layers", type=int, default=40,
+                    help="layer caches the steps rotate over, one plan per pass over them (40 = the layers of LLaMA-13B: a pass is one model step)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="budget of the CPU-baseline leg")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-graph", action="store_true",
@@ -689,7 +690,7 @@ def run_layers(args):
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode launch on this workload, from the
 # ncu capture summarised under profiles/ (None while the kernel is newer than the capture).
-DRAM_TRAFFIC_PER_LAUNCH = None
+DRAM_TRAFFIC_PER_LAUNCH = 140057856 + 5144320   # dram__bytes_read.sum + dram__bytes_write.sum of one launch (profiles/)
 
 if __name__ == "__main__":
     main()

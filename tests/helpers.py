@@ -35,6 +35,9 @@ def check_attention(got: torch.Tensor, ref: np.ndarray, plain: bool = False, wha
     ulp = np.where(r != 0, 2.0 ** (np.floor(np.log2(np.maximum(np.abs(r), 1e-300))) - 7), 0.0)
     own = np.abs(got[mask] - r_bf16)
     assert np.all(own <= MAX_ABS + ulp), f"{what}: kernel error apart from output rounding {np.max(own - ulp):.4g}"
+    # shown by `pytest -s` / `-rP`: the figures the results table quotes
+    print(f"[parity] {what or 'attention'}{' (plain bound)' if plain else ''}: {err.size} outputs, max-abs {err.max():.3g}, "
+          f"mean-abs {err.mean():.3g}, max |ref| {np.abs(r).max():.3g}, kernel's own max error {own.max():.3g}")
     return float(err.max()), float(err.mean())
 
 
