@@ -93,7 +93,9 @@ struct PuCfg {
   static constexpr int kBarOff = kV16Off + 2 * kOperand16;
   static constexpr int kNumBars = kPuSlots + 2 + 2 + 2 + 2 + 2 + 2;   // full, kdone, vdone, vread, sfull, sfree, pfull
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
-  static constexpr int kSmemBytes = kMiscOff + 64;
+  static constexpr int kXchOff = kMiscOff + 64;                   // [team][parity][half][row] upper halves of fp32 maxima
+  static constexpr int kSclOff = kXchOff + 2 * 2 * 2 * kPuRows * 2;   // [team][block][K scale, V scale] of the tile being worked on
+  static constexpr int kSmemBytes = kSclOff + 2 * kPuTileBlocks * 2 * 4;
   static_assert(kVSlot % 128 == 0 && kQOff % 128 == 0 && kSmemBytes <= 232448, "shared memory of one CTA");
 };
 
@@ -114,6 +116,7 @@ __device__ __forceinline__ uint32_t e4m3x2_to_f16x2_small(uint32_t w, uint32_t s
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+template <bool kE5m2>
 __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const PrefillUmmaParams p, const __grid_constant__ CUtensorMap map_part,
                                                                           const __grid_constant__ CUtensorMap map_hdr) {
   using C = PuCfg;
@@ -132,6 +135,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   uint64_t* bar_sfull = bar_vread + 2;               // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
   uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's eight warps have read them for the last time
   uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's two f16 operands of a tile are in shared memory
+  unsigned short* xch = reinterpret_cast<unsigned short*>(smem + C::kXchOff);
   int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory
   volatile int* abort_flag = misc + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(misc + 3);
@@ -333,7 +337,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         for (int term = 0; term < 2; ++term)
 #pragma unroll
           for (int ks = 0; ks < D / 32; ++ks)
-            umma_f8(tmem + 128 * buf, desc_q + ((term * C::kOperand) >> 4) + ks * 16, dk + ks * 16, umma_idesc(128, 0, p.kv_e5m2), (term | ks) != 0);
+            umma_f8(tmem + 128 * buf, desc_q + ((term * C::kOperand) >> 4) + ks * 16, dk + ks * 16, umma_idesc(128, 0, kE5m2 ? 1 : 0), (term | ks) != 0);
         umma_commit(&bar_sfull[buf]);
       }
       if (!ok) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
@@ -392,7 +396,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     // A wait that runs out is made known to the whole team by the named barrier behind it, and the team leaves
     // the loop together; the other roles give up on their own waits once the abort flag is up.
 #ifdef COOPT_TRACE
-    long long tr_wait_in = 0, tr_pass_a = 0, tr_wait_pv = 0, tr_pass_b = 0, tr_wait_s = 0, tr_wait_v = 0, tr_skew = 0, tr_t = clock64();
+    long long tr_wait_in = 0, tr_pass_a = 0, tr_wait_pv = 0, tr_widen = 0, tr_pass_b = 0, tr_skew = 0, tr_t = clock64();
     const long long tr_start = tr_t;
 #define PF_TRACE(acc) do { const long long now_ = clock64(); acc += now_ - tr_t; tr_t = now_; } while (0)
 #else
@@ -417,38 +421,62 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       if (bad) break;
       tc_fence_after();
       PF_TRACE(tr_wait_in);
-      float sk8[kPuTileBlocks], sv8[kPuTileBlocks];
-      float v_tile = 0.0f;
-#pragma unroll
-      for (int c = 0; c < kPuTileBlocks; ++c) {
-        const float2 h = *reinterpret_cast<const float2*>(st + C::kHdrOff + c * kFp8Header);
-        sk8[c] = c < nb ? h.x * qscale : 0.0f;
-        sv8[c] = c < nb ? h.y : 0.0f;
-        v_tile = fmaxf(v_tile, sv8[c]);
-      }
+      // The loops over the tile are kept rolled (32 logits = two cache blocks per trip to tensor memory): unrolled,
+      // the body of this loop was tens of KB of instructions and the teams waited for instruction fetch.
+      const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff);    // [block][8]: K scale, V scale, zeros
+      const int nb_mine = min(nb - c_lo, kPuTileBlocks / 2);                 // this thread's blocks of the tile (<= 0: none)
 
-      // ---- first pass: the row's maximum over the whole tile -------------------------------------------------
-      float m_tile = -INFINITY;
+      // ---- first pass: the maximum of this thread's half of the row; the tile's largest V scale ------------------
+      float m_half = -INFINITY, v_tile = 0.0f;
 #pragma unroll
-      for (int c2 = 0; c2 < kPuTileBlocks; c2 += 2) {             // two cache blocks (32 logits) per trip to tensor memory
-        if (c2 >= nb) break;                              // uniform over the warp
+      for (int c = 0; c < kPuTileBlocks; ++c) v_tile = fmaxf(v_tile, c < nb ? hdr[c * 8 + 1] : 0.0f);
+#pragma unroll 1
+      for (int ci = 0; ci < nb_mine; ci += 2) {
+        const int c = c_lo + ci;
         uint32_t s[32];
-        tmem_ld32_issue(s_cols + 16 * c2, s);
-        const int visible = lim - (key0 + c2 * kBlockSize);        // keys 0 .. visible of these blocks are seen by the row
+        tmem_ld32_issue(s_cols + 16 * c, s);
+        const bool two = ci + 1 < nb_mine;
+        const float sk_a = hdr[c * 8] * qscale, sk_b = two ? hdr[(c + 1) * 8] * qscale : 0.0f;
+        // keys 0 .. visible of the two blocks are seen by the row (Eq. 1: K_{<=t}; Eq. 9: none past the context)
+        const int visible = min(lim - (key0 + c * kBlockSize), two ? 2 * kBlockSize - 1 : kBlockSize - 1);
         tmem_ld_wait32(s);
-        if (visible >= 2 * kBlockSize - 1 && c2 + 1 < nb) {
-          // both blocks wholly visible (all but those on the causal diagonal and the tile's last): a K scale is
-          // not negative, so a block's largest logit is its largest accumulator times the scale
-          float mx_a = __uint_as_float(s[0]), mx_b = __uint_as_float(s[16]);
+        if (visible < 2 * kBlockSize - 1) {
 #pragma unroll
-          for (int j = 1; j < 16; ++j) { mx_a = fmaxf(mx_a, __uint_as_float(s[j])); mx_b = fmaxf(mx_b, __uint_as_float(s[16 + j])); }
-          m_tile = fmaxf(m_tile, fmaxf(mx_a * sk8[c2], mx_b * sk8[c2 + 1]));
-        } else {
+          for (int j = 0; j < 32; ++j) s[j] = j <= visible ? s[j] : 0xFF800000u;      // -inf
+        }
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (j <= visible && (j < 16 || c2 + 1 < nb)) m_tile = fmaxf(m_tile, __uint_as_float(s[j]) * (j < 16 ? sk8[c2] : sk8[c2 + 1]));
+        for (int h = 0; h < 2; ++h) {
+          float mx[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mx[j] = __uint_as_float(s[16 * h + j]);
+#pragma unroll
+          for (int j = 4; j < 16; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(s[16 * h + j]));
+          // a K scale is not negative, so a block's largest logit is its largest accumulator times the scale
+          const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          if (m_blk > -INFINITY) m_half = fmaxf(m_half, m_blk * (h ? sk_b : sk_a));
         }
       }
+      // The two threads of a row tell each other their half's maximum, cut to its upper 16 bits, and both take the
+      // larger of the two cut values as the tile's: a reference need not be the exact maximum, but the two must
+      // agree on it.  (Two buffers by the parity of the team's tile: the partner may be a tile ahead, not two.)
+      unsigned short* xrow = xch + ((team * 2 + (use & 1u)) * 2) * kPuRows + r;
+      xrow[half * kPuRows] = static_cast<unsigned short>(__float_as_uint(m_half) >> 16);
+      // the tile's scales move to a place of the team's own: the second pass needs them after the V slot, where
+      // they arrived, has been handed back to the copy warp
+      float* scl = reinterpret_cast<float*>(smem + C::kSclOff) + team * (2 * kPuTileBlocks);
+      if ((tid & (kPuTeam - 1)) < 2 * kPuTileBlocks) scl[tid & (kPuTeam - 1)] = hdr[((tid & (kPuTeam - 1)) >> 1) * 8 + (tid & 1)];
+      PF_TRACE(tr_pass_a);
+      // the P V instructions of the team's tile before must have left the team's operands (and its accumulator);
+      // they ran while the first pass was made
+      if (use > 0 && (warp & 7) == 0) {
+        const bool ok = wait_bar(&bar_vdone[team], (use - 1) & 1u, abort_flag);
+        bad = !__all_sync(0xffffffffu, ok);
+      }
+      bad = barrier_or(1 + team, kPuTeam, bad);
+      if (bad) break;
+      tc_fence_after();
+      PF_TRACE(tr_wait_pv);
+      const float m_tile = fmaxf(__uint_as_float(static_cast<uint32_t>(xrow[0]) << 16), __uint_as_float(static_cast<uint32_t>(xrow[kPuRows]) << 16));
       // lazy references: moved only when the tile would push a probability (or a scale ratio) past the margin
       const bool move_m = m_tile > m_ref + kPuMaxLag;             // also true for the row's first visible key (m_ref = -inf)
       const bool move_v = v_tile > v_ref * kPuScaleLag;           // uniform over the team; true for the first non-zero scale
@@ -460,21 +488,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       if (move_v) factor *= v_ref > 0.0f ? __fdividef(v_ref, v_new) : 0.0f;
       // tensor-memory accesses are warp-wide: the warp rescales if any of its rows has to (the others by 1)
       const bool rescale = __any_sync(0xffffffffu, move_m || move_v) && use > 0;
-      PF_TRACE(tr_pass_a);
-      // the P V instructions of the team's tile before must have left the team's operands (and its accumulator);
-      // they ran while the first pass was made
-      if (use > 0) {
-        if ((warp & 7) == 0) {
-          const bool ok = wait_bar(&bar_vdone[team], (use - 1) & 1u, abort_flag);
-          bad = !__all_sync(0xffffffffu, ok);
-        }
-        bad = barrier_or(1 + team, kPuTeam, bad);
-        if (bad) break;
-        tc_fence_after();
-      }
-      PF_TRACE(tr_wait_pv);
       if (rescale) {
-#pragma unroll
+#pragma unroll 1
         for (int i = 0; i < 4; ++i) {
           uint32_t o[16];
           tmem_ld16_issue(o_cols + 16 * i, o);
@@ -491,10 +506,9 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       const float m_use = m_ref == -INFINITY ? 0.0f : m_ref;
       const float v_inv = v_ref > 0.0f ? 1.0f / v_ref : 0.0f;
       // ---- the V tile widened into the team's f16 operand; the copy slot is then free for the team's next tile ---
-#pragma unroll
-      for (int ci = 0; ci < kPuTileBlocks / 2; ++ci) {
+#pragma unroll 1
+      for (int ci = 0; ci < nb_mine; ++ci) {
         const int c = c_lo + ci;
-        if (c >= nb) break;                               // uniform over the warp: the P V instructions stop at block nb
         // dim r of V^T, the 16 tokens of block c: widened to f16 (exact; E4M3 codes come out divided by 2^8)
         const uint4 vc = *reinterpret_cast<const uint4*>(st + c * C::kPart + (r >> 3) * 128 + (r & 7) * 16);
         const int keep = nkeys - c * kBlockSize;          // tokens of the block inside the context (Eq. 9)
@@ -508,30 +522,32 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         }
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          vw[2 * j] = p.kv_e5m2 ? e5m2x2_to_f16x2_lo(cw[j]) : e4m3x2_to_f16x2_small(cw[j], 0x1404u);
-          vw[2 * j + 1] = p.kv_e5m2 ? e5m2x2_to_f16x2_hi(cw[j]) : e4m3x2_to_f16x2_small(cw[j], 0x3424u);
+          vw[2 * j] = kE5m2 ? e5m2x2_to_f16x2_lo(cw[j]) : e4m3x2_to_f16x2_small(cw[j], 0x1404u);
+          vw[2 * j + 1] = kE5m2 ? e5m2x2_to_f16x2_hi(cw[j]) : e4m3x2_to_f16x2_small(cw[j], 0x3424u);
         }
         *reinterpret_cast<uint4*>(vrow + (2 * c) * 128) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
         *reinterpret_cast<uint4*>(vrow + (2 * c + 1) * 128) = make_uint4(vw[4], vw[5], vw[6], vw[7]);
       }
       __syncwarp();
       if (lane == 0) mbar_arrive(&bar_vread[team]);       // the V slot may take the team's next tile
-      PF_TRACE(tr_pass_b);
-
+      PF_TRACE(tr_widen);
 
       // ---- second pass: probabilities of this thread's blocks against the reference (f16) ----------------------
+      // p * pv = 2^(s * sk - m + log2 pv): the V scale rides in the exponent, and a block's sum of p is recovered
+      // from the sum of p * pv with one division.  A V scale of zero (an all-zero block: its codes are zero too)
+      // is replaced by a tiny one, a K scale of zero likewise (so that a masked logit stays -inf).
       bool s_freed = false;
-#pragma unroll
-      for (int ci = 0; ci < kPuTileBlocks / 2; ci += 2) {         // two cache blocks per trip to tensor memory
+#pragma unroll 1
+      for (int ci = 0; ci < nb_mine; ci += 2) {
         const int c = c_lo + ci;
-        if (c >= nb) break;                               // uniform over the warp
         uint32_t s[32];
         tmem_ld32_issue(s_cols + 16 * c, s);
-        const float sk_a = half ? sk8[4 + ci] : sk8[ci], sk_b = half ? sk8[5 + ci] : sk8[1 + ci];
-        const float pv_a = (half ? sv8[4 + ci] : sv8[ci]) * v_inv, pv_b = (half ? sv8[5 + ci] : sv8[1 + ci]) * v_inv;   // at most 2^4
-        const int visible = lim - (key0 + c * kBlockSize);
+        const bool two = ci + 1 < nb_mine;
+        const float sk_a = fmaxf(scl[2 * c] * qscale, 1e-30f), sk_b = fmaxf(two ? scl[2 * c + 2] * qscale : 0.0f, 1e-30f);
+        const float pv_a = fmaxf(scl[2 * c + 1] * v_inv, 0x1p-24f), pv_b = fmaxf(two ? scl[2 * c + 3] * v_inv : 0.0f, 0x1p-24f);   // at most 2^4
+        const int visible = min(lim - (key0 + c * kBlockSize), two ? 2 * kBlockSize - 1 : kBlockSize - 1);
         tmem_ld_wait32(s);
-        if (ci + 2 >= kPuTileBlocks / 2 || c + 2 >= nb) {
+        if (ci + 2 >= nb_mine) {
           // the thread's last logits of the tile are in registers: the buffer goes back before the probabilities
           // are made, so that the tile after next is multiplied meanwhile
           tc_fence_before();
@@ -539,38 +555,30 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
           if (lane == 0) mbar_arrive(&bar_sfree[team]);
           s_freed = true;
         }
+        if (visible < 2 * kBlockSize - 1) {
 #pragma unroll
-        for (int blk = 0; blk < 2; ++blk) {
-          if (c + blk >= nb) break;                       // uniform
-          const float sk = blk ? sk_b : sk_a, pv = blk ? pv_b : pv_a;
+          for (int j = 0; j < 32; ++j) s[j] = j <= visible ? s[j] : 0xFF800000u;
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const float sk = h ? sk_b : sk_a, pv = h ? pv_b : pv_a;
+          float lg;
+          asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(pv));
+          const float shift = lg - m_use;
+          float l_a = 0.0f, l_b = 0.0f;
           uint32_t pw[8];
-          if (visible >= 16 * blk + kBlockSize - 1 && pv > 0.0f) {
-            // the block is wholly visible: the V scale rides in the exponent, p * pv = 2^(s * sk - m + log2 pv),
-            // and the block's sum of p is recovered from the sum of p * pv with one division
-            float lg;
-            asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(pv));
-            const float shift = lg - m_use;
-            float l_blk = 0.0f;
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int j = 16 * blk + 2 * e;
-              const float y0 = ex2(fmaf(__uint_as_float(s[j]), sk, shift)), y1 = ex2(fmaf(__uint_as_float(s[j + 1]), sk, shift));
-              l_blk += y0 + y1;
-              pw[e] = pack_f16x2(y0, y1);                 // at most 2^8 * 2^4: well inside f16
-            }
-            l_row += __fdividef(l_blk, pv);
-          } else {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) {
-              const int j = 16 * blk + 2 * e;
-              const float x0 = ex2(__uint_as_float(s[j]) * sk - m_use), x1 = ex2(__uint_as_float(s[j + 1]) * sk - m_use);
-              const float p0 = (j <= visible) ? x0 : 0.0f, p1 = (j + 1 <= visible) ? x1 : 0.0f;
-              l_row += p0 + p1;
-              pw[e] = pack_f16x2(p0 * pv, p1 * pv);
-            }
+          for (int e = 0; e < 8; ++e) {
+            const float y0 = ex2(fmaf(__uint_as_float(s[16 * h + 2 * e]), sk, shift)), y1 = ex2(fmaf(__uint_as_float(s[16 * h + 2 * e + 1]), sk, shift));
+            l_a += y0;
+            l_b += y1;
+            pw[e] = pack_f16x2(y0, y1);                   // at most 2^8 * 2^4: well inside f16
           }
-          *reinterpret_cast<uint4*>(prow + (2 * (c + blk)) * 128) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
-          *reinterpret_cast<uint4*>(prow + (2 * (c + blk) + 1) * 128) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
+          l_row += __fdividef(l_a + l_b, pv);
+          if (h == 0 || two) {
+            *reinterpret_cast<uint4*>(prow + (2 * (c + h)) * 128) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
+            *reinterpret_cast<uint4*>(prow + (2 * (c + h) + 1) * 128) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
+          }
         }
       }
       if (!s_freed) {                                     // a warp whose blocks lie past the end of the context
@@ -590,7 +598,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       const int rec = blockIdx.y * gridDim.x + blockIdx.x;
       if (rec < kTraceMaxCtas) {
         unsigned long long* out = p.trace + static_cast<size_t>(rec) * kTraceSlots;
-        out[0] = n_tiles; out[1] = tr_wait_in; out[2] = tr_pass_a; out[3] = tr_wait_pv; out[4] = tr_pass_b; out[5] = clock64() - tr_start; out[6] = tr_wait_s; out[7] = tr_wait_v; out[13] = tr_skew;
+        out[0] = n_tiles; out[1] = tr_wait_in; out[2] = tr_pass_a; out[3] = tr_wait_pv; out[4] = tr_pass_b; out[5] = clock64() - tr_start; out[7] = tr_widen; out[13] = tr_skew;
       }
     }
 #endif
@@ -618,7 +626,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       const float w_me = l_me > 0.0f ? ex2(m_ref - M) : 0.0f, w_ot = l_ot > 0.0f ? ex2(m_ot - M) : 0.0f;
       const float den = w_me * l_me + w_ot * l_ot;
       const float inv = den > 0.0f ? 1.0f / den : 0.0f;
-      const float unit = p.kv_e5m2 ? 1.0f : 256.0f;        // the widened E4M3 codes carry their values / 2^8
+      const float unit = kE5m2 ? 1.0f : 256.0f;        // the widened E4M3 codes carry their values / 2^8
       const float k_me = w_me * v_ref * inv * unit, k_ot = w_ot * v_ot * inv * unit;
       const bool other_ran = n_tiles > (team ^ 1);
       // the four threads of row r store 32 dims each
@@ -695,9 +703,12 @@ int launch_paged_prefill_umma(const coopt_cache* c, const void* q, void* out, co
   if (!encode_cache_map(&map_part, c->data, granules, PuCfg::kGran, PuCfg::kPart / 8) ||
       !encode_cache_map(&map_hdr, c->data, granules, PuCfg::kGran, kFp8Header / 8))
     return COOPT_ERR_CUDA;
-  if (!configure_kernel_smem(reinterpret_cast<const void*>(&paged_prefill_umma_kernel), PuCfg::kSmemBytes)) return COOPT_ERR_CUDA;
+  const bool e5m2 = c->dtype == COOPT_KV_FP8_E5M2;
+  const void* kernel = e5m2 ? reinterpret_cast<const void*>(&paged_prefill_umma_kernel<true>) : reinterpret_cast<const void*>(&paged_prefill_umma_kernel<false>);
+  if (!configure_kernel_smem(kernel, PuCfg::kSmemBytes)) return COOPT_ERR_CUDA;
   const dim3 grid(static_cast<unsigned>(tiles), static_cast<unsigned>(c->num_kv_heads));
-  paged_prefill_umma_kernel<<<grid, kPuThreads, PuCfg::kSmemBytes, stream>>>(p, map_part, map_hdr);
+  if (e5m2) paged_prefill_umma_kernel<true><<<grid, kPuThreads, PuCfg::kSmemBytes, stream>>>(p, map_part, map_hdr);
+  else paged_prefill_umma_kernel<false><<<grid, kPuThreads, PuCfg::kSmemBytes, stream>>>(p, map_part, map_hdr);
   return cudaGetLastError() == cudaSuccess ? COOPT_OK : COOPT_ERR_CUDA;
 }
 
