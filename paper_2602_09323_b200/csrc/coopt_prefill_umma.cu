@@ -5,14 +5,15 @@
 // A CTA owns one (sequence, kv head, tile of consecutive query tokens).  Its 128 rows are the (query
 // token, query head of the group) pairs of the tile, so the K/V stream of the kv head is fetched once
 // for all G heads (Algorithm 2).
-//     S [128 rows x 128 keys] = Q  [128 x D] . Ktile^T      kind::f8f6f4: the cache codes as they are, Q as two exact
-//                                                            E4M3 terms of the bf16 query
-//     O [128 rows x D]       += P  [128 x 128 keys] . Vtile  kind::f16: P rounded once to f16, the V codes widened to f16 (exact)
+//     S [128 rows x 128 keys] = Q  [128 x D] . Ktile^T      kind::f8f6f4: the cache codes as they are, Q as two E4M3
+//                                                            terms of the bf16 query, both operands in shared memory
+//     O [128 rows x D]       += P  [128 x 128 keys] . Vtile  kind::f16: P rounded once to f16 and read from tensor
+//                                                            memory, the V codes widened to f16 (exact) in shared memory
 // with fp32 accumulators in tensor memory.  The K scale of a block multiplies the logits of its 16 keys,
 // the V scale is folded into the probabilities.  (Carrying P as E4M3 terms instead, three per probability for
 // the same 11 bits, kept the V codes as they are but cost five conversions per pair of probabilities on the
-// SM's conversion pipe; widening V costs one conversion per pair of codes, and a tile of V is a sixteenth of a
-// tile of P per query row.)
+// SM's conversion pipe; widening V costs a few integer instructions per pair of codes, and a tile of V is a
+// sixteenth of a tile of P per query row.)
 //
 // The context is walked once, 128 keys (eight cache blocks) at a time; even tiles go to softmax team 0, odd
 // tiles to team 1, and each team keeps an online softmax of its own for all 128 rows: a reference maximum per
@@ -22,20 +23,23 @@
 // reference means reading, scaling and writing back the row's 128 accumulators; f16 probabilities have room
 // for that factor, and after the first tiles a reference hardly ever moves.  At the end the two teams'
 // results are merged like two split-KV pieces.  Per tile the tensor core does 8 instructions for the logits
-// and 8 for P V; nothing is computed twice.  (An earlier version walked the context twice, row maxima first,
-// so that nothing was ever rescaled: a third more tensor work, every tile's logits read and scaled twice by
-// the teams, and a team idle while its own P V instructions ran.)
+// and 8 for P V; nothing is computed twice.
+//
+// Tensor memory (512 columns): the logits of team b's tile in columns 128 b .. 128 b + 127, its accumulator in
+// 256 + 128 b ...  A team writes its probabilities, two f16 to a column, over logits it has already consumed
+// (keys 0-63 of the tile in columns 0-31 of its buffer, keys 64-127 in columns 64-95), so a team's next logits
+// can be computed only once the P V instructions of its tile before are done; the other team's tile and the
+// widening of the next V tile fill that time.
 //
 // Warp roles (608 threads):
 //   warps 0-7, 8-15  two softmax teams.  Two threads of a team share row r: warps 0-3 of the team take the
-//               tile's first four cache blocks, warps 4-7 the last four.  A tile's logits are read from tensor
-//               memory twice: a first pass for the row's maximum, which both threads of a row make over the whole
-//               row (so that they agree on the reference without meeting) and which touches none of the team's
-//               operand buffers, so it runs while the P V instructions of the team's tile before are still in
-//               flight; and a second pass for the probabilities of the thread's own blocks;
+//               tile's first four cache blocks, warps 4-7 the last four, in both passes over the logits (a first
+//               pass for the maximum, a second for the probabilities); the two halves' maxima meet through
+//               shared memory.  Before a tile's logits arrive, the team widens the tile's V^T into one of its two
+//               f16 operands (the other may still be read by the P V instructions of the tile before);
 //   warp 16     copies: gather requests over the tensor map of the cache into two slots for K tiles, freed as
 //               soon as the logits are computed, and two slots for V tiles with the tile's scales, freed as
-//               soon as the team has widened the codes into its f16 operand;
+//               soon as the team has widened the codes;
 //   warp 17     one lane issues the S instructions; warp 18 one lane issues the P V instructions.
 // Every wait is bounded; a wait that runs out is reported in the status word and all roles leave through
 // the common exit, which frees the tensor memory.
@@ -88,10 +92,9 @@ struct PuCfg {
   static constexpr int kRingOff = 0;                              // K slot 0, K slot 1, V slot 0, V slot 1
   static constexpr int kVRingOff = kRingOff + 2 * kKSlot;
   static constexpr int kQOff = kVRingOff + 2 * kVSlot;            // Q: lead term, remainder term
-  static constexpr int kPOff = kQOff + 2 * kOperand;              // P: [team], f16
-  static constexpr int kV16Off = kPOff + 2 * kOperand16;          // V^T of a tile widened to f16: [team]
-  static constexpr int kBarOff = kV16Off + 2 * kOperand16;
-  static constexpr int kNumBars = kPuSlots + 2 + 2 + 2 + 2 + 2 + 2;   // full, kdone, vdone, vread, sfull, sfree, pfull
+  static constexpr int kV16Off = kQOff + 2 * kOperand;            // V^T of a tile widened to f16: [team][parity of the team's tile]
+  static constexpr int kBarOff = kV16Off + 4 * kOperand16;
+  static constexpr int kNumBars = kPuSlots + 2 + 2 + 2 + 2 + 2;   // full, kdone, vdone, vread, sfull, pfull
   static constexpr int kMiscOff = kBarOff + kNumBars * 8;
   static constexpr int kXchOff = kMiscOff + 64;                   // [team][parity][half][row] upper halves of fp32 maxima
   static constexpr int kSclOff = kXchOff + 2 * 2 * 2 * kPuRows * 2;   // [team][block][K scale, V scale] of the tile being worked on
@@ -125,7 +128,6 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   uint8_t* kring = smem + C::kRingOff;
   uint8_t* vring = smem + C::kVRingOff;
   uint8_t* qbuf = smem + C::kQOff;
-  uint8_t* pbuf = smem + C::kPOff;
   uint8_t* v16buf = smem + C::kV16Off;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + C::kBarOff);
   uint64_t* bar_full = bars;                         // [4] the copies into the slot have landed (K slots 0-1, V slots 2-3)
@@ -133,8 +135,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   uint64_t* bar_vdone = bar_kdone + 2;               // [2] the P V instructions of the team's tile are done
   uint64_t* bar_vread = bar_vdone + 2;               // [2] the team has widened the V tile in the slot (and read its scales)
   uint64_t* bar_sfull = bar_vread + 2;               // [2] logits of a tile are in tensor memory (buffer = tile & 1 = team)
-  uint64_t* bar_sfree = bar_sfull + 2;               // [2] the team's eight warps have read them for the last time
-  uint64_t* bar_pfull = bar_sfree + 2;               // [2] the team's two f16 operands of a tile are in shared memory
+  uint64_t* bar_pfull = bar_sfull + 2;               // [2] the team's probabilities of a tile are in tensor memory, its V operand in shared memory
   unsigned short* xch = reinterpret_cast<unsigned short*>(smem + C::kXchOff);
   int* misc = reinterpret_cast<int*>(smem + C::kMiscOff);   // [0] sequence, [1] first query, [2] abort flag, [3] tensor memory
   volatile int* abort_flag = misc + 2;
@@ -160,7 +161,7 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     for (int i = 0; i < kPuSlots; ++i) mbar_init(&bar_full[i], 1);
     for (int i = 0; i < 2; ++i) {
       mbar_init(&bar_kdone[i], 1); mbar_init(&bar_vdone[i], 1); mbar_init(&bar_vread[i], 8);
-      mbar_init(&bar_sfull[i], 1); mbar_init(&bar_sfree[i], 8); mbar_init(&bar_pfull[i], kPuTeam);
+      mbar_init(&bar_sfull[i], 1); mbar_init(&bar_pfull[i], kPuTeam);
     }
     mbar_fence_init();
   }
@@ -291,22 +292,31 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       }
       const int sl = t & 1;
       const uint32_t use = static_cast<uint32_t>(t >> 1);
+      // The V parts and the scales are requested as soon as the team has widened the V tile that was in the slot
+      // (early in its work on that tile), the K parts once the logits of the K tile in the slot exist.  (The
+      // slots' users before are the team's tile two back; a wait for phase k follows the one for phase k - 1.)
       if (lane == 0) {
-        // the slots' users before: the team's tile two back (a wait for phase k follows the one for phase k - 1)
-        if (t >= 2) ok = wait_bar(&bar_kdone[sl], (use - 1) & 1u, abort_flag) && wait_bar(&bar_vread[sl], (use - 1) & 1u, abort_flag);
+        if (t >= 2) ok = wait_bar(&bar_vread[sl], (use - 1) & 1u, abort_flag);
         if (ok) {
-          mbar_expect_tx(&bar_full[sl], ngroups * 4 * C::kPart);
           mbar_expect_tx(&bar_full[2 + sl], ngroups * 4 * (C::kPart + kFp8Header));
-          pend_mask |= (1u << sl) | (4u << sl);
-          pend_par = (pend_par & ~((1u << sl) | (4u << sl))) | ((use & 1u) << sl) | ((use & 1u) << (2 + sl));
+          pend_mask |= 4u << sl;
+          pend_par = (pend_par & ~(4u << sl)) | ((use & 1u) << (2 + sl));
         }
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
-      if (lane < 3 * ngroups) {
-        uint8_t* dst = what == 0 ? kring + sl * C::kKSlot : vring + sl * C::kVSlot;
-        gather4_g2s(dst + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[what == 0 ? sl : 2 + sl]);
+      if (lane < 3 * ngroups && what != 0) gather4_g2s(vring + sl * C::kVSlot + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[2 + sl]);
+      if (lane == 0) {
+        if (t >= 2) ok = wait_bar(&bar_kdone[sl], (use - 1) & 1u, abort_flag);
+        if (ok) {
+          mbar_expect_tx(&bar_full[sl], ngroups * 4 * C::kPart);
+          pend_mask |= 1u << sl;
+          pend_par = (pend_par & ~(1u << sl)) | ((use & 1u) << sl);
+        }
       }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      if (lane < 3 * ngroups && what == 0) gather4_g2s(kring + sl * C::kKSlot + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[sl]);
     }
     if (!ok && lane == 0) atomicCAS(p.status, 0, COOPT_ERR_TIMEOUT);
   } else if (warp == kPuSWarp) {
@@ -323,7 +333,8 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
 #ifdef COOPT_TRACE
         const long long ts1 = clock64();
 #endif
-        if (ok && use > 0) ok = wait_bar(&bar_sfree[buf], (use - 1) & 1u, abort_flag);
+        // the buffer also holds the probabilities of the team's tile before, until their P V instructions are done
+        if (ok && use > 0) ok = wait_bar(&bar_vdone[buf], (use - 1) & 1u, abort_flag);
         if (!ok) break;
 #ifdef COOPT_TRACE
         if (p.trace != nullptr && blockIdx.y * gridDim.x + blockIdx.x < kTraceMaxCtas) {
@@ -346,9 +357,10 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
     // ================= outputs: O_team += P . Vtile (one lane) ===============================================
     if (lane == 0) {
       bool ok = true;
-      // both operands of P V are f16, K-major: 8 rows x 16 bytes (8 values) per core matrix, cores of a row group 128 bytes
-      // apart along the keys, row groups 2048 bytes apart
-      const uint64_t desc_v = umma_desc(smem_u32(v16buf), 128, 2048), desc_p = umma_desc(smem_u32(pbuf), 128, 2048);
+      // P is read from tensor memory, where the team left it over its own logits (keys 0-63 of the tile in columns
+      // 0-31 of the team's buffer, keys 64-127 in columns 64-95); V^T is f16 in shared memory, K-major: 8 rows x 16
+      // bytes (8 values) per core matrix, cores of a row group 128 bytes apart along the keys, row groups 2048 bytes apart
+      const uint64_t desc_v = umma_desc(smem_u32(v16buf), 128, 2048);
       for (int t = 0; t < n_tiles && ok; ++t) {
         const uint32_t team = t & 1u, use = static_cast<uint32_t>(t >> 1);
 #ifdef COOPT_TRACE
@@ -363,9 +375,17 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
 #endif
         tc_fence_after();
         const int nb = min(kPuTileBlocks, n_blocks - t * kPuTileBlocks);      // 16 keys (one cache block) per instruction
-        const uint64_t dv = desc_v + ((team * C::kOperand16) >> 4), dp = desc_p + ((team * C::kOperand16) >> 4);
-        for (int ks = 0; ks < nb; ++ks) umma_f16(tmem_o + 128 * team, dp + ks * 16, dv + ks * 16, umma_idesc(D), (use | ks) != 0);
-        umma_commit(&bar_vdone[team]);      // the team's two f16 operands are free again, its accumulator is at rest
+        const uint64_t dv = desc_v + (((team * 2 + (use & 1u)) * C::kOperand16) >> 4);
+        const uint32_t p_cols = tmem + 128 * team;
+        if (nb == kPuTileBlocks) {                        // all but a context's last tile: eight instructions in a row
+#pragma unroll
+          for (int ks = 0; ks < kPuTileBlocks; ++ks)
+            umma_f16_ts(tmem_o + 128 * team, p_cols + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), dv + ks * 16, umma_idesc(D), (use | ks) != 0);
+        } else {
+          for (int ks = 0; ks < nb; ++ks)
+            umma_f16_ts(tmem_o + 128 * team, p_cols + (ks < 4 ? 8 * ks : 64 + 8 * (ks - 4)), dv + ks * 16, umma_idesc(D), (use | ks) != 0);
+        }
+        umma_commit(&bar_vdone[team]);      // the team's logits buffer and this V operand are free again, its accumulator is at rest
 #ifdef COOPT_TRACE
         {
           const long long ti = clock64();
@@ -382,16 +402,16 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
   } else {
     // ================= softmax teams ================================================================================
     const int team = warp >> 3;
-    const int c_lo = half * (kPuTileBlocks / 2);            // the first of this thread's four cache blocks of a tile
+    const int tt = tid & (kPuTeam - 1);           // this thread within its team
+    const int c_lo = half * (kPuTileBlocks / 2);  // the first of this thread's four cache blocks of a tile
     bool bad = false;
     float m_ref = -INFINITY;     // the row's reference maximum (the same in both threads of the row)
     float l_row = 0.0f;          // this thread's share of the row's sum of exponentials, against m_ref
     float v_ref = 0.0f;          // the team's reference V scale (uniform over the team)
-    uint8_t* prow = pbuf + team * C::kOperand16 + (r >> 3) * 2048 + (r & 7) * 16;      // row r of the team's P operand
-    uint8_t* vrow = v16buf + team * C::kOperand16 + (r >> 3) * 2048 + (r & 7) * 16;    // dim r of the team's V^T operand
     const uint32_t o_cols = tmem_o + 128 * team + 64 * half + lane_base;               // this thread's 64 of the row's accumulators
     const uint8_t* st = vring + team * C::kVSlot;                                      // the team's V slot: V parts, then the scales
     const uint32_t s_cols = tmem + 128 * team + lane_base;                             // the team's logits buffer
+    float* scl = reinterpret_cast<float*>(smem + C::kSclOff) + team * (2 * kPuTileBlocks);   // the tile's [block][K scale, V scale]
 
     // A wait that runs out is made known to the whole team by the named barrier behind it, and the team leaves
     // the loop together; the other roles give up on their own waits once the abort flag is up.
@@ -402,110 +422,28 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
 #else
 #define PF_TRACE(acc) do { } while (0)
 #endif
+    // The loops over a tile are kept rolled (32 logits = two cache blocks per trip to tensor memory): unrolled,
+    // the body of this loop was tens of KB of instructions and the teams waited for instruction fetch.
     for (int t = team; t < n_tiles && !bad; t += 2) {
       const uint32_t use = static_cast<uint32_t>(t >> 1);
       const int key0 = t * kPuTileKeys;
       const int nkeys = min(kPuTileKeys, kv_end - key0);
       const int nb = (nkeys + kBlockSize - 1) / kBlockSize;
-      // ---- the tile's scales (they arrive with its V parts) and its logits -------------------------------------
-      // One warp of the team watches the barriers; the other seven wait for it on a named barrier, where the
-      // hardware parks them, instead of polling along with it.
+      const int nb_mine = min(nb - c_lo, kPuTileBlocks / 2);                 // this thread's blocks of the tile (<= 0: none)
+      // ---- the tile's V parts and scales have landed: V^T widened into one of the team's two f16 operands ---------
+      // (the one that the P V instructions of the team's tile before do not read; those of the tile before that were
+      // done before this tile's logits could be started).  One warp of the team watches the barrier; the other
+      // seven wait for it on a named barrier, where the hardware parks them, instead of polling along with it.
       if ((warp & 7) == 0) {
-        bool ok = wait_bar(&bar_full[2 + team], use & 1u, abort_flag);
-        ok = ok && wait_bar(&bar_sfull[team], use & 1u, abort_flag);
-        // the logits are computed: the tile's K slot can be refilled
-        if (ok && lane == 0) mbar_arrive(&bar_kdone[team]);
+        const bool ok = wait_bar(&bar_full[2 + team], use & 1u, abort_flag);
         bad = !__all_sync(0xffffffffu, ok);
       }
       bad = barrier_or(1 + team, kPuTeam, bad);           // uniform over the team from here
       if (bad) break;
-      tc_fence_after();
       PF_TRACE(tr_wait_in);
-      // The loops over the tile are kept rolled (32 logits = two cache blocks per trip to tensor memory): unrolled,
-      // the body of this loop was tens of KB of instructions and the teams waited for instruction fetch.
-      const float* hdr = reinterpret_cast<const float*>(st + C::kHdrOff);    // [block][8]: K scale, V scale, zeros
-      const int nb_mine = min(nb - c_lo, kPuTileBlocks / 2);                 // this thread's blocks of the tile (<= 0: none)
-
-      // ---- first pass: the maximum of this thread's half of the row; the tile's largest V scale ------------------
-      float m_half = -INFINITY, v_tile = 0.0f;
-#pragma unroll
-      for (int c = 0; c < kPuTileBlocks; ++c) v_tile = fmaxf(v_tile, c < nb ? hdr[c * 8 + 1] : 0.0f);
-#pragma unroll 1
-      for (int ci = 0; ci < nb_mine; ci += 2) {
-        const int c = c_lo + ci;
-        uint32_t s[32];
-        tmem_ld32_issue(s_cols + 16 * c, s);
-        const bool two = ci + 1 < nb_mine;
-        const float sk_a = hdr[c * 8] * qscale, sk_b = two ? hdr[(c + 1) * 8] * qscale : 0.0f;
-        // keys 0 .. visible of the two blocks are seen by the row (Eq. 1: K_{<=t}; Eq. 9: none past the context)
-        const int visible = min(lim - (key0 + c * kBlockSize), two ? 2 * kBlockSize - 1 : kBlockSize - 1);
-        tmem_ld_wait32(s);
-        if (visible < 2 * kBlockSize - 1) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) s[j] = j <= visible ? s[j] : 0xFF800000u;      // -inf
-        }
-#pragma unroll
-        for (int h = 0; h < 2; ++h) {
-          float mx[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) mx[j] = __uint_as_float(s[16 * h + j]);
-#pragma unroll
-          for (int j = 4; j < 16; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(s[16 * h + j]));
-          // a K scale is not negative, so a block's largest logit is its largest accumulator times the scale
-          const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-          if (m_blk > -INFINITY) m_half = fmaxf(m_half, m_blk * (h ? sk_b : sk_a));
-        }
-      }
-      // The two threads of a row tell each other their half's maximum, cut to its upper 16 bits, and both take the
-      // larger of the two cut values as the tile's: a reference need not be the exact maximum, but the two must
-      // agree on it.  (Two buffers by the parity of the team's tile: the partner may be a tile ahead, not two.)
-      unsigned short* xrow = xch + ((team * 2 + (use & 1u)) * 2) * kPuRows + r;
-      xrow[half * kPuRows] = static_cast<unsigned short>(__float_as_uint(m_half) >> 16);
-      // the tile's scales move to a place of the team's own: the second pass needs them after the V slot, where
-      // they arrived, has been handed back to the copy warp
-      float* scl = reinterpret_cast<float*>(smem + C::kSclOff) + team * (2 * kPuTileBlocks);
-      if ((tid & (kPuTeam - 1)) < 2 * kPuTileBlocks) scl[tid & (kPuTeam - 1)] = hdr[((tid & (kPuTeam - 1)) >> 1) * 8 + (tid & 1)];
-      PF_TRACE(tr_pass_a);
-      // the P V instructions of the team's tile before must have left the team's operands (and its accumulator);
-      // they ran while the first pass was made
-      if (use > 0 && (warp & 7) == 0) {
-        const bool ok = wait_bar(&bar_vdone[team], (use - 1) & 1u, abort_flag);
-        bad = !__all_sync(0xffffffffu, ok);
-      }
-      bad = barrier_or(1 + team, kPuTeam, bad);
-      if (bad) break;
-      tc_fence_after();
-      PF_TRACE(tr_wait_pv);
-      const float m_tile = fmaxf(__uint_as_float(static_cast<uint32_t>(xrow[0]) << 16), __uint_as_float(static_cast<uint32_t>(xrow[kPuRows]) << 16));
-      // lazy references: moved only when the tile would push a probability (or a scale ratio) past the margin
-      const bool move_m = m_tile > m_ref + kPuMaxLag;             // also true for the row's first visible key (m_ref = -inf)
-      const bool move_v = v_tile > v_ref * kPuScaleLag;           // uniform over the team; true for the first non-zero scale
-      const float m_new = move_m ? m_tile : m_ref;
-      const float v_new = move_v ? v_tile : v_ref;
-      // the factor that brings what has been accumulated so far onto the new references
-      float factor = 1.0f;
-      if (move_m) factor = m_ref == -INFINITY ? 0.0f : ex2(m_ref - m_new);
-      if (move_v) factor *= v_ref > 0.0f ? __fdividef(v_ref, v_new) : 0.0f;
-      // tensor-memory accesses are warp-wide: the warp rescales if any of its rows has to (the others by 1)
-      const bool rescale = __any_sync(0xffffffffu, move_m || move_v) && use > 0;
-      if (rescale) {
-#pragma unroll 1
-        for (int i = 0; i < 4; ++i) {
-          uint32_t o[16];
-          tmem_ld16_issue(o_cols + 16 * i, o);
-          tmem_ld_wait(o);
-#pragma unroll
-          for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
-          tmem_st16(o_cols + 16 * i, o);
-        }
-        tmem_st_wait();
-      }
-      if (move_m) l_row *= m_ref == -INFINITY ? 0.0f : ex2(m_ref - m_new);
-      m_ref = m_new;
-      v_ref = v_new;
-      const float m_use = m_ref == -INFINITY ? 0.0f : m_ref;
-      const float v_inv = v_ref > 0.0f ? 1.0f / v_ref : 0.0f;
-      // ---- the V tile widened into the team's f16 operand; the copy slot is then free for the team's next tile ---
+      // the scales move to a place of the team's own: both passes need them after the V slot has been handed back
+      if (tt < 2 * kPuTileBlocks) scl[tt] = reinterpret_cast<const float*>(st + C::kHdrOff)[(tt >> 1) * 8 + (tt & 1)];
+      uint8_t* vrow = v16buf + (team * 2 + (use & 1u)) * C::kOperand16 + (r >> 3) * 2048 + (r & 7) * 16;    // dim r of V^T
 #pragma unroll 1
       for (int ci = 0; ci < nb_mine; ++ci) {
         const int c = c_lo + ci;
@@ -528,15 +466,98 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         *reinterpret_cast<uint4*>(vrow + (2 * c) * 128) = make_uint4(vw[0], vw[1], vw[2], vw[3]);
         *reinterpret_cast<uint4*>(vrow + (2 * c + 1) * 128) = make_uint4(vw[4], vw[5], vw[6], vw[7]);
       }
+      fence_proxy_async();                                // the tensor core will read what this thread has just written
       __syncwarp();
       if (lane == 0) mbar_arrive(&bar_vread[team]);       // the V slot may take the team's next tile
       PF_TRACE(tr_widen);
 
+      // ---- the tile's logits ------------------------------------------------------------------------------------
+      if ((warp & 7) == 0) {
+        const bool ok = wait_bar(&bar_sfull[team], use & 1u, abort_flag);
+        // the logits are computed: the tile's K slot can be refilled
+        if (ok && lane == 0) mbar_arrive(&bar_kdone[team]);
+        bad = !__all_sync(0xffffffffu, ok);
+      }
+      bad = barrier_or(1 + team, kPuTeam, bad);
+      if (bad) break;
+      tc_fence_after();
+      PF_TRACE(tr_wait_pv);
+
+      // ---- first pass: the maximum of this thread's half of the row; the tile's largest V scale ------------------
+      float m_half = -INFINITY, v_tile = 0.0f;
+#pragma unroll
+      for (int c = 0; c < kPuTileBlocks; ++c) v_tile = fmaxf(v_tile, c < nb ? scl[2 * c + 1] : 0.0f);
+#pragma unroll 1
+      for (int ci = 0; ci < nb_mine; ci += 2) {
+        const int c = c_lo + ci;
+        uint32_t s[32];
+        tmem_ld32_issue(s_cols + 16 * c, s);
+        const bool two = ci + 1 < nb_mine;
+        const float sk_a = scl[2 * c] * qscale, sk_b = two ? scl[2 * c + 2] * qscale : 0.0f;
+        // keys 0 .. visible of the two blocks are seen by the row (Eq. 1: K_{<=t}; Eq. 9: none past the context)
+        const int visible = min(lim - (key0 + c * kBlockSize), two ? 2 * kBlockSize - 1 : kBlockSize - 1);
+        tmem_ld_wait32(s);
+        if (visible < 2 * kBlockSize - 1) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) s[j] = j <= visible ? s[j] : 0xFF800000u;      // -inf
+        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          float mx[4];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) mx[j] = __uint_as_float(s[16 * h + j]);
+#pragma unroll
+          for (int j = 4; j < 16; ++j) mx[j & 3] = fmaxf(mx[j & 3], __uint_as_float(s[16 * h + j]));
+          // a K scale is not negative, so a block's largest logit is its largest accumulator times the scale
+          const float m_blk = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+          if (m_blk > -INFINITY) m_half = fmaxf(m_half, m_blk * (h ? sk_b : sk_a));
+        }
+      }
+      // The two threads of a row tell each other their half's maximum, cut to its upper 16 bits, and both take the
+      // larger of the two cut values as the tile's: a reference need not be the exact maximum, but the two must
+      // agree on it.
+      unsigned short* xrow = xch + (team * 2) * kPuRows + r;
+      xrow[half * kPuRows] = static_cast<unsigned short>(__float_as_uint(m_half) >> 16);
+      bad = barrier_or(1 + team, kPuTeam, bad);
+      if (bad) break;
+      PF_TRACE(tr_pass_a);
+      const float m_tile = fmaxf(__uint_as_float(static_cast<uint32_t>(xrow[0]) << 16), __uint_as_float(static_cast<uint32_t>(xrow[kPuRows]) << 16));
+      // lazy references: moved only when the tile would push a probability (or a scale ratio) past the margin
+      const bool move_m = m_tile > m_ref + kPuMaxLag;             // also true for the row's first visible key (m_ref = -inf)
+      const bool move_v = v_tile > v_ref * kPuScaleLag;           // uniform over the team; true for the first non-zero scale
+      const float m_new = move_m ? m_tile : m_ref;
+      const float v_new = move_v ? v_tile : v_ref;
+      // the factor that brings what has been accumulated so far onto the new references
+      float factor = 1.0f;
+      if (move_m) factor = m_ref == -INFINITY ? 0.0f : ex2(m_ref - m_new);
+      if (move_v) factor *= v_ref > 0.0f ? __fdividef(v_ref, v_new) : 0.0f;
+      // Tensor-memory accesses are warp-wide: the warp rescales if any of its rows has to (the others by 1).  The
+      // accumulator is at rest: the P V instructions of the team's tile before were done before this tile's logits
+      // were started.
+      const bool rescale = __any_sync(0xffffffffu, move_m || move_v) && use > 0;
+      if (rescale) {
+#pragma unroll 1
+        for (int i = 0; i < 4; ++i) {
+          uint32_t o[16];
+          tmem_ld16_issue(o_cols + 16 * i, o);
+          tmem_ld_wait(o);
+#pragma unroll
+          for (int j = 0; j < 16; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * factor);
+          tmem_st16(o_cols + 16 * i, o);
+        }
+      }
+      if (move_m) l_row *= m_ref == -INFINITY ? 0.0f : ex2(m_ref - m_new);
+      m_ref = m_new;
+      v_ref = v_new;
+      const float m_use = m_ref == -INFINITY ? 0.0f : m_ref;
+      const float v_inv = v_ref > 0.0f ? 1.0f / v_ref : 0.0f;
+
       // ---- second pass: probabilities of this thread's blocks against the reference (f16) ----------------------
       // p * pv = 2^(s * sk - m + log2 pv): the V scale rides in the exponent, and a block's sum of p is recovered
       // from the sum of p * pv with one division.  A V scale of zero (an all-zero block: its codes are zero too)
-      // is replaced by a tiny one, a K scale of zero likewise (so that a masked logit stays -inf).
-      bool s_freed = false;
+      // is replaced by a tiny one, a K scale of zero likewise (so that a masked logit stays -inf).  The
+      // probabilities of 32 keys, two to a column, go back to tensor memory over the first half of the 32 logits
+      // this thread has consumed most recently: the tensor core takes P from there.
 #pragma unroll 1
       for (int ci = 0; ci < nb_mine; ci += 2) {
         const int c = c_lo + ci;
@@ -547,18 +568,11 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
         const float pv_a = fmaxf(scl[2 * c + 1] * v_inv, 0x1p-24f), pv_b = fmaxf(two ? scl[2 * c + 3] * v_inv : 0.0f, 0x1p-24f);   // at most 2^4
         const int visible = min(lim - (key0 + c * kBlockSize), two ? 2 * kBlockSize - 1 : kBlockSize - 1);
         tmem_ld_wait32(s);
-        if (ci + 2 >= nb_mine) {
-          // the thread's last logits of the tile are in registers: the buffer goes back before the probabilities
-          // are made, so that the tile after next is multiplied meanwhile
-          tc_fence_before();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&bar_sfree[team]);
-          s_freed = true;
-        }
         if (visible < 2 * kBlockSize - 1) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) s[j] = j <= visible ? s[j] : 0xFF800000u;
         }
+        uint32_t pw[16];
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
           const float sk = h ? sk_b : sk_a, pv = h ? pv_b : pv_a;
@@ -566,27 +580,19 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
           asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(pv));
           const float shift = lg - m_use;
           float l_a = 0.0f, l_b = 0.0f;
-          uint32_t pw[8];
 #pragma unroll
           for (int e = 0; e < 8; ++e) {
             const float y0 = ex2(fmaf(__uint_as_float(s[16 * h + 2 * e]), sk, shift)), y1 = ex2(fmaf(__uint_as_float(s[16 * h + 2 * e + 1]), sk, shift));
             l_a += y0;
             l_b += y1;
-            pw[e] = pack_f16x2(y0, y1);                   // at most 2^8 * 2^4: well inside f16
+            pw[8 * h + e] = pack_f16x2(y0, y1);           // at most 2^8 * 2^4: well inside f16
           }
           l_row += __fdividef(l_a + l_b, pv);
-          if (h == 0 || two) {
-            *reinterpret_cast<uint4*>(prow + (2 * (c + h)) * 128) = make_uint4(pw[0], pw[1], pw[2], pw[3]);
-            *reinterpret_cast<uint4*>(prow + (2 * (c + h) + 1) * 128) = make_uint4(pw[4], pw[5], pw[6], pw[7]);
-          }
         }
+        tmem_st16(s_cols + 64 * half + 8 * ci, pw);       // keys 16 c .. 16 c + 31 of the tile
       }
-      if (!s_freed) {                                     // a warp whose blocks lie past the end of the context
-        tc_fence_before();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&bar_sfree[team]);
-      }
-      fence_proxy_async();
+      tmem_st_wait();                                      // the probabilities (and a rescaled accumulator) are in place
+      tc_fence_before();
       mbar_arrive(&bar_pfull[team]);
       PF_TRACE(tr_pass_b);
 #ifdef COOPT_TRACE
@@ -610,10 +616,10 @@ __global__ void __launch_bounds__(kPuThreads, 1) paged_prefill_umma_kernel(const
       bad = !__all_sync(0xffffffffu, ok);
     }
     bad = barrier_or(1 + team, kPuTeam, bad);
-    // what the other team needs of this one, in this team's own (now idle) P operand: per row its reference and
+    // what the other team needs of this one, in this team's own (now idle) V operand: per row its reference and
     // the two halves' sums, and the team's reference scale
-    float* mine = reinterpret_cast<float*>(pbuf + team * C::kOperand16);
-    const float* theirs = reinterpret_cast<const float*>(pbuf + (team ^ 1) * C::kOperand16);
+    float* mine = reinterpret_cast<float*>(v16buf + team * 2 * C::kOperand16);
+    const float* theirs = reinterpret_cast<const float*>(v16buf + (team ^ 1) * 2 * C::kOperand16);
     mine[half * kPuRows + r] = l_row;
     if (half == 0) mine[2 * kPuRows + r] = m_ref;
     if (tid == team * kPuTeam) mine[3 * kPuRows] = v_ref;

@@ -33,6 +33,12 @@ __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a, uint64_t b
   asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
                ::"r"(d_tmem), "l"(a), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
 }
+// The same with the A operand in tensor memory: row m of A is lane m, its 16 f16 elements along the contraction are
+// the halves of 8 consecutive 32-bit columns from `a_tmem` on (element 2 j in the low half of column j).
+__device__ __forceinline__ void umma_f16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+               ::"r"(d_tmem), "r"(a_tmem), "l"(b), "r"(idesc), "r"(accumulate) : "memory");
+}
 // One commit per group of instructions: a second commit with no instruction in between was seen to
 // arrive before the group had finished, so every consumer of a group waits on the same mbarrier.
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {

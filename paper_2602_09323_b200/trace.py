@@ -137,11 +137,11 @@ def main():
 
 
 PREFILL_PHASES = (
-    (1, "team: waits for the tile's V part, scales and logits"), (2, "team: first pass (maximum of the thread's half row)"),
-    (3, "team: waits for its previous P V product, halves meet"), (7, "team: references, rescale, V widened to f16"),
-    (4, "team: second pass (probabilities)"),
+    (1, "team: waits for the tile's V part and scales"), (7, "team: V widened to f16"),
+    (3, "team: waits for the tile's logits"), (2, "team: first pass (maximum of the thread's half row), halves meet"),
+    (4, "team: references, rescale, second pass (probabilities to tensor memory)"),
     (13, "team: first thread done -> whole team arrived"), (5, "team: whole loop"),
-    (8, "logits lane: waits for the K tile"), (9, "logits lane: waits for the team to free the logits buffer"),
+    (8, "logits lane: waits for the K tile"), (9, "logits lane: waits for the team's previous P V product"),
     (10, "P V lane: waits for the probabilities"), (11, "P V lane: issues 8 instructions + commit"),
     (12, "P V lane: commit -> completion"))
 
