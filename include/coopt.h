@@ -274,10 +274,13 @@ int coopt_decode_layers(const coopt_layer_io* layers, int32_t num_layers, int64_
 
 /*
  * coopt_decode_step_host -- one serving step for callers whose step inputs live in HOST memory (Section 2's
- * token-insertion phase followed by the attention phase): ONE copy brings the step's inputs to the device,
- * coopt_decode_plan and coopt_decode_step_planned run on them, ONE copy takes the bf16 result back.
- * Everything is enqueued on `stream`; the host buffers must stay valid (and should be pinned) until the
- * stream has been synchronised.
+ * token-insertion phase followed by the attention phase).  If both host buffers are page-locked and mapped
+ * (cudaHostAlloc, cudaHostRegister; 16-byte aligned), the kernel reads the queries and the new tokens from
+ * them and stores the bf16 result into them directly, and only the index arrays (slots, block table, context
+ * lengths) are copied to the device for coopt_decode_plan.  Otherwise ONE copy brings the step's inputs to the
+ * device, the plan and the step run on them, and ONE copy takes the result back.  Results are identical either
+ * way.  Everything is enqueued on `stream`; the host buffers must stay valid until the stream has been
+ * synchronised, and out_host holds the result only then.
  *   step_inputs_host   HOST, coopt_step_layout.in_bytes bytes: the step's inputs packed at the offsets that
  *                      coopt_step_staging_layout() gives -- q bf16 [batch][num_q_heads][head_dim]; k_new,
  *                      v_new bf16 [batch][num_kv_heads][head_dim]; slot_mapping int64 [batch]; block_table

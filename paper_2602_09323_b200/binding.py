@@ -361,8 +361,9 @@ def step_staging_layout(batch: int, num_q_heads: int, num_kv_heads: int, head_di
 
 def decode_step_host(cache: Cache, step_inputs: torch.Tensor, out: torch.Tensor, max_blocks_per_seq: int, num_q_heads: int,
                      sm_scale: float, staging: torch.Tensor, plan: torch.Tensor, workspace: torch.Tensor) -> None:
-    """coopt_decode_step_host: ``step_inputs`` (uint8, packed per step_staging_layout) and ``out`` are HOST (pinned)
-    tensors; asynchronous."""
+    """coopt_decode_step_host: ``step_inputs`` (uint8, packed per step_staging_layout) and ``out`` are HOST tensors
+    (page-locked ones are read and written in place by the kernel, pageable ones go through copies); asynchronous:
+    ``out`` holds the result once the stream has been synchronised."""
     assert not step_inputs.is_cuda and step_inputs.is_contiguous() and not out.is_cuda and out.is_contiguous()
     st = load_library().coopt_decode_step_host(cache.ref(), _ptr(step_inputs), _ptr(out), max_blocks_per_seq, out.shape[0],
                                                num_q_heads, float(sm_scale), _ptr(staging), staging.numel(), _ptr(plan),

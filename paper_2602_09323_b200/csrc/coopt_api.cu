@@ -339,6 +339,18 @@ int coopt_paged_chunked(const coopt_cache* cache, const void* q, void* out, cons
 }
 
 namespace {
+// The device's address of a host pointer if the memory is page-locked and mapped (cudaHostAlloc, cudaHostRegister),
+// null for pageable memory (and for anything that is not host memory).
+const uint8_t* mapped_host_pointer(const void* host) {
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, host) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return nullptr;
+  }
+  if (attr.type != cudaMemoryTypeHost || attr.devicePointer == nullptr) return nullptr;
+  return static_cast<const uint8_t*>(attr.devicePointer);
+}
+
 coopt_step_layout step_layout(int batch, int hq, int hkv, int d, int max_blocks) {
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
   coopt_step_layout s;
@@ -385,9 +397,25 @@ int coopt_decode_step_host(const coopt_cache* cache, const void* step_inputs_hos
   if (rc != COOPT_OK) return rc;
   if (!workspace || workspace_bytes < coopt_workspace_bytes(batch, num_q_heads, hkv, d, max_blocks_per_seq, 0, batch)) return COOPT_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // one copy in, the plan and the fused step, one copy out
-  if (cudaMemcpyAsync(dev, step_inputs_host, s.in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return COOPT_ERR_CUDA;
   const int P = planned_ctas(batch, hkv, max_blocks_per_seq);
+  // Host buffers that are page-locked and mapped into the device's address space are used where they are: the
+  // kernel fetches the queries and the new tokens from them and stores the result into them, and only the
+  // index arrays (slots, block table, context lengths: what the planner walks) are copied to the device.
+  const uint8_t* in_dev = mapped_host_pointer(step_inputs_host);
+  uint8_t* out_dev = const_cast<uint8_t*>(mapped_host_pointer(out_host));
+  if (in_dev != nullptr && out_dev != nullptr && reinterpret_cast<uintptr_t>(in_dev) % 16 == 0 && reinterpret_cast<uintptr_t>(out_dev) % 16 == 0) {
+    if (cudaMemcpyAsync(dev + s.slot_mapping, static_cast<const uint8_t*>(step_inputs_host) + s.slot_mapping, s.in_bytes - s.slot_mapping,
+                        cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return COOPT_ERR_CUDA;
+    rc = launch_decode_plan(reinterpret_cast<const int32_t*>(dev + s.block_table), max_blocks_per_seq,
+                            reinterpret_cast<const int32_t*>(dev + s.context_lens), batch, hkv, cache->num_blocks, 0, P, plan, st);
+    if (rc != COOPT_OK) return rc;
+    return launch_decode_planned(cache, plan, in_dev + s.k_new, in_dev + s.v_new, static_cast<int64_t>(hkv) * d,
+                                 reinterpret_cast<const int64_t*>(dev + s.slot_mapping), in_dev + s.q, out_dev, max_blocks_per_seq,
+                                 batch, num_q_heads, sm_scale, 0, nullptr, workspace, P, false, st);
+  }
+  // pageable host memory: one copy in, the plan and the fused step, one copy out
+  if (cudaMemcpyAsync(dev, step_inputs_host, s.in_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return COOPT_ERR_CUDA;
   rc = launch_decode_plan(reinterpret_cast<const int32_t*>(dev + s.block_table), max_blocks_per_seq,
                           reinterpret_cast<const int32_t*>(dev + s.context_lens), batch, hkv, cache->num_blocks, 0, P, plan, st);
   if (rc != COOPT_OK) return rc;

@@ -170,3 +170,41 @@ def test_a_plan_of_another_problem_and_a_misplaced_slot_are_reported():
     binding.decode_step_planned(cache, plan, w.q.cuda(), table.shape[1], w.sm_scale, ws, k_new, v_new, s_bad.cuda())
     torch.cuda.synchronize()
     assert binding.workspace_status(ws) == -1
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_host_step_equals_the_planned_step_bit_for_bit(pinned):
+    """coopt_decode_step_host with page-locked buffers (queries and new tokens read in place, result stored in
+    place) and with pageable ones (staged through copies): cache bytes and outputs identical to coopt_decode_plan +
+    coopt_decode_step_planned on device tensors, and within tolerance of the oracle."""
+    hq, hkv, d = 10, 2, 128
+    w = workloads.make_workload("host_step", [300, 64, 2048, 1500, 47, 900, 17, 1], hq, hkv, d, seed=23)
+    hist = np.concatenate([np.arange(w.kv_offsets[b], w.kv_offsets[b] + L - 1) for b, L in enumerate(w.context_lens)])
+    new = torch.tensor([w.kv_offsets[b] + L - 1 for b, L in enumerate(w.context_lens)])
+    k_new, v_new, s_new = w.k[new].contiguous(), w.v[new].contiguous(), w.slot_mapping[new].contiguous()
+    table = w.block_table.clamp(min=0)
+    max_blocks = table.shape[1]
+    lay = binding.step_staging_layout(w.batch, hq, hkv, d, max_blocks)
+    host_in = torch.zeros(lay.in_bytes, dtype=torch.uint8)
+    for off, t in ((lay.q, w.q), (lay.k_new, k_new), (lay.v_new, v_new), (lay.slot_mapping, s_new), (lay.block_table, table),
+                   (lay.context_lens, w.context_lens_tensor)):
+        raw = t.contiguous().view(torch.uint8).reshape(-1)
+        host_in[off:off + raw.numel()] = raw
+    host_out = torch.full_like(w.q, float("nan"))
+    if pinned:
+        host_in, host_out = host_in.pin_memory(), host_out.pin_memory()
+    staging = torch.empty(lay.total_bytes, dtype=torch.uint8, device="cuda")
+    plan = torch.empty(binding.plan_bytes(w.batch, hkv, max_blocks), dtype=torch.uint8, device="cuda")
+    ws = binding.new_workspace(w.batch, hq, hkv, d, max_blocks)
+    cache_a, cache_b = helpers.gpu_fill(w, calls=[hist]), helpers.gpu_fill(w, calls=[hist])
+    binding.decode_step_host(cache_a, host_in, host_out, max_blocks, hq, w.sm_scale, staging, plan, ws)
+    torch.cuda.synchronize()
+    assert binding.workspace_status(ws) == 0
+    plan_b = binding.decode_plan(table.cuda(), w.context_lens_tensor.cuda(), hkv, w.num_blocks)
+    want = binding.decode_step_planned(cache_b, plan_b, w.q.cuda(), max_blocks, w.sm_scale, ws, k_new.cuda(), v_new.cuda(), s_new.cuda())
+    torch.cuda.synchronize()
+    assert torch.equal(cache_a.data, cache_b.data)
+    assert torch.equal(host_out.cuda(), want)
+    codes, scales = helpers.oracle_fp8_cache(w, calls=[hist, new.numpy()])
+    ref = attention.paged_attention(w.q.float().numpy(), (codes, scales), w.block_table.numpy(), w.context_lens)
+    helpers.check_attention(host_out, ref, what=f"host step, {'page-locked' if pinned else 'pageable'} buffers")
