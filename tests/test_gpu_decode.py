@@ -124,7 +124,7 @@ def _pairs_of_heads(batch, group, kv_heads):
 
 
 def test_llama13b_decode_full_size_every_output():
-    """BASELINE configuration 2 at full size, in the launch configuration the benchmark times: the whole
+    """The LLaMA-13B-shaped decode configuration at full size, in the launch configuration the benchmark times: the whole
     device cache against the oracle's bit for bit, and every (sequence, query head) output."""
     w = workloads.config_llama13b_decode()
     cache = helpers.gpu_fill(w)
@@ -148,7 +148,7 @@ def test_llama13b_decode_full_size_without_v_outliers_meets_the_plain_bound():
 
 
 def test_llama13b_mha_ablation_full_size_every_output():
-    """BASELINE configuration 2's ablation at full size: 40 KV heads (one per query head) and a bf16 cache.
+    """The ablation of the LLaMA-13B-shaped decode configuration at full size: 40 KV heads (one per query head) and a bf16 cache.
     The oracle's un-quantised write and float64 attention, eight heads at a time to bound host memory."""
     w = workloads.config_llama13b_mha_ablation()
     cache = helpers.gpu_fill(w, dtype=binding.KV_BF16)
@@ -248,7 +248,7 @@ def _serving_step_calls(w):
 
 @pytest.mark.parametrize("plain", [False, True])
 def test_mixed_length_serving_step_full_size_every_output(plain):
-    """BASELINE configuration 3 at full size: 64 sequences with contexts uniform in [128, 8192]; the history is
+    """The mixed-length serving configuration at full size: 64 sequences with contexts uniform in [128, 8192]; the history is
     filled in bulk, then one token per sequence is appended with coopt_kv_write (which may grow a block's
     scale and re-express its resident codes) and the decode runs over the updated cache.  The oracle replays
     the same two writes; the whole cache is compared bit for bit and every output within the tolerance
@@ -268,7 +268,7 @@ def test_mixed_length_serving_step_full_size_every_output(plain):
 
 @pytest.mark.parametrize("plain", [False, True])
 def test_long_context_chunked_full_size_every_output(plain):
-    """BASELINE configuration 4 at full size: contexts of 32768 .. 131072 tokens, chunk size 2048; every
+    """The long-context configuration at full size: contexts of 32768 .. 131072 tokens, chunk size 2048; every
     per-chunk (m, l, o) and every merged output against the oracle's chunk-and-merge path."""
     w = workloads.config_long_context(v_outliers=not plain)
     heads = PLAIN_HEADS if plain else None

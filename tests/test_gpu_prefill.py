@@ -67,7 +67,7 @@ def test_causal_row_equals_decode_over_the_truncated_context():
 
 @pytest.mark.parametrize("plain", [False, True])
 def test_chunked_prefill_full_size(plain):
-    """BASELINE configuration 5 at full size: 8 sequences, 4096 cached + 512 new tokens, causal.  The whole
+    """The chunked-prefill configuration at full size: 8 sequences, 4096 cached + 512 new tokens, causal.  The whole
     device cache against the oracle's bit for bit; every query row and head of one (sequence, kv head) group,
     and for every sequence and kv head the rows on both sides of every boundary between the kernel's tiles of
     25 query tokens (plus the first and the last row), for one query head of the group."""
