@@ -102,6 +102,14 @@ class ClockSampler(threading.Thread):
                 pass
             time.sleep(self.period)
 
+    def sample_now(self):
+        """One sample taken by the caller itself (a timed region shorter than the sampling thread's start-up)."""
+        if self.ok:
+            try:
+                self.samples.append(self.nv.nvmlDeviceGetClockInfo(self.h, self.nv.NVML_CLOCK_SM))
+            except Exception:
+                pass
+
     def summary(self):
         if not self.ok or not self.samples:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
@@ -387,7 +395,7 @@ def main():
 
     # ---- synthetic workload: NL layer caches with one block table (a model's layers share it), a history of
     # 2047 tokens per sequence; every step appends token 2048 of one layer and attends over that layer's cache
-    NL = args.layers
+    NL = max(2, min(args.layers, args.steps))         # a short run passes over as many layer caches as it has steps
     base = workloads.config_llama13b_decode(seed=rank, batch=BATCH, context=CONTEXT)
     k_dev, v_dev = base.k.cuda(), base.v.cuda()
     hist = torch.ones(BATCH * CONTEXT, dtype=torch.bool)
@@ -468,6 +476,7 @@ def main():
     start.record()
     run_steps(args.steps)
     stop.record()
+    sampler.sample_now()                           # the steps are enqueued and still running
     torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
@@ -518,7 +527,7 @@ def main():
         put(lay.q, base.q); put(lay.k_new, k_new.cpu()); put(lay.v_new, v_new.cpu()); put(lay.slot_mapping, s_new.cpu())
         put(lay.block_table, base.block_table.clamp(min=0)); put(lay.context_lens, base.context_lens_tensor)
         host_out = torch.empty_like(base.q).pin_memory()
-        n_e2e = max(1, min(args.steps, 2000))
+        n_e2e = max(200, min(args.steps, 2000))                         # (its own step count, stated in the e2e object)
 
         def host_step(i):
             binding.decode_step_host(caches[i % NL], host_in, host_out, max_blocks, HQ, base.sm_scale, staging, plan, ws)
