@@ -361,6 +361,7 @@ __global__ void __launch_bounds__(kUmmaThreads, 1) paged_decode_umma_kernel(cons
           }
           ok = __shfl_sync(0xffffffffu, ok, 0);
           if (!ok) break;
+          COOPT_TRACE_CYCLES(p.trace, kTrFirstCopyReady, lane == 0 && tile_no == 0);
           if (lane < 3 * ngroups) gather4_g2s(st + dst_off, map, x, rows[0], rows[1], rows[2], rows[3], &bar_full[stage]);
           COOPT_TRACE_CYCLES(p.trace, kTrFirstCopy, lane == 0 && tile_no == 0);
           COOPT_TRACE_CYCLES(p.trace, kTrLastCopy, lane == 0);

@@ -32,6 +32,7 @@ enum TraceSlot {
   kTrSmId,             // the SM the CTA ran on
   kTrProducerPlan,     // the copy warp has seen the plan
   kTrPrevExitNs,       // what kTrExitNs held at entry: the exit of this CTA's slot in the launch before
+  kTrFirstCopyReady,   // the copy warp is about to request the first tile (rows worked out, byte count posted)
   kTrSegBase = 24,     // 24 + i: epilogue warp received segment i (i < 20)
   kTrTeamSegBase = 44, // 44 + i: team 0 began segment i (i < 20)
   kTrCopyTileBase = 64,    // 64 + i: tile i requested (i < 32)

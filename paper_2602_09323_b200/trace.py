@@ -22,7 +22,7 @@ SLOTS = 256
 MAX_CTAS = 1024
 NAMES = ["entry", "entry_ns", "setup_done", "plan_in_smem", "first_copy", "first_landed", "first_probs", "last_copy",
          "last_landed", "last_pv", "teams_done", "last_hand_off", "piece_stored", "counted", "epilogue_done", "exit",
-         "exit_ns", "write_done", "num_seg", "num_tiles", "sm_id", "producer_plan", "prev_exit_ns"]
+         "exit_ns", "write_done", "num_seg", "num_tiles", "sm_id", "producer_plan", "prev_exit_ns", "first_copy_ready"]
 SEG_BASE, TEAM_SEG_BASE = 24, 44
 
 
