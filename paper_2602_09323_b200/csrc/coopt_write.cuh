@@ -179,11 +179,14 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
 #pragma unroll
     for (int c = 0; c < kPart / 512; ++c) st4[c * 32 + lane] = resident[c];
   }
-  float amax = 0.0f;
+  // The largest magnitude, on the packed pairs: magnitudes of bf16 values order like their 15-bit patterns, and
+  // the rows past the group's size repeat its last row, so no row has to be left out.
+  uint32_t amax2 = 0;
 #pragma unroll
   for (int t = 0; t < kTok; ++t)
 #pragma unroll
-    for (int e = 0; e < kPerLane; ++e) amax = fmaxf(amax, t < n ? fabsf(row_elem(raw[t], e)) : 0.0f);
+    for (int e = 0; e < kPerLane / 2; ++e) amax2 = __vmaxu2(amax2, raw[t][e] & 0x7FFF7FFFu);
+  float amax = __uint_as_float(max(amax2 << 16, amax2 & 0xFFFF0000u));
   amax = warp_max(amax);
   const float s_new = fmaxf(s_old, __fdiv_rn(amax, kE5m2 ? kE5m2Max : kE4m3Max));
   __syncwarp();
