@@ -168,7 +168,13 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
     resident[c] = (fresh || full) ? make_uint4(0, 0, 0, 0) : reinterpret_cast<const uint4*>(part)[c * 32 + lane];
   uint32_t raw[kTok][kPerLane / 2];
   const __nv_bfloat16* rows = src + h * D + lane * kPerLane;
-  if (vec) {
+  // a whole block of tokens that follow one another in the call (a bulk fill): no look-up of the rows
+  const bool in_a_row = kTok > 1 && n == kTok && g.tok[kTok - 1] - g.tok[0] == kTok - 1;
+  if (vec && in_a_row) {
+    const __nv_bfloat16* r0 = rows + static_cast<int64_t>(g.tok[0]) * p.token_stride;
+#pragma unroll
+    for (int t = 0; t < kTok; ++t) load_row<kPerLane, true>(r0 + t * p.token_stride, raw[t]);
+  } else if (vec) {
 #pragma unroll
     for (int t = 0; t < kTok; ++t) load_row<kPerLane, true>(rows + static_cast<int64_t>(g.tok[min(t, n - 1)]) * p.token_stride, raw[t]);
   } else {
@@ -213,12 +219,17 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
     const float q0 = __fmul_rn(xv, rcp);
     return copysignf(__fmaf_rn(__fmaf_rn(-s_new, q0, xv), rcp, q0), xv);     // a zero keeps the sign of x
   };
+  auto by_reciprocal_magnitude = [&](int t, int e) -> float {                // the same without the sign of a zero
+    const float xv = row_elem(raw[t], e);
+    const float q0 = __fmul_rn(xv, rcp);
+    return __fmaf_rn(__fmaf_rn(-s_new, q0, xv), rcp, q0);
+  };
   auto by_division = [&](int t, int e) -> float {
     const float xv = row_elem(raw[t], e);
     return s_new > 0.0f ? __fdiv_rn(xv, s_new) : xv;
   };
 
-  auto encode = [&](auto scaled) {
+  auto encode = [&](auto scaled, auto scaled_k, bool k_signs_from_x) {
     if (kTok == kBlockSize && full && which == 1) {
       // V of a whole block: the 16 tokens of one dim are 16 consecutive bytes of the part
 #pragma unroll
@@ -239,9 +250,13 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
           if (which == 0) {
             // the lane's dims are consecutive bytes of a K row
             uint8_t* dst = st + k_elem_offset(D, true, off, lane * kPerLane);
-            if constexpr (kPerLane == 4)
-              *reinterpret_cast<uint32_t*>(dst) = f32x2_to_codes<kE5m2>(scaled(t, 0), scaled(t, 1)) | (f32x2_to_codes<kE5m2>(scaled(t, 2), scaled(t, 3)) << 16);
-            else
+            if constexpr (kPerLane == 4) {
+              // four codes of one token; the signs (which a zero quotient may have lost) are those of the four
+              // values themselves: the top bits of the upper bytes of the packed pairs, gathered in one go
+              uint32_t word = f32x2_to_codes<kE5m2>(scaled_k(t, 0), scaled_k(t, 1)) | (f32x2_to_codes<kE5m2>(scaled_k(t, 2), scaled_k(t, 3)) << 16);
+              if (k_signs_from_x) word |= __byte_perm(raw[t][0], raw[t][1], 0x7531) & 0x80808080u;
+              *reinterpret_cast<uint32_t*>(dst) = word;
+            } else
               *reinterpret_cast<uint16_t*>(dst) = static_cast<uint16_t>(f32x2_to_codes<kE5m2>(scaled(t, 0), scaled(t, 1)));
           } else {
 #pragma unroll
@@ -256,7 +271,7 @@ __device__ __forceinline__ void write_part(const WriteParams& p, const Group& g,
       for (int c = 0; c < kPart / 512; ++c) out4[c * 32 + lane] = st4[c * 32 + lane];
     }
   };
-  if (by_rcp) encode(by_reciprocal); else encode(by_division);
+  if (by_rcp) encode(by_reciprocal, by_reciprocal_magnitude, true); else encode(by_division, by_division, false);
   if (lane == 0) scales[which] = s_new;
   if (which == 0 && fresh && lane < 6) scales[2 + lane] = 0.0f;       // rest of the header
   __syncwarp();
